@@ -1,0 +1,305 @@
+/*
+ * dq_oracle.c -- plain CPU oracle of the DQ-SGD quantizer hot path.
+ * TEST INFRASTRUCTURE ONLY; see dq_oracle.h.  Build with
+ *   gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC
+ * (-ffp-contract=off: every fp32 operation below rounds on its own, in the
+ * order written; that order is part of the definition of the codes).
+ */
+#include "dq_oracle.h"
+
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+static int32_t g_threads = 1;
+
+void oracle_set_threads(int32_t n) { g_threads = n < 1 ? 1 : n; }
+int32_t oracle_get_threads(void) { return g_threads; }
+
+static int64_t roundup32(int64_t n) { return (n + 31) / 32 * 32; }
+
+/* ------------------------------------------------------------------ layout */
+
+int64_t oracle_padded_elems(const int64_t* seg_elems, int32_t n_seg)
+{
+    int64_t total = 0;
+    for (int32_t i = 0; i < n_seg; ++i) total += roundup32(seg_elems[i]);
+    return total;
+}
+
+int64_t oracle_num_buckets(const int64_t* seg_elems, int32_t n_seg, int32_t bucket)
+{
+    int64_t nb = 0;
+    for (int32_t i = 0; i < n_seg; ++i) nb += (seg_elems[i] + bucket - 1) / bucket;
+    return nb;
+}
+
+void oracle_seg_offsets(const int64_t* seg_elems, int32_t n_seg, int64_t* offsets)
+{
+    int64_t p = 0;
+    for (int32_t i = 0; i < n_seg; ++i) {
+        offsets[i] = p;
+        p += roundup32(seg_elems[i]);
+    }
+}
+
+void oracle_bucket_table(const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                         int64_t* start, int64_t* len)
+{
+    int64_t p = 0, k = 0;
+    for (int32_t i = 0; i < n_seg; ++i) {
+        const int64_t n = seg_elems[i];
+        for (int64_t o = 0; o < n; o += bucket) {
+            start[k] = p + o;
+            len[k] = (n - o < bucket) ? (n - o) : bucket;
+            ++k;
+        }
+        p += roundup32(n);
+    }
+}
+
+/* the table is small; build it once per call */
+typedef struct { int64_t nb; int64_t* start; int64_t* len; } table_t;
+
+static table_t make_table(const int64_t* seg_elems, int32_t n_seg, int32_t bucket)
+{
+    table_t t;
+    t.nb = oracle_num_buckets(seg_elems, n_seg, bucket);
+    t.start = (int64_t*)malloc(sizeof(int64_t) * (size_t)(t.nb > 0 ? t.nb : 1));
+    t.len = (int64_t*)malloc(sizeof(int64_t) * (size_t)(t.nb > 0 ? t.nb : 1));
+    oracle_bucket_table(seg_elems, n_seg, bucket, t.start, t.len);
+    return t;
+}
+
+static void free_table(table_t* t) { free(t->start); free(t->len); }
+
+/* ------------------------------------------------------------------- norms */
+
+void oracle_bucket_norms(const float* grads, int64_t worker_stride, int32_t M,
+                         const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                         float* norms)
+{
+    table_t tb = make_table(seg_elems, n_seg, bucket);
+    const int64_t total = (int64_t)M * tb.nb;
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int64_t w = 0; w < total; ++w) {
+        const int64_t m = w / tb.nb, k = w % tb.nb;
+        const float* g = grads + m * worker_stride + tb.start[k];
+        double ss = 0.0;
+        for (int64_t j = 0; j < tb.len[k]; ++j) ss += (double)g[j] * (double)g[j];
+        norms[w] = (float)sqrt(ss);
+    }
+    free_table(&tb);
+}
+
+/* ---------------------------------------------------------------- bit rule */
+
+int32_t oracle_choose_bits(const float* norms, int64_t nb, int32_t M,
+                           int32_t T, int32_t t, double eps_hat, double alpha,
+                           int32_t b_min, int32_t b_max, int32_t fixed_b,
+                           int32_t* s_out, double* x_out)
+{
+    /* G-bar^2 = (1/W) sum_i ||g^(i)||^2 ; with p = 2 the squared norm of a
+     * worker's vector is the sum of its squared bucket norms. */
+    double sum = 0.0;
+    for (int64_t i = 0; i < (int64_t)M * nb; ++i) sum += (double)norms[i] * (double)norms[i];
+    const double G2 = sum / (double)M;
+    /* Eq. 17: b = log2(x + 1) + 1 with x as below */
+    const double x = sqrt((double)T / eps_hat) * pow(alpha, (double)(T - 1 - t) / 2.0) * sqrt(G2);
+    if (x_out) *x_out = x;
+    int32_t b;
+    if (fixed_b != 0) {
+        b = fixed_b;
+    } else {
+        /* smallest integer b in [b_min, b_max] with 2^(b-1) - 1 >= x,
+         * i.e. ceil(log2(x + 1)) + 1 without a transcendental */
+        b = b_max;
+        for (int32_t c = b_min; c <= b_max; ++c) {
+            if ((double)((1 << (c - 1)) - 1) >= x) { b = c; break; }
+        }
+    }
+    if (s_out) *s_out = (1 << (b - 1)) - 1;
+    return b;
+}
+
+/* ------------------------------------------------------------------ Philox */
+
+static void mulhilo(uint32_t a, uint32_t b, uint32_t* hi, uint32_t* lo)
+{
+    const uint64_t p = (uint64_t)a * (uint64_t)b;
+    *hi = (uint32_t)(p >> 32);
+    *lo = (uint32_t)p;
+}
+
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+    uint32_t k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0, lo0, hi1, lo1;
+        mulhilo(0xD2511F53u, c0, &hi0, &lo0);
+        mulhilo(0xCD9E8D57u, c2, &hi1, &lo1);
+        const uint32_t n0 = hi1 ^ c1 ^ k0;
+        const uint32_t n1 = lo1;
+        const uint32_t n2 = hi0 ^ c3 ^ k1;
+        const uint32_t n3 = lo0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u;   /* golden-ratio Weyl increments of the key */
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* uniform in [0,1) with 24 bits, for padded element index j of worker m */
+static float uniform24(uint64_t seed, uint32_t step, uint32_t m, int64_t j)
+{
+    const uint64_t q = (uint64_t)j >> 2;
+    const uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), m, step };
+    const uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
+    uint32_t r[4];
+    oracle_philox4x32_10(ctr, key, r);
+    return (float)(r[j & 3] >> 8) * 0x1p-24f;
+}
+
+/* ---------------------------------------------------------------- quantize */
+
+/* Norms below this are treated as zero: s / norm would overflow fp32. */
+#define ORACLE_TINY_NORM 0x1p-100f
+
+void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
+                     const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                     const float* norms, int32_t b, uint64_t seed, uint32_t step,
+                     uint32_t* codes, float* frac_out, float* u_out)
+{
+    table_t tb = make_table(seg_elems, n_seg, bucket);
+    const int64_t D32 = oracle_padded_elems(seg_elems, n_seg);
+    const int32_t s = (1 << (b - 1)) - 1;
+    const float sf = (float)s;
+
+    memset(codes, 0, sizeof(uint32_t) * (size_t)((int64_t)M * D32));   /* pads: code 0 */
+    if (frac_out) memset(frac_out, 0, sizeof(float) * (size_t)((int64_t)M * D32));
+    if (u_out) memset(u_out, 0, sizeof(float) * (size_t)((int64_t)M * D32));
+
+    const int64_t total = (int64_t)M * tb.nb;
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int64_t w = 0; w < total; ++w) {
+        const int64_t m = w / tb.nb, k = w % tb.nb;
+        const float norm = norms[w];
+        const float inv = (norm >= ORACLE_TINY_NORM) ? sf / norm : 0.0f;
+        for (int64_t e = 0; e < tb.len[k]; ++e) {
+            const int64_t j = tb.start[k] + e;
+            const float g = grads[m * worker_stride + j];
+            const float a = fabsf(g);
+            float r = a * inv;               /* s * |g_j| / ||g||  (Eq. 6) */
+            r = fminf(r, sf);                /* an ulp above s must not carry into the sign */
+            const float l = floorf(r);
+            const float f = r - l;           /* p_r of Eq. 6, exact in fp32 */
+            const float u = uniform24(seed, step, (uint32_t)m, j);
+            const uint32_t level = (uint32_t)l + (u < f ? 1u : 0u);
+            uint32_t gbits;
+            memcpy(&gbits, &g, sizeof gbits);
+            const uint32_t sign = gbits >> 31;
+            codes[m * D32 + j] = (sign << (b - 1)) | level;
+            if (frac_out) frac_out[m * D32 + j] = f;
+            if (u_out) u_out[m * D32 + j] = u;
+        }
+    }
+    free_table(&tb);
+}
+
+/* ------------------------------------------------------------- pack/unpack */
+
+void oracle_pack(const uint32_t* codes, int64_t n, int32_t b, uint32_t* words)
+{
+    const int64_t nwords = n / 32 * b;
+    memset(words, 0, sizeof(uint32_t) * (size_t)nwords);
+    /* element e of the stream owns bits [e*b, e*b + b) of the bit string
+     * whose bit i is bit (i % 32) of word (i / 32) */
+    for (int64_t e = 0; e < n; ++e) {
+        for (int32_t i = 0; i < b; ++i) {
+            const int64_t bit = e * b + i;
+            if ((codes[e] >> i) & 1u) words[bit >> 5] |= 1u << (bit & 31);
+        }
+    }
+}
+
+void oracle_unpack(const uint32_t* words, int64_t n, int32_t b, uint32_t* codes)
+{
+    for (int64_t e = 0; e < n; ++e) {
+        uint32_t c = 0;
+        for (int32_t i = 0; i < b; ++i) {
+            const int64_t bit = e * b + i;
+            c |= ((words[bit >> 5] >> (bit & 31)) & 1u) << i;
+        }
+        codes[e] = c;
+    }
+}
+
+void oracle_quantize_pack(const float* grads, int64_t worker_stride, int32_t M,
+                          const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                          const float* norms, int32_t b, uint64_t seed, uint32_t step,
+                          uint32_t* packed, int64_t packed_stride)
+{
+    const int64_t D32 = oracle_padded_elems(seg_elems, n_seg);
+    uint32_t* codes = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)((int64_t)M * D32 + 1));
+    oracle_quantize(grads, worker_stride, M, seg_elems, n_seg, bucket, norms, b, seed, step,
+                    codes, NULL, NULL);
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int32_t m = 0; m < M; ++m)
+        oracle_pack(codes + (int64_t)m * D32, D32, b, packed + (int64_t)m * packed_stride);
+    free(codes);
+}
+
+/* -------------------------------------------------------------- dequantize */
+
+void oracle_dequantize(const uint32_t* codes, const float* norms,
+                       const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                       int32_t b, double* values)
+{
+    table_t tb = make_table(seg_elems, n_seg, bucket);
+    const int64_t D32 = oracle_padded_elems(seg_elems, n_seg);
+    const int32_t s = (1 << (b - 1)) - 1;
+    for (int64_t j = 0; j < D32; ++j) values[j] = 0.0;
+    for (int64_t k = 0; k < tb.nb; ++k) {
+        for (int64_t e = 0; e < tb.len[k]; ++e) {
+            const int64_t j = tb.start[k] + e;
+            const uint32_t c = codes[j];
+            const double sgn = ((c >> (b - 1)) & 1u) ? -1.0 : 1.0;
+            const double level = (double)(c & (uint32_t)s);
+            values[j] = (s > 0) ? sgn * level * (double)norms[k] / (double)s : 0.0;
+        }
+    }
+    free_table(&tb);
+}
+
+void oracle_unpack_dequant_average(const uint32_t* packed, int64_t packed_stride,
+                                   const float* norms, int32_t M, int32_t b,
+                                   const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                                   float* out)
+{
+    table_t tb = make_table(seg_elems, n_seg, bucket);
+    const int64_t D32 = oracle_padded_elems(seg_elems, n_seg);
+    const int32_t s = (1 << (b - 1)) - 1;
+    uint32_t* codes = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)((int64_t)M * D32 + 1));
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int32_t m = 0; m < M; ++m)
+        oracle_unpack(packed + (int64_t)m * packed_stride, D32, b, codes + (int64_t)m * D32);
+
+    for (int64_t j = 0; j < D32; ++j) out[j] = 0.0f;      /* pads: +0 */
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int64_t k = 0; k < tb.nb; ++k) {
+        for (int64_t e = 0; e < tb.len[k]; ++e) {
+            const int64_t j = tb.start[k] + e;
+            double acc = 0.0;
+            for (int32_t m = 0; m < M; ++m) {
+                const uint32_t c = codes[(int64_t)m * D32 + j];
+                const double sgn = ((c >> (b - 1)) & 1u) ? -1.0 : 1.0;
+                const double level = (double)(c & (uint32_t)s);
+                if (s > 0) acc += sgn * level * (double)norms[(int64_t)m * tb.nb + k] / (double)s;
+            }
+            out[j] = (float)(acc / (double)M);
+        }
+    }
+    free(codes);
+    free_table(&tb);
+}
