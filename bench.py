@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the DQ-SGD quantizer hot path on B200.
+
+One step = one communication round of Algorithm 1 on one batch of synthetic
+gradients: bucket norms -> bit rule -> quantize+pack -> unpack+dequantize+average,
+all through the C-ABI library.  The workload is the ResNet-18-shaped gradient
+(62 tensors, 11,173,962 fp32 per worker, M = 8 workers, bucket 512, Laplace
+values, dynamic b over T = 100 steps, norms shrinking by 0.98 per step).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line.  ``value`` is GB/s of fp32 gradient processed
+(4 * M * d bytes per step over the step time), inputs resident in HBM;
+``e2e`` is the same with pinned host buffers and the copies timed.
+``--impl reference`` times the CPU checker on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "quantize+pack and unpack+average GB/s of fp32 gradient"
+UNIT = "GB/s"
+WORKLOAD = "resnet18-cifar10 gradient, 62 tensors, d=11173962 fp32/worker, M=8, bucket=512, Laplace, dynamic b, T=100"
+SEED = 2107
+POOL_BYTES = 40 << 30          # device memory the pre-generated inputs may take
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+def _traffic(kernel_key: str):
+    """DRAM bytes per launch from the committed ncu capture, or None if the kernel
+    source changed since the capture."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    with open(path) as fh:
+        rec = json.load(fh).get(kernel_key)
+    if not rec:
+        return None
+    src = os.path.join(ROOT, rec["source"])
+    digest = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    if digest != rec["sha256"]:
+        return None
+    return rec
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.rows = []
+        self.proc = None
+        self.uuid = uuid
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, val in zip(names, r[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------
+# reference arm: the CPU checker, as it stands, on the host cores
+# --------------------------------------------------------------------------
+
+def _oracle_round(oracle, np, w, ref, g, t, eps_hat, alpha):
+    norms = oracle.bucket_norms(ref, g)
+    b, s, _ = oracle.choose_bits(norms, w.T, t, eps_hat, alpha)
+    packed = oracle.quantize_pack(ref, g, norms, b, SEED, t)
+    out = oracle.unpack_dequant_average(ref, packed, norms, b)
+    return b, out
+
+
+def run_reference(args) -> dict:
+    import numpy as np
+
+    import oracle
+    from paper_2107_14575_b200 import workloads
+    factor = 16
+    full = workloads.config_resnet18()
+    w = workloads.scaled_down(full, factor)
+    ref = oracle.Layout(w.segments, w.bucket)
+    cores = os.cpu_count() or 1
+    oracle.set_threads(cores)
+    pool = [workloads.make_grads(w, ref.offsets, ref.D32, step=t) for t in range(4)]
+    n0 = oracle.bucket_norms(ref, pool[0])
+    G2 = float((n0.astype(np.float64) ** 2).sum() / w.M)
+    alpha = full.alpha
+    eps_hat = full.T * alpha ** (full.T - 1) * G2 / full.x0 ** 2
+    for i in range(args.warmup):
+        _oracle_round(oracle, np, w, ref, pool[i % 4], i % full.T, eps_hat, alpha)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        _oracle_round(oracle, np, w, ref, pool[i % 4], i % full.T, eps_hat, alpha)
+    dt = time.perf_counter() - t0
+    gbs = 4.0 * w.M * w.d * args.steps / dt / 1e9
+    sample = "every tensor of the workload cut to 1/%d of its size (d=%d per worker), all M=8 workers" % (factor, w.d)
+    return {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+
+
+# --------------------------------------------------------------------------
+# CUDA arm
+# --------------------------------------------------------------------------
+
+def _gen_step(torch, gen, scale_vec, M, D32, step):
+    """Laplace(0, scale_l * 0.98^step) per tensor l, zero on padding; [M, D32] fp32 on the device."""
+    u = torch.rand((M, D32), generator=gen, device=scale_vec.device, dtype=torch.float32) - 0.5
+    g = -torch.sign(u) * torch.log1p(-2.0 * u.abs().clamp_(max=0.4999999))
+    g.mul_(scale_vec * (0.98 ** step))
+    return g
+
+
+def run_cuda(args) -> dict:
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2107_14575_b200 import dq, workloads
+    from paper_2107_14575_b200.pipeline import Round
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    w = workloads.config_resnet18()
+    rnd = Round(w.segments, w.bucket, w.M, device=str(dev))
+    L = rnd.layout
+    M, D32, T = w.M, L.D32, w.T
+    nseg = len(w.segments)
+
+    scale_vec = torch.zeros(D32, dtype=torch.float32, device=dev)
+    for i, n in enumerate(w.segments):
+        scale_vec[L.offsets[i]: L.offsets[i] + n] = 1e-2 * 10.0 ** (-i / (nseg - 1))
+
+    K, W = args.steps, args.warmup
+    step_bytes = 4 * M * D32
+    npool = max(2, min(K + W, POOL_BYTES // step_bytes))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(SEED + 1000 * rank)
+    # pool entry p is the input of every step i with i % npool == p; it carries the
+    # norm decay of schedule step t = p % T
+    pool = [_gen_step(torch, gen, scale_vec, M, D32, p % T) for p in range(npool)]
+
+    # calibrate eps_hat so that x(t = 0) = x0 (b = 4 at the start of the schedule)
+    rnd.norms_(pool[0])
+    G2 = float((rnd.norms.double() ** 2).sum().item() / M)
+    alpha = w.alpha
+    eps_hat = T * alpha ** (T - 1) * G2 / w.x0 ** 2
+
+    def rule_for(i):
+        return dq.Rule.dynamic(T, i % T, eps_hat, alpha)
+
+    # untimed pass: the b each step will choose (needed for the byte model); also warms up
+    bits = []
+    for i in range(K):
+        rnd.norms_(pool[i % npool])
+        rnd.bits_(rule_for(i))
+        bits.append(rnd.bits())
+    for i in range(max(W, 3)):
+        rnd.step(pool[i % npool], rule_for(i), SEED, i)
+    torch.cuda.synchronize()
+    assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
+
+    names = ["bucket_norms", "choose_bits", "quantize_pack", "unpack_dequant_average"]
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(K)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", ""))
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record()
+    for i in range(K):
+        g = pool[i % npool]
+        rule = rule_for(i)
+        e = ev[i]
+        e[0].record()
+        rnd.norms_(g)
+        e[1].record()
+        rnd.bits_(rule)
+        e[2].record()
+        rnd.quantize_(g, SEED, i)
+        e[3].record()
+        rnd.average_()
+        e[4].record()
+    end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = start.elapsed_time(end)
+    assert rnd.read_status() == 0
+    if world > 1:
+        tmax = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+
+    per_kernel_ms = {n: [ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)] for j, n in enumerate(names)}
+    totals = {n: sum(v) for n, v in per_kernel_ms.items()}
+    dominant = max(totals, key=totals.get)
+    elems = M * D32
+    mean_b = sum(bits) / len(bits)
+    alg_bytes = {
+        "bucket_norms": 4.0 * elems,
+        "choose_bits": 4.0 * M * L.nb,
+        "quantize_pack": (4.0 + mean_b / 8.0) * elems,
+        "unpack_dequant_average": (M * mean_b / 8.0 + 4.0) * D32,
+    }
+    peak, peak_src = _peaks()
+    kernels = {}
+    for n in names:
+        avg_ms = totals[n] / K
+        gbs = alg_bytes[n] / (avg_ms * 1e-3) / 1e9
+        kernels[n] = {"avg_ms": round(avg_ms, 5), "achieved_gbs": round(gbs, 1), "frac": round(gbs / peak, 4),
+                      "share": round(totals[n] / sum(totals.values()), 4)}
+    tr = _traffic(dominant)
+    roofline = {
+        "kernel": dominant, "bound": "hbm", "achieved": kernels[dominant]["achieved_gbs"], "peak": peak,
+        "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": (tr or {}).get("bytes_per_launch"),
+        "peak_source": peak_src + "; of measured" if peak_src.startswith("measured") else peak_src + "; of fallback",
+        "algorithmic_bytes_per_launch": alg_bytes[dominant], "mean_b": round(mean_b, 3),
+        "kernels": kernels,
+    }
+
+    value = world * 4.0 * M * w.d * K / (ms * 1e-3) / 1e9
+
+    # ---- end to end: pinned host gradients in, averaged gradient out, copies timed ----
+    Ke = min(K, 10)
+    host = [pool[p].cpu().pin_memory() for p in range(2)]
+    for i in range(2):
+        rnd.step_host(host[i % 2], rule_for(i), SEED, i)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for i in range(Ke):
+        res = rnd.step_host(host[i % 2], rule_for(i), SEED, i)
+    e2.record()
+    torch.cuda.synchronize()
+    checksum = float(res[:1024].double().abs().sum())        # the result is read on the host
+    ms2 = s2.elapsed_time(e2)
+    if world > 1:
+        tmax = torch.tensor([ms2], dtype=torch.float64, device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms2 = float(tmax.item())
+    e2e = {"value": world * 4.0 * M * w.d * Ke / (ms2 * 1e-3) / 1e9, "unit": UNIT,
+           "h2d_bytes_per_step": 4 * M * D32, "d2h_bytes_per_step": 4 * D32, "steps": Ke,
+           "ms_per_step": ms2 / Ke, "checksum": checksum}
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "bits_first_last": [bits[0], bits[-1]], "mean_bits": round(mean_b, 3),
+                   "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
+                   "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * K, "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = _cpu_baseline(pool, w, eps_hat, alpha)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return out if rank == 0 else {}
+
+
+def _cpu_baseline(pool, w, eps_hat, alpha) -> dict:
+    """The CPU checker timed on one full step of the same workload (same arrays)."""
+    import numpy as np
+
+    import oracle
+    ref = oracle.Layout(w.segments, w.bucket)
+    cores = os.cpu_count() or 1
+    oracle.set_threads(cores)
+    g = pool[0].cpu().numpy()
+    t0 = time.perf_counter()
+    _oracle_round(oracle, np, w, ref, g, 0, eps_hat, alpha)
+    dt = time.perf_counter() - t0
+    return {"value": 4.0 * w.M * w.d / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "one full step (all 8 workers, all 62 tensors, t=0), %.1f s" % dt}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return
+        print(json.dumps(run_reference(args)))
+        return
+    out = run_cuda(args)
+    if out:
+        print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    main()

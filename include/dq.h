@@ -1,0 +1,173 @@
+/*
+ * dq.h -- C ABI of the DQ-SGD gradient quantizer hot path for NVIDIA B200 (sm_100a).
+ *
+ * Method: "DQ-SGD: Dynamic Quantization in SGD for Communication-Efficient
+ * Distributed Learning" (arXiv 2107.14575).  One training step of Algorithm 1
+ * maps to four calls, all asynchronous on the caller's CUDA stream:
+ *
+ *   dq_bucket_norms            ||g||_2 of Eq. 5, per bucket          (workers)
+ *   dq_choose_bits             bit rule Eq. 17 -> b, s on the device (server)
+ *   dq_quantize_pack           Q_b[g] of Eq. 5/6, b-bit codes packed (workers)
+ *   dq_unpack_dequant_average  "Average" step of Algorithm 1         (server)
+ *
+ * M workers are M gradient buffers on one GPU: worker m's data is at
+ * base + m * stride for every per-worker array.  There is no CPU fallback.
+ *
+ * Conventions
+ *  - "dev" pointers are device pointers owned by the caller.  The library never
+ *    allocates or frees device memory and never synchronises the host.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *  - Return value: DQ_OK or a negative DQ_ERR_* for errors found on the host
+ *    before anything is launched (nothing is written in that case).
+ *  - Conditions only the device can see are OR-ed into *dev_status (DQ_STAT_*
+ *    bits, a caller-owned int32 the caller zeroes and reads when it wants).
+ *    A kernel that raises DQ_STAT_BAD_BITS or DQ_STAT_CAPACITY writes no
+ *    output.  No kernel traps or spins without bound.
+ *  - Data layout ("padded layout"): tensor i of n_i elements starts at element
+ *    offset P_i = sum_{j<i} roundup32(n_j) of a worker's fp32 buffer; the
+ *    buffer holds D32 = sum_i roundup32(n_i) elements.  Buckets of `bucket`
+ *    elements tile each tensor separately; the last bucket of a tensor may be
+ *    short.  Elements between a tensor's end and the next multiple of 32 are
+ *    padding: ignored on input, code 0 in the packed stream, +0 in the output.
+ *  - Packed stream of one worker: group q (padded elements 32q .. 32q+31) owns
+ *    words b*q .. b*q+b-1; element e of the group owns bits [e*b, e*b+b) of
+ *    that little-endian bit string.  A code is sign << (b-1) | level
+ *    (Sec. IV-A: one sign bit and b-1 bits for zeta), s = 2^(b-1) - 1.
+ */
+#ifndef DQ_H
+#define DQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- host return codes ---- */
+#define DQ_OK          0
+#define DQ_ERR_ARG    (-1)  /* NULL pointer, M < 1, bad enum                          */
+#define DQ_ERR_ALIGN  (-2)  /* pointer not 16-byte aligned, stride not a multiple of 32
+                               elements (fp32) / 4 words (packed)                     */
+#define DQ_ERR_RANGE  (-3)  /* size, bucket, rule field or capacity out of range       */
+#define DQ_ERR_CUDA   (-4)  /* a CUDA call (launch, copy, descriptor encode) failed    */
+#define DQ_ERR_STATE  (-5)  /* multi-tensor layout used before its device table was bound */
+
+/* ---- device status bits (OR-ed into *dev_status) ---- */
+#define DQ_STAT_NONFINITE   1  /* a bucket norm or G-bar is NaN/Inf                    */
+#define DQ_STAT_BAD_BITS    2  /* device b outside 1..16                               */
+#define DQ_STAT_CAPACITY    4  /* b * D32/32 words exceed packed_stride_words          */
+#define DQ_STAT_WAIT        8  /* a bounded wait on an asynchronous copy ran out       */
+
+#define DQ_MAX_BITS       16
+#define DQ_MAX_BUCKET   4096
+#define DQ_MAX_WORKERS  4096
+
+typedef struct dq_layout dq_layout_t;   /* host object, immutable after create */
+
+/* Parameters of the bit rule, Eq. 17:
+ *   b_t = log2( sqrt(T / eps_hat) * alpha^((T-1-t)/2) * G-bar_t + 1 ) + 1
+ * eps_hat is the paper's hat-epsilon_Q = 8 W eps_Q / (L d eta^2).  The integer b
+ * is the smallest b in [b_min, b_max] whose s = 2^(b-1) - 1 reaches the
+ * argument of the logarithm minus one (ceiling of Eq. 17), else b_max.
+ * fixed_b in 1..16 bypasses the rule; fixed_b = 0 selects it. */
+typedef struct dq_rule {
+    int32_t T;        /* total iterations, >= 1                */
+    int32_t t;        /* current iteration, 0 <= t < T         */
+    double  eps_hat;  /* > 0                                   */
+    double  alpha;    /* convergence factor of Theorem 1, > 0  */
+    int32_t b_min;    /* 1..16 (2 keeps the quantizer unbiased) */
+    int32_t b_max;    /* b_min..16                              */
+    int32_t fixed_b;  /* 0 or 1..16                             */
+} dq_rule_t;
+
+/* ------------------------------------------------------------------ layout
+ * Host-only bookkeeping of the padded layout above (no CUDA call).
+ * seg_elems[n_seg] are the tensor sizes (>= 0), bucket a multiple of 32 in
+ * 32..DQ_MAX_BUCKET.  The padded total must stay below 2^31 elements.
+ * Errors: DQ_ERR_ARG (NULL, n_seg < 1), DQ_ERR_RANGE. */
+int     dq_layout_create(const int64_t* seg_elems, int32_t n_seg, int32_t bucket, dq_layout_t** out);
+void    dq_layout_destroy(dq_layout_t* layout);
+int32_t dq_layout_num_segments(const dq_layout_t* layout);
+int64_t dq_layout_padded_elems(const dq_layout_t* layout);            /* D32                     */
+int64_t dq_layout_seg_offset(const dq_layout_t* layout, int32_t i);   /* P_i, -1 if i is invalid */
+int64_t dq_layout_num_buckets(const dq_layout_t* layout);             /* nb per worker           */
+int64_t dq_layout_packed_words(const dq_layout_t* layout, int32_t b); /* b * D32 / 32            */
+/* start (padded element index) and valid length of bucket k; DQ_ERR_RANGE if k is invalid */
+int     dq_layout_bucket(const dq_layout_t* layout, int64_t k, int64_t* start, int64_t* len);
+
+/* Layouts with more than one tensor need a small table on the device.  The
+ * caller provides dq_layout_table_bytes() bytes of 16-byte aligned device
+ * memory and keeps it alive while the layout is in use; bind copies the table
+ * there (cudaMemcpyAsync on `stream`, from memory the layout owns) and
+ * remembers the pointer.  Single-tensor layouts need no table (bytes = 0 is
+ * reported and bind is a no-op).  Errors: DQ_ERR_ARG, DQ_ERR_ALIGN,
+ * DQ_ERR_RANGE (buffer too small), DQ_ERR_CUDA. */
+size_t  dq_layout_table_bytes(const dq_layout_t* layout);
+int     dq_layout_bind_device_table(dq_layout_t* layout, void* dev_buf, size_t bytes, void* stream);
+
+/* ------------------------------------------------------------- norms, Eq. 5
+ * dev_norms[m*nb + k] = sqrt( sum of squares of the valid elements of bucket k
+ * of worker m ), the l_2 member of the paper's ||g||_p applied per bucket.
+ * in : dev_grads  fp32, worker m at dev_grads + m*worker_stride_elems,
+ *                 each holding D32 elements in the padded layout
+ * out: dev_norms  fp32 [M][nb]
+ * Sets DQ_STAT_NONFINITE if a norm is not finite (the norm is still written).
+ * Accumulation is fp32 in a fixed order: results are deterministic and within
+ * 1e-6 relative of an fp64 evaluation. */
+int dq_bucket_norms(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
+                    int32_t M, float* dev_norms, int32_t* dev_status, void* stream);
+
+/* --------------------------------------------------------- bit rule, Eq. 17
+ * G-bar^2 = (1/M) sum_m sum_k dev_norms[m][k]^2 (Lemma 1; for p = 2 the sum of
+ * squared bucket norms is the squared norm of the worker's gradient), then the
+ * rule above.  Writes dev_b[0] = b and dev_b[1] = s.  The reduction is fp64 in
+ * a fixed order.  The later calls read b from dev_b, so no host
+ * synchronisation is needed between the calls of a step.
+ * dev_scratch: dq_choose_bits_scratch_bytes() bytes of 16-byte aligned device
+ * memory, used only during the call's kernels.
+ * Sets DQ_STAT_NONFINITE if G-bar is not finite (b = b_max is written). */
+size_t dq_choose_bits_scratch_bytes(const dq_layout_t* layout, int32_t M);
+int dq_choose_bits(const dq_layout_t* layout, const float* dev_norms, int32_t M, const dq_rule_t* rule,
+                   int32_t* dev_b, void* dev_scratch, size_t scratch_bytes,
+                   int32_t* dev_status, void* stream);
+
+/* ----------------------------------------------------- quantizer, Eq. 5 and 6
+ * For every valid element j of worker m, with norm the norm of its bucket and
+ * s = 2^(b-1) - 1, all in fp32 with each operation rounded on its own:
+ *   inv = norm >= 2^-100 ? s / norm : 0      r = min(|g_j| * inv, s)
+ *   l = floor(r)   p_r = r - l   level = l + [u < p_r]   code = sign(g_j) << (b-1) | level
+ * u = (w >> 8) * 2^-24 where w is word (j & 3) of Philox4x32-10 with counter
+ * (j >> 2, 0, m, step) and key (seed low word, seed high word); j is the
+ * element's index in the padded layout.  b = 1 stores the sign bit only.
+ * The codes are packed as described at the top of this file.
+ * in : dev_grads, dev_norms [M][nb], dev_b (written by dq_choose_bits)
+ * out: dev_packed uint32, worker m at dev_packed + m*packed_stride_words; the
+ *      first b*D32/32 words are written, the rest left untouched.
+ * Device conditions: DQ_STAT_BAD_BITS, DQ_STAT_CAPACITY (nothing is written),
+ * DQ_STAT_WAIT. */
+int dq_quantize_pack(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
+                     int32_t M, const float* dev_norms, const int32_t* dev_b,
+                     uint64_t seed, uint32_t step,
+                     uint32_t* dev_packed, int64_t packed_stride_words,
+                     int32_t* dev_status, void* stream);
+
+/* ----------------------------------- Algorithm 1, server side: "Average"
+ * dev_out[j] = (1/M) sum_m sgn * level * norm_m / s   (Eq. 5 inverted, then
+ * the mean over workers); 0 for padding and when s = 0.  fp32 accumulation in
+ * worker order: deterministic, within 1e-6 relative L2 of an fp64 evaluation.
+ * in : dev_packed, dev_norms [M][nb], dev_b
+ * out: dev_out fp32 [D32]
+ * Device conditions: DQ_STAT_BAD_BITS, DQ_STAT_CAPACITY (nothing is written),
+ * DQ_STAT_WAIT. */
+int dq_unpack_dequant_average(const dq_layout_t* layout, const uint32_t* dev_packed,
+                              int64_t packed_stride_words, const float* dev_norms, int32_t M,
+                              const int32_t* dev_b, float* dev_out, int32_t* dev_status, void* stream);
+
+/* Text for a DQ_ERR_* return value (static storage). */
+const char* dq_status_string(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DQ_H */

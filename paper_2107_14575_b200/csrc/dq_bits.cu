@@ -1,0 +1,126 @@
+// dq_choose_bits: the bit rule of Eq. 17 evaluated on the device.
+//
+//   G-bar^2 = (1/M) sum over workers and buckets of norm^2        (Lemma 1)
+//   x       = sqrt(T/eps_hat) * alpha^((T-1-t)/2) * G-bar
+//   b       = smallest b in [b_min, b_max] with 2^(b-1) - 1 >= x   (else b_max)
+//
+// Two small kernels: fixed-size chunks of the norm array are summed in fp64
+// (fixed assignment of elements to threads, fixed tree), then one CTA adds
+// the chunk sums in a fixed order and applies the rule.  The factor
+// sqrt(T/eps_hat) * alpha^((T-1-t)/2) is a host scalar.
+#include "dq_common.cuh"
+
+#include <cmath>
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kChunk = 8192;     // norms per CTA of the first kernel
+
+__device__ __forceinline__ double block_sum(double v, double* sh)
+{
+    sh[threadIdx.x] = v;
+    __syncthreads();
+#pragma unroll
+    for (int o = kThreads / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+        __syncthreads();
+    }
+    return sh[0];
+}
+
+__global__ void __launch_bounds__(kThreads)
+norm_square_partials(const float* __restrict__ norms, const int64_t n, double* __restrict__ partial)
+{
+    __shared__ double sh[kThreads];
+    const int64_t base = (int64_t)blockIdx.x * kChunk;
+    double acc = 0.0;
+#pragma unroll 4
+    for (int i = threadIdx.x; i < kChunk; i += kThreads) {
+        const int64_t j = base + i;
+        if (j < n) {
+            const double x = (double)__ldg(norms + j);
+            acc = fma(x, x, acc);
+        }
+    }
+    const double s = block_sum(acc, sh);
+    if (threadIdx.x == 0) partial[blockIdx.x] = s;
+}
+
+__global__ void __launch_bounds__(kThreads)
+apply_rule(const double* __restrict__ partial, const int npartial, const int M, const double coef,
+           const int b_min, const int b_max, const int fixed_b,
+           int32_t* __restrict__ dev_b, int32_t* __restrict__ status)
+{
+    __shared__ double sh[kThreads];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < npartial; i += kThreads) acc += partial[i];
+    const double sum = block_sum(acc, sh);
+    if (threadIdx.x != 0) return;
+
+    int b;
+    if (fixed_b != 0) {
+        b = fixed_b;
+    } else {
+        const double x = coef * sqrt(sum / (double)M);
+        b = b_max;
+        if (isfinite(x)) {
+            for (int c = b_min; c <= b_max; ++c) {
+                if ((double)((1 << (c - 1)) - 1) >= x) { b = c; break; }
+            }
+        } else {
+            atomicOr(status, DQ_STAT_NONFINITE);
+        }
+    }
+    dev_b[0] = b;
+    dev_b[1] = (1 << (b - 1)) - 1;
+}
+
+inline int64_t num_chunks(int64_t n) { return (n + kChunk - 1) / kChunk; }
+
+}  // namespace
+
+extern "C" size_t dq_choose_bits_scratch_bytes(const dq_layout_t* L, int32_t M)
+{
+    if (!L || M < 1) return 0;
+    const int64_t c = num_chunks((int64_t)M * L->nb);
+    return (size_t)((c * sizeof(double) + 255) / 256 * 256);
+}
+
+extern "C" int dq_choose_bits(const dq_layout_t* L, const float* dev_norms, int32_t M, const dq_rule_t* rule,
+                              int32_t* dev_b, void* dev_scratch, size_t scratch_bytes,
+                              int32_t* dev_status, void* stream)
+{
+    if (!L || !rule) return DQ_ERR_ARG;
+    if (M < 1) return DQ_ERR_ARG;
+    if (M > DQ_MAX_WORKERS) return DQ_ERR_RANGE;
+    if (!dev_norms || !dev_b || !dev_status || !dev_scratch) return DQ_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(dev_norms) & 3u) || (reinterpret_cast<uintptr_t>(dev_b) & 3u) ||
+        (reinterpret_cast<uintptr_t>(dev_status) & 3u) || !aligned16(dev_scratch))
+        return DQ_ERR_ALIGN;
+    if (rule->fixed_b < 0 || rule->fixed_b > DQ_MAX_BITS) return DQ_ERR_RANGE;
+    if (rule->b_min < 1 || rule->b_max > DQ_MAX_BITS || rule->b_min > rule->b_max) return DQ_ERR_RANGE;
+    if (rule->fixed_b == 0 &&
+        (rule->T < 1 || rule->t < 0 || rule->t >= rule->T || !(rule->eps_hat > 0.0) || !(rule->alpha > 0.0) ||
+         !std::isfinite(rule->eps_hat) || !std::isfinite(rule->alpha)))
+        return DQ_ERR_RANGE;
+    if (scratch_bytes < dq_choose_bits_scratch_bytes(L, M)) return DQ_ERR_RANGE;
+
+    const int64_t n = (int64_t)M * L->nb;
+    const int64_t chunks = num_chunks(n);
+    double coef = 0.0;
+    if (rule->fixed_b == 0)
+        coef = std::sqrt((double)rule->T / rule->eps_hat) *
+               std::pow(rule->alpha, (double)(rule->T - 1 - rule->t) / 2.0);
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* partial = static_cast<double*>(dev_scratch);
+    if (rule->fixed_b == 0) {
+        norm_square_partials<<<(unsigned)chunks, kThreads, 0, st>>>(dev_norms, n, partial);
+        if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    }
+    apply_rule<<<1, kThreads, 0, st>>>(partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
+                                      rule->b_min, rule->b_max, rule->fixed_b, dev_b, dev_status);
+    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}

@@ -1,0 +1,146 @@
+// Host layout object of the padded, bucketed gradient layout, and helpers
+// shared by the entry points.
+#include "dq_common.cuh"
+
+#include <mutex>
+#include <new>
+
+static inline int64_t up32(int64_t n) { return (n + 31) / 32 * 32; }
+
+extern "C" int dq_layout_create(const int64_t* seg_elems, int32_t n_seg, int32_t bucket, dq_layout_t** out)
+{
+    if (!seg_elems || !out || n_seg < 1) return DQ_ERR_ARG;
+    if (bucket < 32 || bucket > DQ_MAX_BUCKET || bucket % 32 != 0) return DQ_ERR_RANGE;
+    int64_t padded = 0, nb = 0;
+    for (int32_t i = 0; i < n_seg; ++i) {
+        if (seg_elems[i] < 0 || seg_elems[i] >= (int64_t(1) << 31)) return DQ_ERR_RANGE;
+        padded += up32(seg_elems[i]);
+        nb += (seg_elems[i] + bucket - 1) / bucket;
+        if (padded >= (int64_t(1) << 31)) return DQ_ERR_RANGE;
+    }
+    if (padded == 0) return DQ_ERR_RANGE;
+    dq_layout* L = new (std::nothrow) dq_layout;
+    if (!L) return DQ_ERR_ARG;
+    L->n_seg = n_seg;
+    L->bucket = bucket;
+    L->padded = padded;
+    L->nb = nb;
+    L->seg_elems.assign(seg_elems, seg_elems + n_seg);
+    L->seg_offset.resize(n_seg);
+    const int32_t n1 = n_seg + 1;
+    L->table.assign(size_t(3) * n1, 0);
+    int64_t p = 0, k = 0;
+    for (int32_t i = 0; i < n_seg; ++i) {
+        L->seg_offset[i] = p;
+        L->table[i] = (int32_t)(p / 32);
+        L->table[n1 + i] = (int32_t)k;
+        L->table[2 * n1 + i] = (int32_t)seg_elems[i];
+        p += up32(seg_elems[i]);
+        k += (seg_elems[i] + bucket - 1) / bucket;
+    }
+    L->table[n_seg] = (int32_t)(p / 32);
+    L->table[n1 + n_seg] = (int32_t)k;
+    L->table[2 * n1 + n_seg] = 0;
+    *out = L;
+    return DQ_OK;
+}
+
+extern "C" void dq_layout_destroy(dq_layout_t* layout) { delete layout; }
+
+extern "C" int32_t dq_layout_num_segments(const dq_layout_t* L) { return L ? L->n_seg : 0; }
+extern "C" int64_t dq_layout_padded_elems(const dq_layout_t* L) { return L ? L->padded : 0; }
+extern "C" int64_t dq_layout_num_buckets(const dq_layout_t* L) { return L ? L->nb : 0; }
+
+extern "C" int64_t dq_layout_seg_offset(const dq_layout_t* L, int32_t i)
+{
+    if (!L || i < 0 || i >= L->n_seg) return -1;
+    return L->seg_offset[i];
+}
+
+extern "C" int64_t dq_layout_packed_words(const dq_layout_t* L, int32_t b)
+{
+    if (!L || b < 1 || b > DQ_MAX_BITS) return 0;
+    return L->padded / 32 * b;
+}
+
+extern "C" int dq_layout_bucket(const dq_layout_t* L, int64_t k, int64_t* start, int64_t* len)
+{
+    if (!L || !start || !len) return DQ_ERR_ARG;
+    if (k < 0 || k >= L->nb) return DQ_ERR_RANGE;
+    const int32_t n1 = L->n_seg + 1;
+    // last tensor whose first bucket is <= k
+    int32_t lo = 0, hi = L->n_seg;
+    while (hi - lo > 1) {
+        const int32_t mid = (lo + hi) / 2;
+        if (L->table[n1 + mid] <= k) lo = mid; else hi = mid;
+    }
+    const int64_t local = k - L->table[n1 + lo];
+    *start = L->seg_offset[lo] + local * L->bucket;
+    const int64_t left = L->seg_elems[lo] - local * L->bucket;
+    *len = left < L->bucket ? left : L->bucket;
+    return DQ_OK;
+}
+
+extern "C" size_t dq_layout_table_bytes(const dq_layout_t* L)
+{
+    if (!L || L->n_seg == 1) return 0;
+    return L->table.size() * sizeof(int32_t);
+}
+
+extern "C" int dq_layout_bind_device_table(dq_layout_t* L, void* dev_buf, size_t bytes, void* stream)
+{
+    if (!L) return DQ_ERR_ARG;
+    if (L->n_seg == 1) return DQ_OK;
+    if (!dev_buf) return DQ_ERR_ARG;
+    if (!aligned16(dev_buf)) return DQ_ERR_ALIGN;
+    const size_t need = L->table.size() * sizeof(int32_t);
+    if (bytes < need) return DQ_ERR_RANGE;
+    if (cudaMemcpyAsync(dev_buf, L->table.data(), need, cudaMemcpyHostToDevice,
+                        static_cast<cudaStream_t>(stream)) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DQ_ERR_CUDA;
+    }
+    L->dev_table = static_cast<const int32_t*>(dev_buf);
+    return DQ_OK;
+}
+
+int dq_check_common(const dq_layout* L, int32_t M)
+{
+    if (!L) return DQ_ERR_ARG;
+    if (M < 1) return DQ_ERR_ARG;
+    if (M > DQ_MAX_WORKERS) return DQ_ERR_RANGE;
+    if (L->n_seg > 1 && !L->dev_table) return DQ_ERR_STATE;
+    return DQ_OK;
+}
+
+int dq_sm_count()
+{
+    static std::mutex mu;
+    static int cached_dev = -1, cached_sms = 0;
+    std::lock_guard<std::mutex> lock(mu);
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { (void)cudaGetLastError(); return 148; }
+    if (dev != cached_dev) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+            (void)cudaGetLastError();
+            sms = 148;
+        }
+        cached_dev = dev;
+        cached_sms = sms;
+    }
+    return cached_sms;
+}
+
+extern "C" const char* dq_status_string(int code)
+{
+    switch (code) {
+        case DQ_OK:        return "ok";
+        case DQ_ERR_ARG:   return "invalid argument (NULL pointer, M < 1)";
+        case DQ_ERR_ALIGN: return "misaligned pointer or stride";
+        case DQ_ERR_RANGE: return "value out of range";
+        case DQ_ERR_CUDA:  return "CUDA call failed";
+        case DQ_ERR_STATE: return "layout has several tensors but no device table is bound";
+        default:           return "unknown status";
+    }
+}

@@ -1,0 +1,204 @@
+"""Thin ctypes binding of the C-ABI CUDA library (``include/dq.h``).
+
+Argument marshalling only: every step of the path runs in the library's
+kernels.  Tensors are torch CUDA tensors (device memory and streams are
+torch's); the functions have the names and the argument order of the C calls.
+There is no fallback: a missing ``libdq.so`` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libdq.so")
+
+OK, ERR_ARG, ERR_ALIGN, ERR_RANGE, ERR_CUDA, ERR_STATE = 0, -1, -2, -3, -4, -5
+STAT_NONFINITE, STAT_BAD_BITS, STAT_CAPACITY, STAT_WAIT = 1, 2, 4, 8
+
+# every symbol include/dq.h declares
+SYMBOLS = [
+    "dq_layout_create", "dq_layout_destroy", "dq_layout_num_segments", "dq_layout_padded_elems",
+    "dq_layout_seg_offset", "dq_layout_num_buckets", "dq_layout_packed_words", "dq_layout_bucket",
+    "dq_layout_table_bytes", "dq_layout_bind_device_table",
+    "dq_bucket_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
+    "dq_quantize_pack", "dq_unpack_dequant_average", "dq_status_string",
+]
+
+
+class DQError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} ({code})")
+
+
+class Rule(C.Structure):
+    """``dq_rule_t``: parameters of the bit rule, Eq. 17."""
+    _fields_ = [("T", C.c_int32), ("t", C.c_int32), ("eps_hat", C.c_double), ("alpha", C.c_double),
+                ("b_min", C.c_int32), ("b_max", C.c_int32), ("fixed_b", C.c_int32)]
+
+    @classmethod
+    def dynamic(cls, T: int, t: int, eps_hat: float, alpha: float, b_min: int = 2, b_max: int = 16):
+        return cls(T, t, eps_hat, alpha, b_min, b_max, 0)
+
+    @classmethod
+    def fixed(cls, b: int):
+        return cls(1, 0, 1.0, 1.0, 1, 16, b)
+
+
+_lib = None
+
+
+def lib():
+    """Loads ``libdq.so`` (built by ``python -m paper_2107_14575_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2107_14575_b200.build` "
+                "(there is no fallback implementation)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, u32, u64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_size_t
+        L.dq_layout_create.restype = C.c_int
+        L.dq_layout_create.argtypes = [C.POINTER(i64), i32, i32, C.POINTER(vp)]
+        L.dq_layout_destroy.restype = None
+        L.dq_layout_destroy.argtypes = [vp]
+        L.dq_layout_num_segments.restype = i32
+        L.dq_layout_num_segments.argtypes = [vp]
+        L.dq_layout_padded_elems.restype = i64
+        L.dq_layout_padded_elems.argtypes = [vp]
+        L.dq_layout_seg_offset.restype = i64
+        L.dq_layout_seg_offset.argtypes = [vp, i32]
+        L.dq_layout_num_buckets.restype = i64
+        L.dq_layout_num_buckets.argtypes = [vp]
+        L.dq_layout_packed_words.restype = i64
+        L.dq_layout_packed_words.argtypes = [vp, i32]
+        L.dq_layout_bucket.restype = C.c_int
+        L.dq_layout_bucket.argtypes = [vp, i64, C.POINTER(i64), C.POINTER(i64)]
+        L.dq_layout_table_bytes.restype = sz
+        L.dq_layout_table_bytes.argtypes = [vp]
+        L.dq_layout_bind_device_table.restype = C.c_int
+        L.dq_layout_bind_device_table.argtypes = [vp, vp, sz, vp]
+        L.dq_bucket_norms.restype = C.c_int
+        L.dq_bucket_norms.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+        L.dq_choose_bits_scratch_bytes.restype = sz
+        L.dq_choose_bits_scratch_bytes.argtypes = [vp, i32]
+        L.dq_choose_bits.restype = C.c_int
+        L.dq_choose_bits.argtypes = [vp, vp, i32, C.POINTER(Rule), vp, vp, sz, vp, vp]
+        L.dq_quantize_pack.restype = C.c_int
+        L.dq_quantize_pack.argtypes = [vp, vp, i64, i32, vp, vp, u64, u32, vp, i64, vp, vp]
+        L.dq_unpack_dequant_average.restype = C.c_int
+        L.dq_unpack_dequant_average.argtypes = [vp, vp, i64, vp, i32, vp, vp, vp, vp]
+        L.dq_status_string.restype = C.c_char_p
+        L.dq_status_string.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().dq_status_string(int(code)).decode()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OK:
+        raise DQError(rc, where)
+
+
+def _ptr(t) -> int:
+    """Device (or host) address of a torch tensor, or an int passed through."""
+    if t is None:
+        return 0
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class Layout:
+    """``dq_layout_t``: the padded, bucketed layout of a list of tensors."""
+
+    def __init__(self, seg_elems: Sequence[int], bucket: int):
+        arr = (C.c_int64 * len(seg_elems))(*[int(x) for x in seg_elems])
+        h = C.c_void_p()
+        _check(lib().dq_layout_create(arr, len(seg_elems), int(bucket), C.byref(h)), "dq_layout_create")
+        self._h = h
+        self.bucket = int(bucket)
+        self.n_seg = int(lib().dq_layout_num_segments(h))
+        self.D32 = int(lib().dq_layout_padded_elems(h))
+        self.nb = int(lib().dq_layout_num_buckets(h))
+        self.offsets = [int(lib().dq_layout_seg_offset(h, i)) for i in range(self.n_seg)]
+        self._table = None          # keeps the bound device table alive
+
+    def __del__(self):
+        h, self._h = getattr(self, "_h", None), None
+        if h is not None and _lib is not None:
+            _lib.dq_layout_destroy(h)
+
+    @property
+    def handle(self):
+        return self._h
+
+    def packed_words(self, b: int) -> int:
+        return int(lib().dq_layout_packed_words(self._h, int(b)))
+
+    def bucket_range(self, k: int):
+        s, n = C.c_int64(), C.c_int64()
+        _check(lib().dq_layout_bucket(self._h, int(k), C.byref(s), C.byref(n)), "dq_layout_bucket")
+        return int(s.value), int(n.value)
+
+    def table_bytes(self) -> int:
+        return int(lib().dq_layout_table_bytes(self._h))
+
+    def bind_device_table(self, dev_buf, nbytes: Optional[int] = None, stream=None) -> None:
+        """dev_buf: a torch uint8/int32 CUDA tensor (kept alive by this object) or a raw address."""
+        if nbytes is None:
+            nbytes = dev_buf.numel() * dev_buf.element_size()
+        _check(lib().dq_layout_bind_device_table(self._h, _ptr(dev_buf), int(nbytes), _stream(stream)),
+               "dq_layout_bind_device_table")
+        self._table = dev_buf
+
+    def bind(self, device="cuda", stream=None) -> "Layout":
+        """Allocates the device table with torch (if the layout needs one) and binds it."""
+        need = self.table_bytes()
+        if need:
+            import torch
+            self.bind_device_table(torch.empty(need, dtype=torch.uint8, device=device), need, stream)
+        return self
+
+
+def bucket_norms(layout: Layout, grads, worker_stride_elems: int, M: int, norms, status, stream=None) -> None:
+    _check(lib().dq_bucket_norms(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(norms),
+                                 _ptr(status), _stream(stream)), "dq_bucket_norms")
+
+
+def choose_bits_scratch_bytes(layout: Layout, M: int) -> int:
+    return int(lib().dq_choose_bits_scratch_bytes(layout.handle, int(M)))
+
+
+def choose_bits(layout: Layout, norms, M: int, rule: Rule, dev_b, scratch, scratch_bytes: int, status,
+                stream=None) -> None:
+    _check(lib().dq_choose_bits(layout.handle, _ptr(norms), int(M), C.byref(rule), _ptr(dev_b), _ptr(scratch),
+                                int(scratch_bytes), _ptr(status), _stream(stream)), "dq_choose_bits")
+
+
+def quantize_pack(layout: Layout, grads, worker_stride_elems: int, M: int, norms, dev_b, seed: int, step: int,
+                  packed, packed_stride_words: int, status, stream=None) -> None:
+    _check(lib().dq_quantize_pack(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(norms),
+                                  _ptr(dev_b), int(seed) & (2 ** 64 - 1), int(step) & 0xFFFFFFFF, _ptr(packed),
+                                  int(packed_stride_words), _ptr(status), _stream(stream)), "dq_quantize_pack")
+
+
+def unpack_dequant_average(layout: Layout, packed, packed_stride_words: int, norms, M: int, dev_b, out, status,
+                           stream=None) -> None:
+    _check(lib().dq_unpack_dequant_average(layout.handle, _ptr(packed), int(packed_stride_words), _ptr(norms),
+                                           int(M), _ptr(dev_b), _ptr(out), _ptr(status), _stream(stream)),
+           "dq_unpack_dequant_average")

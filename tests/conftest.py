@@ -28,3 +28,12 @@ def read_golden(name):
 @pytest.fixture(scope="session")
 def golden():
     return read_golden
+
+
+@pytest.fixture(scope="session")
+def dqlib():
+    """The CUDA library, built in-tree if needed (nvcc cross-compiles without a GPU)."""
+    from paper_2107_14575_b200 import build, dq
+    build.build()
+    dq.lib()
+    return dq
