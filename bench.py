@@ -291,6 +291,28 @@ def run_cuda(args) -> dict:
     value = world * 4.0 * M * w.d * K / (ms * 1e-3) / 1e9
 
     # ---- end to end: pinned host gradients in, averaged gradient out, copies timed ----
+    e2e = None
+    if not args.no_e2e:
+        e2e = _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, w.d, D32)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
+        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "bits_first_last": [bits[0], bits[-1]], "mean_bits": round(mean_b, 3),
+                   "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
+                   "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * K, "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = _cpu_baseline(pool, w, eps_hat, alpha)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return out if rank == 0 else {}
+
+
+def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> dict:
     Ke = min(K, 10)
     host = [pool[p].cpu().pin_memory() for p in range(2)]
     for i in range(2):
@@ -310,26 +332,9 @@ def run_cuda(args) -> dict:
         tmax = torch.tensor([ms2], dtype=torch.float64, device=dev)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         ms2 = float(tmax.item())
-    e2e = {"value": world * 4.0 * M * w.d * Ke / (ms2 * 1e-3) / 1e9, "unit": UNIT,
-           "h2d_bytes_per_step": 4 * M * D32, "d2h_bytes_per_step": 4 * D32, "steps": Ke,
-           "ms_per_step": ms2 / Ke, "checksum": checksum}
-
-    out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "bits_first_last": [bits[0], bits[-1]], "mean_bits": round(mean_b, 3),
-                   "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
-                   "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * K, "roofline": roofline,
-    }
-
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = _cpu_baseline(pool, w, eps_hat, alpha)
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
-    return out if rank == 0 else {}
+    return {"value": world * 4.0 * M * d * Ke / (ms2 * 1e-3) / 1e9, "unit": UNIT,
+            "h2d_bytes_per_step": 4 * M * D32, "d2h_bytes_per_step": 4 * D32, "steps": Ke,
+            "ms_per_step": ms2 / Ke, "checksum": checksum}
 
 
 def _cpu_baseline(pool, w, eps_hat, alpha) -> dict:
@@ -354,7 +359,8 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:

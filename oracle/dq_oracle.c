@@ -150,15 +150,19 @@ void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-/* uniform in [0,1) with 24 bits, for padded element index j of worker m */
-static float uniform24(uint64_t seed, uint32_t step, uint32_t m, int64_t j)
+/* Rounding uniform of padded element j of worker m at a step: word (j & 3) of
+ * the Philox block with counter (j >> 2, 0, m, step) and key (seed lo, seed hi).
+ * Its top 23 bits k give u = 1 - (2k + 1) / 2^24, a midpoint grid on (0, 1):
+ * u is never 0, so p_r = 0 never rounds up, and never 1. */
+static float uniform23(uint64_t seed, uint32_t step, uint32_t m, int64_t j)
 {
     const uint64_t q = (uint64_t)j >> 2;
     const uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), m, step };
     const uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
     uint32_t r[4];
     oracle_philox4x32_10(ctr, key, r);
-    return (float)(r[j & 3] >> 8) * 0x1p-24f;
+    const uint32_t k = r[j & 3] >> 9;
+    return 1.0f - (float)(2u * k + 1u) * 0x1p-24f;     /* both steps exact in fp32 */
 }
 
 /* ---------------------------------------------------------------- quantize */
@@ -194,8 +198,8 @@ void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
             r = fminf(r, sf);                /* an ulp above s must not carry into the sign */
             const float l = floorf(r);
             const float f = r - l;           /* p_r of Eq. 6, exact in fp32 */
-            const float u = uniform24(seed, step, (uint32_t)m, j);
-            const uint32_t level = (uint32_t)l + (u < f ? 1u : 0u);
+            const float u = uniform23(seed, step, (uint32_t)m, j);
+            const uint32_t level = (uint32_t)l + (u <= f ? 1u : 0u);   /* up with probability p_r */
             uint32_t gbits;
             memcpy(&gbits, &g, sizeof gbits);
             const uint32_t sign = gbits >> 31;

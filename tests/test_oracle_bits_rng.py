@@ -123,7 +123,8 @@ def test_philox_counter_and_key_separation():
 
 def test_uniform_is_philox_word_of_the_element():
     # element j of worker m at a step draws word (j & 3) of the block with counter
-    # (j >> 2, 0, m, step) and key (seed lo, seed hi); u = top 24 bits * 2^-24
+    # (j >> 2, 0, m, step) and key (seed lo, seed hi); with k its top 23 bits,
+    # u = 1 - (2k + 1) / 2^24
     lay = oracle.Layout([64], 32)
     g = np.ones((3, 64), np.float32)
     norms = oracle.bucket_norms(lay, g)
@@ -132,18 +133,20 @@ def test_uniform_is_philox_word_of_the_element():
     for m in range(3):
         for j in (0, 1, 5, 31, 32, 63):
             blk = oracle.philox4x32_10([j >> 2, 0, m, step], [0x12345678, 0xDEADBEEF])
-            assert u[m, j] == np.float32(int(blk[j & 3]) >> 8) * np.float32(2.0 ** -24)
+            k = int(blk[j & 3]) >> 9
+            assert float(u[m, j]) == 1.0 - (2 * k + 1) / 2.0 ** 24
 
 
 def test_uniform_statistics():
-    # 2^22 draws: mean 1/2 within 5 sigma, chi-square over 256 cells, in [0,1)
+    # 2^22 draws: mean 1/2 within 5 sigma, chi-square over 256 cells, in (0,1)
     lay = oracle.Layout([1 << 20], 4096)
     g = np.ones((4, 1 << 20), np.float32)
     norms = oracle.bucket_norms(lay, g)
     _, _, u = oracle.quantize(lay, g, norms, 4, 123, 0, want_frac_u=True)
     u = u.ravel().astype(np.float64)
     n = u.size
-    assert u.min() >= 0.0 and u.max() < 1.0
+    assert u.min() > 0.0 and u.max() < 1.0
+    assert np.all((u * 2 ** 24) % 2 == 1)                   # odd multiples of 2^-24: the midpoint grid
     assert abs(u.mean() - 0.5) < 5 * math.sqrt(1 / 12 / n)
     counts = np.bincount((u * 256).astype(np.int64), minlength=256)
     chi2 = ((counts - n / 256) ** 2 / (n / 256)).sum()

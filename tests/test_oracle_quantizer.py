@@ -124,7 +124,7 @@ def test_exact_expectation_by_enumeration(b, d):
     # the oracle's p_r against the definition p_r = s|g|/||g|| - l in fp64
     r = s * np.abs(v[0, :d].astype(np.float64)) / norm
     assert np.allclose(frac, r - np.floor(r), atol=4e-7 * max(1.0, s))
-    low = (codes & s) - (u < frac.astype(np.float32))            # floor level l
+    low = (codes & s) - (u <= frac.astype(np.float32))           # floor level l
     assert np.array_equal(low, np.floor(r).astype(np.int64)) or np.all(np.abs(r - np.round(r)) < 1e-5)
     sign = codes & (1 << (b - 1))
     mean = np.zeros(d)
@@ -284,22 +284,32 @@ def test_average_matches_numpy_definition():
 
 # ------------------------------------------------ boundary cases of Eq. 6
 
-def test_zero_uniform_never_rounds_an_on_level_value_up():
-    # p_r = 0 must give the lower level with probability 1, also when u = 0
+def test_smallest_uniform_boundaries():
+    # The uniform lives on (0, 1): with p_r = 0 the lower level is kept for every draw, also
+    # the smallest one (u = 2^-24); p_r = u exactly rounds up ("with probability p_r" counts
+    # the draws u <= p_r), p_r just below u does not.
     from conftest import read_golden
-    b, s = 5, 15
-    for seed, step, m, j in [tuple(int(x) for x in r) for r in read_golden("zero_uniform.txt")]:
+    for seed, step, m, j in [tuple(int(x) for x in r) for r in read_golden("smallest_uniform.txt")]:
         blk = oracle.philox4x32_10([j >> 2, 0, m, step], [seed & 0xFFFFFFFF, seed >> 32])
-        assert int(blk[j & 3]) >> 8 == 0                     # the stored position does draw u = 0
+        assert int(blk[j & 3]) >> 9 == 0x7FFFFF               # the stored position draws the smallest u
         n = (j // 32 + 1) * 32
         lay = oracle.Layout([n], 32)
+        k = j ^ 1                                             # partner element in the same bucket
+        # (a) on-level value: norm 15, levels 9 and 12 with b = 5
         g = np.zeros((1, n), np.float32)
-        k = j ^ 1                                            # partner element in the same bucket
-        g[0, j], g[0, k] = -9.0, 12.0                        # norm 15: levels 9 and 12 exactly
+        g[0, j], g[0, k] = -9.0, 12.0
         norms = oracle.bucket_norms(lay, g)
-        codes, frac, u = oracle.quantize(lay, g, norms, b, seed, step, want_frac_u=True)
-        assert u[0, j] == 0.0 and frac[0, j] == 0.0
-        assert codes[0, j] == (1 << (b - 1)) | 9 and codes[0, k] == 12
+        codes, frac, u = oracle.quantize(lay, g, norms, 5, seed, step, want_frac_u=True)
+        assert u[0, j] == np.float32(2.0 ** -24) and frac[0, j] == 0.0
+        assert codes[0, j] == (1 << 4) | 9 and codes[0, k] == 12
+        # (b) b = 2 (s = 1), norm 1: p_r = |g|; 2^-24 reaches u, 2^-25 does not
+        for val, want_level in ((2.0 ** -24, 1), (2.0 ** -25, 0), (1.5 * 2.0 ** -24, 1)):
+            g[0, j], g[0, k] = val, 1.0
+            norms = oracle.bucket_norms(lay, g)
+            assert norms[0, j // 32] == 1.0
+            codes, frac, u = oracle.quantize(lay, g, norms, 2, seed, step, want_frac_u=True)
+            assert frac[0, j] == np.float32(val)
+            assert codes[0, j] == want_level
 
 
 def test_ratio_one_ulp_above_s_is_clamped():
