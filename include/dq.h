@@ -136,10 +136,12 @@ int dq_choose_bits(const dq_layout_t* layout, const float* dev_norms, int32_t M,
  * For every valid element j of worker m, with norm the norm of its bucket and
  * s = 2^(b-1) - 1, all in fp32 with each operation rounded on its own:
  *   inv = norm >= 2^-100 ? s / norm : 0      r = min(|g_j| * inv, s)
- *   l = floor(r)   p_r = r - l   level = l + [u < p_r]   code = sign(g_j) << (b-1) | level
- * u = (w >> 8) * 2^-24 where w is word (j & 3) of Philox4x32-10 with counter
- * (j >> 2, 0, m, step) and key (seed low word, seed high word); j is the
- * element's index in the padded layout.  b = 1 stores the sign bit only.
+ *   l = floor(r)   p_r = r - l   level = l + [u <= p_r]   code = sign(g_j) << (b-1) | level
+ * u = 1 - (2k + 1) / 2^24 in (0, 1), k = w >> 9, where w is word (j & 3) of
+ * Philox4x32-10 with counter (j >> 2, 0, m, step) and key (seed low word, seed
+ * high word); j is the element's index in the padded layout.  The level goes
+ * up with probability p_r (within 2^-24) as Eq. 6 asks, and values that lie
+ * on a level are reproduced for every draw.  b = 1 stores the sign bit only.
  * The codes are packed as described at the top of this file.
  * in : dev_grads, dev_norms [M][nb], dev_b (written by dq_choose_bits)
  * out: dev_packed uint32, worker m at dev_packed + m*packed_stride_words; the

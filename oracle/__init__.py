@@ -160,12 +160,13 @@ def philox4x32_10(ctr, key) -> np.ndarray:
 
 
 def quantize(lay: Layout, grads: np.ndarray, norms: np.ndarray, b: int, seed: int, step: int,
-             want_frac_u: bool = False):
+             want_x_v: bool = False):
+    """Codes [M, D32]; with want_x_v also x (signed position on the level grid) and v (uniform)."""
     ptr, stride, M = _check_grads(lay, grads)
     norms = np.ascontiguousarray(norms, np.float32)
     assert norms.shape == (M, lay.nb)
     codes = np.zeros((M, lay.D32), np.uint32)
-    if want_frac_u:
+    if want_x_v:
         frac = np.zeros((M, lay.D32), np.float32)
         u = np.zeros((M, lay.D32), np.float32)
         lib().oracle_quantize(ptr, stride, M, *lay._args(), norms, b, seed, step, codes,

@@ -150,19 +150,20 @@ void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-/* Rounding uniform of padded element j of worker m at a step: word (j & 3) of
- * the Philox block with counter (j >> 2, 0, m, step) and key (seed lo, seed hi).
- * Its top 23 bits k give u = 1 - (2k + 1) / 2^24, a midpoint grid on (0, 1):
- * u is never 0, so p_r = 0 never rounds up, and never 1. */
-static float uniform23(uint64_t seed, uint32_t step, uint32_t m, int64_t j)
+/* Rounding uniform of padded element j of worker m at a step: Philox block
+ * with counter (j >> 3, 0, m, step) and key (seed lo, seed hi); element j owns
+ * half (j & 1) (0 = low 16 bits) of word ((j >> 1) & 3).  With k that 16-bit
+ * value, v = (2k + 1) / 2^17: a midpoint grid on (0, 1), never 0 and never 1. */
+static float uniform16(uint64_t seed, uint32_t step, uint32_t m, int64_t j)
 {
-    const uint64_t q = (uint64_t)j >> 2;
+    const uint64_t q = (uint64_t)j >> 3;
     const uint32_t ctr[4] = { (uint32_t)q, (uint32_t)(q >> 32), m, step };
     const uint32_t key[2] = { (uint32_t)seed, (uint32_t)(seed >> 32) };
     uint32_t r[4];
     oracle_philox4x32_10(ctr, key, r);
-    const uint32_t k = r[j & 3] >> 9;
-    return 1.0f - (float)(2u * k + 1u) * 0x1p-24f;     /* both steps exact in fp32 */
+    const uint32_t word = r[(j >> 1) & 3];
+    const uint32_t k = (j & 1) ? (word >> 16) : (word & 0xFFFFu);
+    return (float)(2u * k + 1u) * 0x1p-17f;            /* exact in fp32 */
 }
 
 /* ---------------------------------------------------------------- quantize */
@@ -173,16 +174,17 @@ static float uniform23(uint64_t seed, uint32_t step, uint32_t m, int64_t j)
 void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
                      const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
                      const float* norms, int32_t b, uint64_t seed, uint32_t step,
-                     uint32_t* codes, float* frac_out, float* u_out)
+                     uint32_t* codes, float* x_out, float* v_out)
 {
     table_t tb = make_table(seg_elems, n_seg, bucket);
     const int64_t D32 = oracle_padded_elems(seg_elems, n_seg);
     const int32_t s = (1 << (b - 1)) - 1;
     const float sf = (float)s;
 
-    memset(codes, 0, sizeof(uint32_t) * (size_t)((int64_t)M * D32));   /* pads: code 0 */
-    if (frac_out) memset(frac_out, 0, sizeof(float) * (size_t)((int64_t)M * D32));
-    if (u_out) memset(u_out, 0, sizeof(float) * (size_t)((int64_t)M * D32));
+    /* pads: value 0, i.e. code s */
+    for (int64_t i = 0; i < (int64_t)M * D32; ++i) codes[i] = (uint32_t)s;
+    if (x_out) memset(x_out, 0, sizeof(float) * (size_t)((int64_t)M * D32));
+    if (v_out) memset(v_out, 0, sizeof(float) * (size_t)((int64_t)M * D32));
 
     const int64_t total = (int64_t)M * tb.nb;
 #pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
@@ -193,19 +195,17 @@ void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
         for (int64_t e = 0; e < tb.len[k]; ++e) {
             const int64_t j = tb.start[k] + e;
             const float g = grads[m * worker_stride + j];
-            const float a = fabsf(g);
-            float r = a * inv;               /* s * |g_j| / ||g||  (Eq. 6) */
-            r = fminf(r, sf);                /* an ulp above s must not carry into the sign */
-            const float l = floorf(r);
-            const float f = r - l;           /* p_r of Eq. 6, exact in fp32 */
-            const float u = uniform23(seed, step, (uint32_t)m, j);
-            const uint32_t level = (uint32_t)l + (u <= f ? 1u : 0u);   /* up with probability p_r */
-            uint32_t gbits;
-            memcpy(&gbits, &g, sizeof gbits);
-            const uint32_t sign = gbits >> 31;
-            codes[m * D32 + j] = (sign << (b - 1)) | level;
-            if (frac_out) frac_out[m * D32 + j] = f;
-            if (u_out) u_out[m * D32 + j] = u;
+            float r = fabsf(g) * inv;        /* s * |g_j| / ||g||  (Eq. 6), fp32 */
+            r = fminf(r, sf);                /* an ulp above s must stay inside the code range */
+            const float x = copysignf(r, g); /* signed position on the level grid */
+            const float v = uniform16(seed, step, (uint32_t)m, j);
+            /* Eq. 6 on the signed grid: floor(x + v) is the neighbour of x away
+             * from zero with probability p_r = frac(|x|) and the one toward zero
+             * otherwise.  x + v is exact in fp64 (x has 24 bits below 2^15, v 17 bits). */
+            const double q = floor((double)x + (double)v);
+            codes[m * D32 + j] = (uint32_t)((int32_t)q + s);      /* excess-s code, 0 .. 2s */
+            if (x_out) x_out[m * D32 + j] = x;
+            if (v_out) v_out[m * D32 + j] = v;
         }
     }
     free_table(&tb);
@@ -267,10 +267,8 @@ void oracle_dequantize(const uint32_t* codes, const float* norms,
     for (int64_t k = 0; k < tb.nb; ++k) {
         for (int64_t e = 0; e < tb.len[k]; ++e) {
             const int64_t j = tb.start[k] + e;
-            const uint32_t c = codes[j];
-            const double sgn = ((c >> (b - 1)) & 1u) ? -1.0 : 1.0;
-            const double level = (double)(c & (uint32_t)s);
-            values[j] = (s > 0) ? sgn * level * (double)norms[k] / (double)s : 0.0;
+            const double q = (double)codes[j] - (double)s;        /* sgn * level */
+            values[j] = (s > 0) ? q * (double)norms[k] / (double)s : 0.0;
         }
     }
     free_table(&tb);
@@ -296,10 +294,8 @@ void oracle_unpack_dequant_average(const uint32_t* packed, int64_t packed_stride
             const int64_t j = tb.start[k] + e;
             double acc = 0.0;
             for (int32_t m = 0; m < M; ++m) {
-                const uint32_t c = codes[(int64_t)m * D32 + j];
-                const double sgn = ((c >> (b - 1)) & 1u) ? -1.0 : 1.0;
-                const double level = (double)(c & (uint32_t)s);
-                if (s > 0) acc += sgn * level * (double)norms[(int64_t)m * tb.nb + k] / (double)s;
+                const double q = (double)codes[(int64_t)m * D32 + j] - (double)s;     /* sgn * level */
+                if (s > 0) acc += q * (double)norms[(int64_t)m * tb.nb + k] / (double)s;
             }
             out[j] = (float)(acc / (double)M);
         }

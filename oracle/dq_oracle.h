@@ -14,16 +14,17 @@
  *                     formula per bucket)
  *   bucket_norms      ||g||_2 of Eq. 5, per bucket
  *   choose_bits       Eq. 17 with G-bar of Lemma 1, integer b by ceiling
- *   quantize          Eq. 5 and Eq. 6 (stochastic map zeta), s = 2^(b-1)-1
- *   pack / unpack     the "1 sign bit + (b-1) magnitude bits" code of Sec. IV-A,
- *                     concatenated LSB-first into 32-bit words
+ *   quantize          Eq. 5 and Eq. 6 (stochastic map zeta), s = 2^(b-1)-1; the b-bit
+ *                     code of Sec. IV-A (a sign and b-1 bits of zeta) is stored as
+ *                     the single number s + sgn * level in 0 .. 2s
+ *   pack / unpack     b-bit codes concatenated LSB-first into 32-bit words
  *   unpack_dequant_average   Algorithm 1, server step "Average", with Eq. 5
  *   philox4x32_10     Salmon, Moraes, Dror, Shaw, "Parallel random numbers:
  *                     as easy as 1, 2, 3" (SC'11), Philox-4x32 with 10 rounds
  *
  * Pinned by tests/test_oracle_*.py.  Unpinned (the paper leaves it undefined):
- * the b = 1 case (s = 0), read here as "sign bit only, value 0" -- parity
- * unpinned for that case.
+ * the b = 1 case (s = 0), read here as "code 0, value 0" -- parity unpinned
+ * for that case.
  *
  * Layout convention: tensor i with n_i elements starts at padded offset
  * P_i = sum_{j<i} roundup32(n_j); the worker buffer holds D32 = sum roundup32(n_i)
@@ -62,13 +63,14 @@ int32_t oracle_choose_bits(const float* norms, int64_t nb, int32_t M,
 /* ---- Philox4x32-10 ---- */
 void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]);
 
-/* ---- Eq. 5/6: codes (sign << (b-1) | level), one uint32 per padded element.
- *      frac_out / u_out (optional, may be NULL) receive p_r and the uniform
- *      drawn for every element. ---- */
+/* ---- Eq. 5/6: codes s + sgn * level, one uint32 per padded element (s for
+ *      padding).  x_out / v_out (optional, may be NULL) receive the signed
+ *      position x = sgn * s|g|/norm on the level grid and the uniform v drawn
+ *      for every element; the code is floor(x + v) + s. ---- */
 void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
                      const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
                      const float* norms, int32_t b, uint64_t seed, uint32_t step,
-                     uint32_t* codes /*[M][D32]*/, float* frac_out, float* u_out);
+                     uint32_t* codes /*[M][D32]*/, float* x_out, float* v_out);
 
 /* ---- pack / unpack n codes of b bits (n a multiple of 32) ---- */
 void oracle_pack(const uint32_t* codes, int64_t n, int32_t b, uint32_t* words /*[b*n/32]*/);
@@ -80,7 +82,7 @@ void oracle_quantize_pack(const float* grads, int64_t worker_stride, int32_t M,
                           const float* norms, int32_t b, uint64_t seed, uint32_t step,
                           uint32_t* packed, int64_t packed_stride);
 
-/* ---- Eq. 5 inverse for one worker: value = norm * sgn * level / s, in fp64 ---- */
+/* ---- Eq. 5 inverse for one worker: value = norm * (code - s) / s, in fp64 ---- */
 void oracle_dequantize(const uint32_t* codes, const float* norms /*[nb]*/,
                        const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
                        int32_t b, double* values /*[D32]*/);

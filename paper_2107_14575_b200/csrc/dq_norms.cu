@@ -3,71 +3,207 @@
 //
 // One team of LANES threads (8, 16 or a full warp, by bucket size) owns a
 // bucket: 128-bit coalesced loads, four independent fp32 accumulators per
-// lane, a shuffle reduction inside the team.  Teams walk the (worker, bucket)
-// list with a grid stride, so neighbouring teams read neighbouring memory.
-// HBM-bound: 4 bytes read per element, 4/bucket bytes written.
+// lane, a shuffle reduction inside the team.  A warp takes runs of consecutive
+// buckets of one worker (blockIdx.y), so the tensor a bucket belongs to is
+// searched once per run and then followed; neighbouring warps read neighbouring
+// memory.  HBM-bound: 4 bytes read per element, 4/bucket bytes written.
 #include "dq_common.cuh"
 
 namespace {
 
 constexpr int kThreads = 256;
+constexpr int kRun = 8;            // bucket rows a warp handles per run
 
 template <int LANES>
 __global__ void __launch_bounds__(kThreads)
 bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const int64_t worker_stride,
-                    const int M, float* __restrict__ norms, int32_t* __restrict__ status)
+                    float* __restrict__ norms, int32_t* __restrict__ status)
 {
-    constexpr int kTeams = kThreads / LANES;
+    constexpr int kTeamsPerWarp = 32 / LANES;
+    constexpr int kChunk = kRun * kTeamsPerWarp;          // buckets per run
     const int lane = threadIdx.x % LANES;
-    const int64_t total = (int64_t)M * v.nb;
-    const int64_t nteams = (int64_t)gridDim.x * kTeams;
+    const int team = (threadIdx.x % 32) / LANES;
+    const int m = blockIdx.y;
+    const float* gw = grads + (int64_t)m * worker_stride;
+    float* nw = norms + (int64_t)m * v.nb;
+    const int warps_total = gridDim.x * (kThreads / 32);
+    const int nchunks = (v.nb + kChunk - 1) / kChunk;
+    const int bsz = v.groups_per_bucket * 32;
     bool bad = false;
 
-    // The loop bound is the same for every lane of a warp (teams of one warp
-    // take consecutive buckets), so the full-mask shuffles below are safe; a
-    // team past the end runs with an empty bucket.
-    constexpr int kTeamsPerWarp = 32 / LANES;
-    int64_t w0 = (int64_t)blockIdx.x * kTeams + (threadIdx.x / 32) * kTeamsPerWarp;
-    for (; w0 < total; w0 += nteams) {
-        const int64_t w = w0 + (threadIdx.x % 32) / LANES;
-        const bool active = w < total;
-        const int m = active ? (int)(w / v.nb) : 0;
-        const int k = active ? (int)(w - (int64_t)m * v.nb) : 0;
-        int64_t start;
-        int len;
-        bucket_info(v, k, start, len);
-        if (!active) len = 0;
-        const float* g = grads + (int64_t)m * worker_stride + start;   // 128-byte aligned
-        const float4* g4 = reinterpret_cast<const float4*>(g);
-        const int n4 = len >> 2;
-
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        int i = lane;
+    // Every lane of a warp runs the same number of iterations of both loops, so
+    // the full-mask shuffles are safe; a team past the end works on an empty bucket.
+    for (int chunk = blockIdx.x * (kThreads / 32) + threadIdx.x / 32; chunk < nchunks; chunk += warps_total) {
+        int k = chunk * kChunk + team;
+        int seg = 0;
+        if (v.n_seg > 1) seg = last_not_above(v.seg_bucket0, v.n_seg, k < v.nb ? k : v.nb - 1);
 #pragma unroll 1
-        for (; i + 3 * LANES < n4; i += 4 * LANES) {
-            const float4 x0 = __ldg(g4 + i);
-            const float4 x1 = __ldg(g4 + i + LANES);
-            const float4 x2 = __ldg(g4 + i + 2 * LANES);
-            const float4 x3 = __ldg(g4 + i + 3 * LANES);
-            a0 = fmaf(x0.x, x0.x, a0); a1 = fmaf(x0.y, x0.y, a1); a2 = fmaf(x0.z, x0.z, a2); a3 = fmaf(x0.w, x0.w, a3);
-            a0 = fmaf(x1.x, x1.x, a0); a1 = fmaf(x1.y, x1.y, a1); a2 = fmaf(x1.z, x1.z, a2); a3 = fmaf(x1.w, x1.w, a3);
-            a0 = fmaf(x2.x, x2.x, a0); a1 = fmaf(x2.y, x2.y, a1); a2 = fmaf(x2.z, x2.z, a2); a3 = fmaf(x2.w, x2.w, a3);
-            a0 = fmaf(x3.x, x3.x, a0); a1 = fmaf(x3.y, x3.y, a1); a2 = fmaf(x3.z, x3.z, a2); a3 = fmaf(x3.w, x3.w, a3);
-        }
-        for (; i < n4; i += LANES) {
-            const float4 x = __ldg(g4 + i);
-            a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
-        }
-        if (lane < (len & 3)) {                       // ragged tail of the tensor's last bucket
-            const float x = __ldg(g + n4 * 4 + lane);
-            a0 = fmaf(x, x, a0);
-        }
-        float sum = (a0 + a1) + (a2 + a3);
+        for (int r = 0; r < kRun; ++r, k += kTeamsPerWarp) {
+            const bool active = k < v.nb;
+            int len = 0;
+            int64_t start = 0;
+            if (active) {
+                int local, n, g0;
+                if (v.n_seg == 1) {
+                    local = k; n = v.seg0_elems; g0 = 0;
+                } else {
+                    while (k >= __ldg(v.seg_bucket0 + seg + 1)) ++seg;     // buckets only move forward
+                    local = k - __ldg(v.seg_bucket0 + seg);
+                    n = __ldg(v.seg_elems + seg);
+                    g0 = __ldg(v.seg_group0 + seg);
+                }
+                start = (int64_t)g0 * 32 + (int64_t)local * bsz;
+                const int left = n - local * bsz;
+                len = left < bsz ? left : bsz;
+            }
+            const float* g = gw + start;                                   // 128-byte aligned
+            const float4* g4 = reinterpret_cast<const float4*>(g);
+            const int n4 = len >> 2;
+
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            int i = lane;
+#pragma unroll 1
+            for (; i + 3 * LANES < n4; i += 4 * LANES) {
+                const float4 x0 = __ldg(g4 + i);
+                const float4 x1 = __ldg(g4 + i + LANES);
+                const float4 x2 = __ldg(g4 + i + 2 * LANES);
+                const float4 x3 = __ldg(g4 + i + 3 * LANES);
+                a0 = fmaf(x0.x, x0.x, a0); a1 = fmaf(x0.y, x0.y, a1); a2 = fmaf(x0.z, x0.z, a2); a3 = fmaf(x0.w, x0.w, a3);
+                a0 = fmaf(x1.x, x1.x, a0); a1 = fmaf(x1.y, x1.y, a1); a2 = fmaf(x1.z, x1.z, a2); a3 = fmaf(x1.w, x1.w, a3);
+                a0 = fmaf(x2.x, x2.x, a0); a1 = fmaf(x2.y, x2.y, a1); a2 = fmaf(x2.z, x2.z, a2); a3 = fmaf(x2.w, x2.w, a3);
+                a0 = fmaf(x3.x, x3.x, a0); a1 = fmaf(x3.y, x3.y, a1); a2 = fmaf(x3.z, x3.z, a2); a3 = fmaf(x3.w, x3.w, a3);
+            }
+            for (; i < n4; i += LANES) {
+                const float4 x = __ldg(g4 + i);
+                a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+            }
+            if (lane < (len & 3)) {                       // ragged tail of the tensor's last bucket
+                const float x = __ldg(g + n4 * 4 + lane);
+                a0 = fmaf(x, x, a0);
+            }
+            float sum = (a0 + a1) + (a2 + a3);
 #pragma unroll
-        for (int o = LANES / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o, LANES);
-        if (lane == 0 && active) {
-            const float nrm = sqrtf(sum);
-            norms[w] = nrm;
+            for (int o = LANES / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o, LANES);
+            if (lane == 0 && active) {
+                const float nrm = sqrtf(sum);
+                nw[k] = nrm;
+                bad |= !isfinite(nrm);
+            }
+        }
+    }
+    if (bad) atomicOr(status, DQ_STAT_NONFINITE);
+}
+
+// Full-warp variant for buckets of at least 128 elements.  A warp takes a run of
+// eight consecutive buckets: it first works out where each of them lies (so
+// that table lookups never sit between a load and its use), then streams the
+// eight buckets with independent accumulators, and finally reduces the eight
+// per-lane sums together with a butterfly that halves the number of live
+// values at each of its first three steps (9 shuffles instead of 40).
+__global__ void __launch_bounds__(kThreads)
+bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, const int64_t worker_stride,
+                         float* __restrict__ norms, int32_t* __restrict__ status)
+{
+    extern __shared__ int32_t tbl_s[];
+    const int lane = threadIdx.x & 31;
+    const int m = blockIdx.y;
+    const float4* gw4 = reinterpret_cast<const float4*>(grads + (int64_t)m * worker_stride);
+    const float* gw = grads + (int64_t)m * worker_stride;
+    float* nw = norms + (int64_t)m * v.nb;
+    const int warps_total = gridDim.x * (kThreads / 32);
+    const int nchunks = (v.nb + kRun - 1) / kRun;
+    const int bsz = v.groups_per_bucket * 32;
+    const int n1 = v.n_seg + 1;
+    bool bad = false;
+
+    const int32_t* tbl = v.seg_group0;                 // [group0 | bucket0 | elems], n_seg + 1 entries each
+    if (v.n_seg > 1 && 3 * n1 * 4 <= 12 * 1024) {
+        for (int i = threadIdx.x; i < 3 * n1; i += kThreads) tbl_s[i] = __ldg(v.seg_group0 + i);
+        __syncthreads();
+        tbl = tbl_s;
+    }
+
+    for (int chunk = blockIdx.x * (kThreads / 32) + threadIdx.x / 32; chunk < nchunks; chunk += warps_total) {
+        const int k0 = chunk * kRun;
+        int first[kRun], len[kRun];                    // first float4 and valid elements of each bucket
+        {
+            int seg = 0;
+            if (v.n_seg > 1) {                         // binary search for the run's first bucket
+                int lo = 0, hi = v.n_seg;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (tbl[n1 + mid] <= k0) lo = mid; else hi = mid;
+                }
+                seg = lo;
+            }
+#pragma unroll
+            for (int r = 0; r < kRun; ++r) {
+                const int k = k0 + r;
+                first[r] = 0;
+                len[r] = 0;
+                if (k < v.nb) {
+                    int local, n, g0;
+                    if (v.n_seg == 1) {
+                        local = k; n = v.seg0_elems; g0 = 0;
+                    } else {
+                        while (k >= tbl[n1 + seg + 1]) ++seg;
+                        local = k - tbl[n1 + seg];
+                        n = tbl[2 * n1 + seg];
+                        g0 = tbl[seg];
+                    }
+                    first[r] = (g0 + local * v.groups_per_bucket) * 8;
+                    const int left = n - local * bsz;
+                    len[r] = left < bsz ? left : bsz;
+                }
+            }
+        }
+        float part[kRun];
+#pragma unroll
+        for (int r = 0; r < kRun; ++r) {
+            const float4* g4 = gw4 + first[r];
+            const int n4 = len[r] >> 2;
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            for (int i = lane; i < n4; i += 128) {
+                const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 x0 = __ldg(g4 + i);
+                const float4 x1 = (i + 32 < n4) ? __ldg(g4 + i + 32) : z;
+                const float4 x2 = (i + 64 < n4) ? __ldg(g4 + i + 64) : z;
+                const float4 x3 = (i + 96 < n4) ? __ldg(g4 + i + 96) : z;
+                a0 = fmaf(x0.x, x0.x, a0); a1 = fmaf(x0.y, x0.y, a1); a2 = fmaf(x0.z, x0.z, a2); a3 = fmaf(x0.w, x0.w, a3);
+                a0 = fmaf(x1.x, x1.x, a0); a1 = fmaf(x1.y, x1.y, a1); a2 = fmaf(x1.z, x1.z, a2); a3 = fmaf(x1.w, x1.w, a3);
+                a0 = fmaf(x2.x, x2.x, a0); a1 = fmaf(x2.y, x2.y, a1); a2 = fmaf(x2.z, x2.z, a2); a3 = fmaf(x2.w, x2.w, a3);
+                a0 = fmaf(x3.x, x3.x, a0); a1 = fmaf(x3.y, x3.y, a1); a2 = fmaf(x3.z, x3.z, a2); a3 = fmaf(x3.w, x3.w, a3);
+            }
+            if (lane < (len[r] & 3)) {                 // ragged tail of a tensor's last bucket
+                const float x = __ldg(gw + (int64_t)first[r] * 4 + n4 * 4 + lane);
+                a0 = fmaf(x, x, a0);
+            }
+            part[r] = (a0 + a1) + (a2 + a3);
+        }
+        // butterfly: after the three halving steps lane l holds bucket (l & 7) summed over its octet
+        float q[4], h[2], t;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float keep = (lane & 1) ? part[2 * i + 1] : part[2 * i];
+            const float give = (lane & 1) ? part[2 * i] : part[2 * i + 1];
+            q[i] = keep + __shfl_xor_sync(0xffffffffu, give, 1);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const float keep = (lane & 2) ? q[2 * i + 1] : q[2 * i];
+            const float give = (lane & 2) ? q[2 * i] : q[2 * i + 1];
+            h[i] = keep + __shfl_xor_sync(0xffffffffu, give, 2);
+        }
+        {
+            const float keep = (lane & 4) ? h[1] : h[0];
+            const float give = (lane & 4) ? h[0] : h[1];
+            t = keep + __shfl_xor_sync(0xffffffffu, give, 4);
+        }
+        t += __shfl_xor_sync(0xffffffffu, t, 8);
+        t += __shfl_xor_sync(0xffffffffu, t, 16);
+        if (lane < kRun && k0 + lane < v.nb) {
+            const float nrm = sqrtf(t);
+            nw[k0 + lane] = nrm;
             bad |= !isfinite(nrm);
         }
     }
@@ -88,20 +224,25 @@ extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int
     if (M > 1 && worker_stride_elems < L->padded && worker_stride_elems != 0) return DQ_ERR_RANGE;
 
     const LayoutView v = make_view(L);
-    const int64_t total = (int64_t)M * L->nb;
     const int lanes = L->bucket >= 128 ? 32 : (L->bucket >= 64 ? 16 : 8);
-    const int teams = kThreads / lanes;
-    int64_t blocks = (total + teams - 1) / teams;
-    const int64_t cap = (int64_t)dq_sm_count() * 8;     // 8 resident CTAs of 256 threads per SM
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
+    const int64_t chunk = (int64_t)kRun * (32 / lanes);
+    const int64_t nchunks = (L->nb + chunk - 1) / chunk;
+    int64_t bx = (nchunks + kThreads / 32 - 1) / (kThreads / 32);
+    // about 8 resident CTAs of 256 threads per SM over all workers
+    int64_t cap = ((int64_t)dq_sm_count() * 8 + M - 1) / M;
+    if (cap < 1) cap = 1;
+    if (bx > cap) bx = cap;
+    if (bx < 1) bx = 1;
+    const dim3 grid((unsigned)bx, (unsigned)M);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (lanes == 32)
-        bucket_norms_kernel<32><<<(unsigned)blocks, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, M, dev_norms, dev_status);
+    if (lanes == 32) {
+        const size_t smem = (L->n_seg > 1 && (size_t)3 * (L->n_seg + 1) * 4 <= 12 * 1024) ? (size_t)3 * (L->n_seg + 1) * 4 : 0;
+        bucket_norms_warp_kernel<<<grid, kThreads, smem, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+    }
     else if (lanes == 16)
-        bucket_norms_kernel<16><<<(unsigned)blocks, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, M, dev_norms, dev_status);
+        bucket_norms_kernel<16><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
     else
-        bucket_norms_kernel<8><<<(unsigned)blocks, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, M, dev_norms, dev_status);
+        bucket_norms_kernel<8><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }

@@ -1,27 +1,59 @@
 // dq_quantize_pack: the EWU quantizer of Eq. 5/6 fused with the b-bit packer.
 //
-// A thread owns one 32-element group: it reads the group's 128 bytes, draws the
-// eight Philox blocks that cover it, encodes the 32 codes and assembles the
-// group's b words in registers (all shifts are constants once b is known), so
-// no code ever leaves the register file before it is packed.  b is read from
-// device memory and selects one of sixteen specialisations with a
-// grid-uniform switch; nothing on the host depends on b.
+// Persistent CTAs walk tiles of 128 groups (one group = 32 consecutive padded
+// elements = one thread).  A tile's 16 KB of gradients arrive by one TMA tensor
+// copy into a ring of shared-memory stages written with the 128-byte
+// swizzle, so that a thread reading its own 128-byte row in 16-byte pieces
+// hits every bank group once per quarter warp.  The thread draws the eight
+// Philox blocks of its group, encodes the 32 codes and assembles the group's
+// b words in a register shift chain (all shifts are constants once b is
+// known).  Each warp transposes its 32*b words through shared memory and writes
+// them with 16-byte coalesced stores.  b is read from device memory and selects
+// one of sixteen specialisations with a grid-uniform switch.
 // HBM traffic: 4 bytes read and b/8 bytes written per element.
 #include "dq_common.cuh"
 #include "dq_device.cuh"
+#include "dq_tma.cuh"
 
 namespace {
 
-constexpr int kThreads = 128;
+constexpr int kThreads = 128;               // groups per tile
+constexpr int kWarps = kThreads / 32;
+constexpr int kStages = 2;
+constexpr int kTileBytes = kThreads * 128;  // 16 KB of fp32 per tile
+constexpr int kMaxSmemSegs = 1023;          // layouts with more tensors read the table from global memory
 
-template <int B>
-__device__ __forceinline__ void store_words(uint32_t* __restrict__ dst, const uint32_t (&acc)[B])
+struct QuantizeArgs {
+    LayoutView v;
+    const float* norms;
+    const int32_t* dev_b;
+    uint32_t* packed;
+    int64_t packed_stride;
+    int32_t* status;
+    PhiloxKeys keys;
+    uint32_t step;
+    int32_t M;
+    int32_t map_has_worker_dim;   // 0 when all workers read the same buffer (stride 0)
+    uint32_t div_magic;           // groups_per_bucket: division by multiply-shift, or by shift if a power of two
+    int32_t div_shift;            // >= 0: power of two, shift; < 0: use div_magic with a 33-bit shift
+};
+
+__device__ __forceinline__ uint32_t div_gpb(const QuantizeArgs& a, uint32_t n)
 {
-    if (B % 4 == 0) {
+    if (a.div_shift >= 0) return n >> a.div_shift;
+    return (uint32_t)(((uint64_t)n * a.div_magic) >> 33);     // exact for n < 2^26, divisor <= 128
+}
+
+// Stores the B words of one group into the warp's staging area (stride B words
+// between lanes; the widest access the alignment allows keeps bank conflicts low).
+template <int B>
+__device__ __forceinline__ void stage_words(uint32_t* __restrict__ dst, const uint32_t (&acc)[B])
+{
+    if constexpr (B % 4 == 0) {
 #pragma unroll
         for (int i = 0; i < B / 4; ++i)
             reinterpret_cast<uint4*>(dst)[i] = make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
-    } else if (B % 2 == 0) {
+    } else if constexpr (B % 2 == 0) {
 #pragma unroll
         for (int i = 0; i < B / 2; ++i)
             reinterpret_cast<uint2*>(dst)[i] = make_uint2(acc[2 * i], acc[2 * i + 1]);
@@ -31,84 +63,179 @@ __device__ __forceinline__ void store_words(uint32_t* __restrict__ dst, const ui
     }
 }
 
-// Encodes chunk C (elements 4C..4C+3) of a group and ORs the codes into acc.
 template <int B, int C>
-__device__ __forceinline__ void encode_chunk(uint32_t (&acc)[B], const float4 x, const float inv, const float sf,
-                                             const uint32_t q, const uint32_t m, const uint32_t step,
+__device__ __forceinline__ void encode_chunk(uint32_t (&acc)[B], uint32_t& cur, const float4 x, const float inv,
+                                             const float sf, const uint32_t q, const uint32_t m, const uint32_t step,
                                              const PhiloxKeys& keys)
 {
     uint32_t w[4] = {0u, 0u, 0u, 0u};
-    if (B > 1) philox4x32_10(q, 0u, m, step, keys, w);
-    put_code<B, 4 * C + 0>(acc, encode<B>(x.x, inv, sf, w[0]));
-    put_code<B, 4 * C + 1>(acc, encode<B>(x.y, inv, sf, w[1]));
-    put_code<B, 4 * C + 2>(acc, encode<B>(x.z, inv, sf, w[2]));
-    put_code<B, 4 * C + 3>(acc, encode<B>(x.w, inv, sf, w[3]));
+    if constexpr (B > 1) philox4x32_10(q, 0u, m, step, keys, w);
+    push_code<B, 4 * C + 0>(acc, cur, encode<B>(x.x, inv, sf, w[0]));
+    push_code<B, 4 * C + 1>(acc, cur, encode<B>(x.y, inv, sf, w[1]));
+    push_code<B, 4 * C + 2>(acc, cur, encode<B>(x.z, inv, sf, w[2]));
+    push_code<B, 4 * C + 3>(acc, cur, encode<B>(x.w, inv, sf, w[3]));
 }
 
 template <int B>
-__device__ __forceinline__ void quantize_groups(const LayoutView& v, const float* __restrict__ grads,
-                                                const int64_t worker_stride, const int M,
-                                                const float* __restrict__ norms, const PhiloxKeys& keys,
-                                                const uint32_t step, uint32_t* __restrict__ packed,
-                                                const int64_t packed_stride)
+__device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUtensorMap* map, unsigned char* tiles,
+                                               uint32_t* out_stage, uint64_t* full, const int32_t* tbl)
 {
     constexpr int s = (1 << (B - 1)) - 1;
     const float sf = (float)s;
-    const int64_t total = (int64_t)M * v.total_groups;
-    const int64_t nthreads = (int64_t)gridDim.x * blockDim.x;
-    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += nthreads) {
-        const int m = (int)(idx / v.total_groups);
-        const int g = (int)(idx - (int64_t)m * v.total_groups);
-        int bucket, valid;
-        group_info(v, g, bucket, valid);
-        const float4* row = reinterpret_cast<const float4*>(grads + (int64_t)m * worker_stride + (int64_t)g * 32);
-        float4 x[8];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = a.v.total_groups;
+    const int tiles_per_worker = (G + kThreads - 1) / kThreads;
+    const int total_tiles = a.M * tiles_per_worker;
+    const int n1 = a.v.n_seg + 1;
+    uint32_t* my_out = out_stage + warp * (32 * B);
+
+    // prologue: fill the ring
+    if (tid == 0) {
 #pragma unroll
-        for (int c = 0; c < 8; ++c) x[c] = __ldg(row + c);
-        const float norm = __ldg(norms + (int64_t)m * v.nb + bucket);
+        for (int st = 0; st < kStages; ++st) {
+            const int tile = blockIdx.x + st * gridDim.x;
+            if (tile < total_tiles) {
+                const int m = tile / tiles_per_worker;
+                const int row0 = (tile - m * tiles_per_worker) * kThreads;
+                tma::mbar_expect_tx(&full[st], kTileBytes);
+                tma::load_tile_3d(tiles + st * kTileBytes, map, &full[st], 0, row0, a.map_has_worker_dim ? m : 0);
+            }
+        }
+    }
+
+    int seg = 0, seg_m = -1;
+    int it = 0;
+    bool timed_out = false;
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+        const int st = it % kStages;
+        const uint32_t parity = (it / kStages) & 1;
+        const int m = tile / tiles_per_worker;
+        const int row0 = (tile - m * tiles_per_worker) * kThreads;
+        const int g = row0 + tid;
+        const bool active = g < G;
+
+        // where this group lives: tensor, bucket, valid elements (independent of the tile's data)
+        int bucket = 0, valid = 32;
+        if (active) {
+            int local, n, b0;
+            if (a.v.n_seg == 1) {
+                local = g; n = a.v.seg0_elems; b0 = 0;
+            } else {
+                if (m != seg_m) { seg = 0; seg_m = m; }
+                while (g >= tbl[seg + 1]) ++seg;                 // groups only move forward within a worker
+                local = g - tbl[seg];
+                b0 = tbl[n1 + seg];
+                n = tbl[2 * n1 + seg];
+            }
+            bucket = b0 + (int)div_gpb(a, (uint32_t)local);
+            const int left = n - local * 32;
+            valid = left < 32 ? left : 32;
+        }
+        const float norm = active ? __ldg(a.norms + (int64_t)m * a.v.nb + bucket) : 0.0f;
         const float inv = (norm >= 0x1p-100f) ? __fdiv_rn(sf, norm) : 0.0f;
-        if (valid < 32) {                      // padding after a tensor's end encodes as +0
-            float* xe = reinterpret_cast<float*>(x);
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-                if (e >= valid) xe[e] = 0.0f;
+
+        if (!tma::mbar_wait(&full[st], parity)) { timed_out = true; break; }
+
+        unsigned char* row = tiles + st * kTileBytes + tid * 128;
+        if (valid < 32) {                       // padding after a tensor's end encodes as +0
+            for (int e = valid; e < 32; ++e)
+                *reinterpret_cast<float*>(row + ((((e >> 2) ^ (tid & 7)) << 4) | ((e & 3) << 2))) = 0.0f;
+            tma::fence_proxy_async();           // these stores precede the next bulk copy into this stage
         }
         uint32_t acc[B];
+        uint32_t cur = 0;
         const uint32_t q0 = (uint32_t)g * 8u;
-        encode_chunk<B, 0>(acc, x[0], inv, sf, q0 + 0, m, step, keys);
-        encode_chunk<B, 1>(acc, x[1], inv, sf, q0 + 1, m, step, keys);
-        encode_chunk<B, 2>(acc, x[2], inv, sf, q0 + 2, m, step, keys);
-        encode_chunk<B, 3>(acc, x[3], inv, sf, q0 + 3, m, step, keys);
-        encode_chunk<B, 4>(acc, x[4], inv, sf, q0 + 4, m, step, keys);
-        encode_chunk<B, 5>(acc, x[5], inv, sf, q0 + 5, m, step, keys);
-        encode_chunk<B, 6>(acc, x[6], inv, sf, q0 + 6, m, step, keys);
-        encode_chunk<B, 7>(acc, x[7], inv, sf, q0 + 7, m, step, keys);
-        store_words<B>(packed + (int64_t)m * packed_stride + (int64_t)g * B, acc);
+        const uint32_t sw = (uint32_t)(tid & 7);
+#define DQ_CHUNK(C)                                                                                        \
+        encode_chunk<B, C>(acc, cur, *reinterpret_cast<const float4*>(row + (((uint32_t)(C) ^ sw) << 4)), \
+                           inv, sf, q0 + (C), (uint32_t)m, a.step, a.keys);
+        DQ_CHUNK(0) DQ_CHUNK(1) DQ_CHUNK(2) DQ_CHUNK(3) DQ_CHUNK(4) DQ_CHUNK(5) DQ_CHUNK(6) DQ_CHUNK(7)
+#undef DQ_CHUNK
+
+        // transpose the warp's 32*B words through shared memory, then coalesced 16-byte stores
+        stage_words<B>(my_out + lane * B, acc);
+        __syncwarp();
+        const int g_warp = row0 + warp * 32;
+        int ng = G - g_warp;
+        ng = ng < 0 ? 0 : (ng > 32 ? 32 : ng);
+        const int nwords = ng * B;
+        uint32_t* dst = a.packed + (int64_t)m * a.packed_stride + (int64_t)g_warp * B;
+        const int n4 = nwords >> 2;
+        for (int i = lane; i < n4; i += 32)
+            reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(my_out)[i];
+        if (lane < (nwords & 3)) dst[n4 * 4 + lane] = my_out[n4 * 4 + lane];
+
+        // everyone is done with this stage (and with the staging area): refill it
+        __syncthreads();
+        if (tid == 0) {
+            const int next = tile + kStages * gridDim.x;
+            if (next < total_tiles) {
+                const int nm = next / tiles_per_worker;
+                const int nrow0 = (next - nm * tiles_per_worker) * kThreads;
+                tma::fence_proxy_async();
+                tma::mbar_expect_tx(&full[st], kTileBytes);
+                tma::load_tile_3d(tiles + st * kTileBytes, map, &full[st], 0, nrow0, a.map_has_worker_dim ? nm : 0);
+            }
+        }
+    }
+
+    if (timed_out) {
+        if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
+        // give copies still in flight a bounded chance to land before the CTA's shared memory is released
+        for (int k = 1; k < kStages; ++k) {
+            const int j = it + k;
+            if (blockIdx.x + (int64_t)j * gridDim.x < total_tiles) (void)tma::mbar_wait(&full[j % kStages], (j / kStages) & 1);
+        }
     }
 }
 
-__global__ void __launch_bounds__(kThreads)
-quantize_pack_kernel(const LayoutView v, const float* __restrict__ grads, const int64_t worker_stride, const int M,
-                     const float* __restrict__ norms, const int32_t* __restrict__ dev_b,
-                     const __grid_constant__ PhiloxKeys keys, const uint32_t step,
-                     uint32_t* __restrict__ packed, const int64_t packed_stride, int32_t* __restrict__ status)
+__global__ void __launch_bounds__(kThreads, 5)
+quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_constant__ CUtensorMap map)
 {
-    const int b = __ldg(dev_b);
+    extern __shared__ unsigned char smem_raw[];
+    // [tiles: kStages * 16 KB, 1024-byte aligned][output staging: kWarps * 32 * 16 words][barriers][table]
+    unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint32_t* out_stage = reinterpret_cast<uint32_t*>(tiles + kStages * kTileBytes);
+    uint64_t* full = reinterpret_cast<uint64_t*>(out_stage + kWarps * 32 * DQ_MAX_BITS);
+    int32_t* tbl_s = reinterpret_cast<int32_t*>(full + kStages);
+
+    const int b = __ldg(a.dev_b);
     if (b < 1 || b > DQ_MAX_BITS) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(status, DQ_STAT_BAD_BITS);
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
         return;
     }
-    if ((int64_t)b * v.total_groups > packed_stride) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(status, DQ_STAT_CAPACITY);
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
         return;
     }
+
+    const int32_t* tbl = a.v.seg_group0;
+    if (a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs) {
+        for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
+        tbl = tbl_s;
+    }
+    if (threadIdx.x == 0) {
+        tma::prefetch_tensor_map(&map);
+#pragma unroll
+        for (int st = 0; st < kStages; ++st) tma::mbar_init(&full[st], 1);
+        tma::fence_barrier_init();
+    }
+    __syncthreads();
+
     switch (b) {
-#define DQ_CASE(BB) case BB: quantize_groups<BB>(v, grads, worker_stride, M, norms, keys, step, packed, packed_stride); break;
+#define DQ_CASE(BB) case BB: quantize_tiles<BB>(a, &map, tiles, out_stage, full, tbl); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
         default: break;
     }
+}
+
+size_t smem_bytes(int n_seg)
+{
+    size_t n = 1024 + (size_t)kStages * kTileBytes + (size_t)kWarps * 32 * DQ_MAX_BITS * 4 + kStages * 8;
+    if (n_seg > 1 && n_seg <= kMaxSmemSegs) n += (size_t)3 * (n_seg + 1) * 4;
+    return n;
 }
 
 }  // namespace
@@ -129,15 +256,47 @@ extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, in
     if (M > 1 && worker_stride_elems < L->padded && worker_stride_elems != 0) return DQ_ERR_RANGE;
     if (packed_stride_words < L->padded / 32) return DQ_ERR_RANGE;   // not even b = 1 fits
 
-    const LayoutView v = make_view(L);
-    const PhiloxKeys keys = make_philox_keys(seed);
-    const int64_t total = (int64_t)M * v.total_groups;
-    int64_t blocks = (total + kThreads - 1) / kThreads;
-    const int64_t cap = (int64_t)dq_sm_count() * 8;
-    if (blocks > cap) blocks = cap;
-    quantize_pack_kernel<<<(unsigned)blocks, kThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        v, dev_grads, worker_stride_elems, M, dev_norms, dev_b, keys, step, dev_packed, packed_stride_words,
-        dev_status);
+    QuantizeArgs a;
+    a.v = make_view(L);
+    a.norms = dev_norms;
+    a.dev_b = dev_b;
+    a.packed = dev_packed;
+    a.packed_stride = packed_stride_words;
+    a.status = dev_status;
+    a.keys = make_philox_keys(seed);
+    a.step = step;
+    a.M = M;
+    const bool worker_dim = (M > 1 && worker_stride_elems != 0);
+    a.map_has_worker_dim = worker_dim ? 1 : 0;
+    const uint32_t gpb = (uint32_t)a.v.groups_per_bucket;
+    if ((gpb & (gpb - 1)) == 0) {
+        a.div_shift = 0;
+        while ((1u << a.div_shift) < gpb) ++a.div_shift;
+        a.div_magic = 0;
+    } else {
+        a.div_shift = -1;
+        a.div_magic = (uint32_t)(((uint64_t(1) << 33) + gpb - 1) / gpb);
+    }
+
+    // tensor map over the gradients: [worker][group][32 floats], box = one tile of 128 groups
+    CUtensorMap map;
+    const uint64_t dims[3] = {32, (uint64_t)a.v.total_groups, worker_dim ? (uint64_t)M : 1};
+    const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
+    const uint32_t box[3] = {32, (uint32_t)kThreads, 1};
+    if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
+                              CU_TENSOR_MAP_SWIZZLE_128B))
+        return DQ_ERR_CUDA;
+
+    const size_t smem = smem_bytes(L->n_seg);
+    // raising the dynamic shared-memory limit is per device and idempotent
+    if (cudaFuncSetAttribute(quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DQ_ERR_CUDA;
+    }
+    const int64_t tiles = (int64_t)M * ((a.v.total_groups + kThreads - 1) / kThreads);
+    int64_t blocks = (int64_t)dq_sm_count() * 5;       // five 42 KB CTAs fit one SM
+    if (blocks > tiles) blocks = tiles;
+    quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem, static_cast<cudaStream_t>(stream)>>>(a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }

@@ -121,20 +121,21 @@ def test_philox_counter_and_key_separation():
     assert not np.array_equal(oracle.philox4x32_10([5, 0, 2, 3], [7, 10]), base)
 
 
-def test_uniform_is_philox_word_of_the_element():
-    # element j of worker m at a step draws word (j & 3) of the block with counter
-    # (j >> 2, 0, m, step) and key (seed lo, seed hi); with k its top 23 bits,
-    # u = 1 - (2k + 1) / 2^24
+def test_uniform_is_philox_half_word_of_the_element():
+    # element j of worker m at a step draws from the block with counter (j >> 3, 0, m, step)
+    # and key (seed lo, seed hi): half (j & 1) of word ((j >> 1) & 3), low half first;
+    # with k that 16-bit value, v = (2k + 1) / 2^17
     lay = oracle.Layout([64], 32)
     g = np.ones((3, 64), np.float32)
     norms = oracle.bucket_norms(lay, g)
     seed, step = (0xDEADBEEF << 32) | 0x12345678, 77
-    _, _, u = oracle.quantize(lay, g, norms, 4, seed, step, want_frac_u=True)
+    _, _, v = oracle.quantize(lay, g, norms, 4, seed, step, want_x_v=True)
     for m in range(3):
-        for j in (0, 1, 5, 31, 32, 63):
-            blk = oracle.philox4x32_10([j >> 2, 0, m, step], [0x12345678, 0xDEADBEEF])
-            k = int(blk[j & 3]) >> 9
-            assert float(u[m, j]) == 1.0 - (2 * k + 1) / 2.0 ** 24
+        for j in (0, 1, 2, 5, 7, 8, 31, 32, 63):
+            blk = oracle.philox4x32_10([j >> 3, 0, m, step], [0x12345678, 0xDEADBEEF])
+            word = int(blk[(j >> 1) & 3])
+            k = (word >> 16) if (j & 1) else (word & 0xFFFF)
+            assert float(v[m, j]) == (2 * k + 1) / 2.0 ** 17
 
 
 def test_uniform_statistics():
@@ -142,11 +143,11 @@ def test_uniform_statistics():
     lay = oracle.Layout([1 << 20], 4096)
     g = np.ones((4, 1 << 20), np.float32)
     norms = oracle.bucket_norms(lay, g)
-    _, _, u = oracle.quantize(lay, g, norms, 4, 123, 0, want_frac_u=True)
+    _, _, u = oracle.quantize(lay, g, norms, 4, 123, 0, want_x_v=True)
     u = u.ravel().astype(np.float64)
     n = u.size
     assert u.min() > 0.0 and u.max() < 1.0
-    assert np.all((u * 2 ** 24) % 2 == 1)                   # odd multiples of 2^-24: the midpoint grid
+    assert np.all((u * 2 ** 17) % 2 == 1)                   # odd multiples of 2^-17: the midpoint grid
     assert abs(u.mean() - 0.5) < 5 * math.sqrt(1 / 12 / n)
     counts = np.bincount((u * 256).astype(np.int64), minlength=256)
     chi2 = ((counts - n / 256) ** 2 / (n / 256)).sum()

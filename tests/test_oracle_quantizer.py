@@ -15,11 +15,10 @@ from paper_2107_14575_b200 import workloads as W
 
 
 def _values(codes, norm, b):
-    """Eq. 5 written out with numpy for one bucket: norm * sgn * level / s."""
+    """Eq. 5 written out with numpy for one bucket: norm * sgn * level / s,
+    with the code holding s + sgn * level."""
     s = (1 << (b - 1)) - 1
-    level = (codes & np.uint32(s)).astype(np.float64)
-    sgn = 1.0 - 2.0 * ((codes >> np.uint32(b - 1)) & 1).astype(np.float64)
-    return sgn * level * float(norm) / s
+    return (codes.astype(np.float64) - s) * float(norm) / s
 
 
 # ----------------------------------------------------------------- norms (P6)
@@ -69,12 +68,10 @@ def test_on_level_inputs_are_reproduced_exactly(b):
         norms = oracle.bucket_norms(lay, v)
         assert norms[0, 0] == np.float32(s * c)
         for seed in range(20):
-            codes, frac, u = oracle.quantize(lay, v, norms, b, seed, 7, want_frac_u=True)
-            assert np.all(frac == 0.0)
-            assert ((codes[0, :3] & s) == L).all()
-            nz = L != 0
-            assert (((codes[0, :3] >> (b - 1)) & 1)[nz] == (signs < 0)[nz]).all()
-            assert np.all(codes[0, 3:] == 0)                       # pads
+            codes, x, u = oracle.quantize(lay, v, norms, b, seed, 7, want_x_v=True)
+            assert np.array_equal(x[0, :3], (signs * L).astype(np.float32))   # exactly on the grid
+            assert np.array_equal(codes[0, :3].astype(np.int64), s + signs * L)
+            assert np.all(codes[0, 3:] == s)                       # pads hold the code of 0
             q = oracle.dequantize(lay, codes[0], norms[0], b)
             assert np.array_equal(q[:3], v[0, :3].astype(np.float64))
 
@@ -87,24 +84,38 @@ def test_signed_zero_and_zero_norm_bucket():
     v[0, 33] = -4.0
     norms = oracle.bucket_norms(lay, v)
     assert norms.tolist() == [[0.0, 5.0]]
-    b = 5                                   # s = 15: 3/5 and 4/5 lie on levels 9 and 12
+    b, s = 5, 15                            # 3/5 and 4/5 lie on levels 9 and 12
     codes = oracle.quantize(lay, v, norms, b, 11, 0)
-    assert codes[0, 0] == 0 and codes[0, 1] == 1 << (b - 1)       # -0.0 keeps its sign bit, level 0
-    assert codes[0, 32] == 9 and codes[0, 33] == (1 << (b - 1)) | 12
+    assert codes[0, 0] == s and codes[0, 1] == s                   # zeros of either sign: code of 0
+    assert codes[0, 32] == s + 9 and codes[0, 33] == s - 12
+    assert np.all(codes[0, 2:32] == s)                             # a zero-norm bucket quantizes to 0
     q = oracle.dequantize(lay, codes[0], norms[0], b)
     assert q[0] == 0 and q[1] == 0 and q[32] == 3.0 and q[33] == -4.0
 
 
-def test_b1_is_sign_only():
-    # b = 1: s = 0, the paper's map is undefined; reading: sign bit only, value 0
+def test_b1_carries_nothing():
+    # b = 1: s = 0, the paper's map is undefined; reading: code 0, value 0
     lay = oracle.Layout([40], 32)
     rng = np.random.default_rng(5)
     v = rng.standard_normal((2, 64)).astype(np.float32)
     norms = oracle.bucket_norms(lay, v)
     codes = oracle.quantize(lay, v, norms, 1, 1, 1)
-    assert np.array_equal(codes[:, :40], (v[:, :40] < 0).astype(np.uint32))
+    assert np.all(codes == 0)
     packed = oracle.quantize_pack(lay, v, norms, 1, 1, 1)
     assert np.all(oracle.unpack_dequant_average(lay, packed, norms, 1) == 0)
+
+
+def test_code_range():
+    # codes live in 0 .. 2s, so they fit b bits and the all-ones pattern never occurs
+    w = W.config_flat(d=4096, M=2, bucket=128, sigma=1.0)
+    lay = oracle.Layout(w.segments, w.bucket)
+    g = W.make_grads(w, lay.offsets, lay.D32)
+    norms = oracle.bucket_norms(lay, g)
+    for b in (2, 3, 8, 16):
+        s = (1 << (b - 1)) - 1
+        codes = oracle.quantize(lay, g, norms, b, 3, 4)
+        assert codes.min() >= 0 and codes.max() <= 2 * s
+        assert np.array_equal(codes > s, (g > 0) & (codes != s))   # the side of s is the sign
 
 
 # --------------------------------------- brute force over all outcomes (P3 i)
@@ -119,21 +130,24 @@ def test_exact_expectation_by_enumeration(b, d):
     lay = oracle.Layout([d], 32)
     norms = oracle.bucket_norms(lay, v)
     norm = float(norms[0, 0])
-    codes, frac, u = oracle.quantize(lay, v, norms, b, 42, 0, want_frac_u=True)
-    codes, frac, u = codes[0, :d], frac[0, :d].astype(np.float64), u[0, :d]
-    # the oracle's p_r against the definition p_r = s|g|/||g|| - l in fp64
+    codes, x, u = oracle.quantize(lay, v, norms, b, 42, 0, want_x_v=True)
+    codes, x, u = codes[0, :d].astype(np.int64), x[0, :d].astype(np.float64), u[0, :d].astype(np.float64)
+    # the oracle's position on the level grid against the definition sgn * s|g|/||g|| in fp64
     r = s * np.abs(v[0, :d].astype(np.float64)) / norm
-    assert np.allclose(frac, r - np.floor(r), atol=4e-7 * max(1.0, s))
-    low = (codes & s) - (u <= frac.astype(np.float32))           # floor level l
-    assert np.array_equal(low, np.floor(r).astype(np.int64)) or np.all(np.abs(r - np.round(r)) < 1e-5)
-    sign = codes & (1 << (b - 1))
+    assert np.allclose(x, np.sign(v[0, :d]) * r, atol=4e-7 * max(1.0, s))
+    sgn = np.where(x < 0, -1, 1)
+    low = np.floor(np.abs(x)).astype(np.int64)                   # level l toward zero
+    frac = np.abs(x) - low                                       # p_r of Eq. 6
+    # the drawn code is one of the two neighbours of x, chosen by floor(x + v)
+    assert np.array_equal(codes - s, np.floor(x + u).astype(np.int64))
+    assert np.all(np.isin(codes - s - sgn * low, (0, 1, -1)))
     mean = np.zeros(d)
     var = np.zeros(d)
     total = 0.0
     for ups in itertools.product((0, 1), repeat=d):
         ups = np.array(ups)
         p = np.prod(np.where(ups == 1, frac, 1.0 - frac))
-        q = _values((sign | (low + ups)).astype(np.uint32), norms[0, 0], b)
+        q = _values((s + sgn * (low + ups)).astype(np.uint32), norms[0, 0], b)
         total += p
         mean += p * q
         var += p * q * q
@@ -274,7 +288,7 @@ def test_average_matches_numpy_definition():
             st, ln = lay.bucket_start[k], lay.bucket_len[k]
             per_elem[st: st + ln] = norms[m, k]
         s = (1 << (b - 1)) - 1
-        acc += (1.0 - 2.0 * ((codes[m] >> (b - 1)) & 1)) * (codes[m] & s) * per_elem / s
+        acc += (codes[m].astype(np.float64) - s) * per_elem / s
     assert np.allclose(out, acc / w.M, rtol=1e-6, atol=1e-12)
     # the averaged quantized gradient is close to the true mean gradient:
     # per-element error below one level of the largest bucket norm
@@ -284,37 +298,34 @@ def test_average_matches_numpy_definition():
 
 # ------------------------------------------------ boundary cases of Eq. 6
 
-def test_smallest_uniform_boundaries():
-    # The uniform lives on (0, 1): with p_r = 0 the lower level is kept for every draw, also
-    # the smallest one (u = 2^-24); p_r = u exactly rounds up ("with probability p_r" counts
-    # the draws u <= p_r), p_r just below u does not.
-    from conftest import read_golden
-    for seed, step, m, j in [tuple(int(x) for x in r) for r in read_golden("smallest_uniform.txt")]:
-        blk = oracle.philox4x32_10([j >> 2, 0, m, step], [seed & 0xFFFFFFFF, seed >> 32])
-        assert int(blk[j & 3]) >> 9 == 0x7FFFFF               # the stored position draws the smallest u
-        n = (j // 32 + 1) * 32
-        lay = oracle.Layout([n], 32)
-        k = j ^ 1                                             # partner element in the same bucket
-        # (a) on-level value: norm 15, levels 9 and 12 with b = 5
-        g = np.zeros((1, n), np.float32)
-        g[0, j], g[0, k] = -9.0, 12.0
-        norms = oracle.bucket_norms(lay, g)
-        codes, frac, u = oracle.quantize(lay, g, norms, 5, seed, step, want_frac_u=True)
-        assert u[0, j] == np.float32(2.0 ** -24) and frac[0, j] == 0.0
-        assert codes[0, j] == (1 << 4) | 9 and codes[0, k] == 12
-        # (b) b = 2 (s = 1), norm 1: p_r = |g|; 2^-24 reaches u, 2^-25 does not
-        for val, want_level in ((2.0 ** -24, 1), (2.0 ** -25, 0), (1.5 * 2.0 ** -24, 1)):
-            g[0, j], g[0, k] = val, 1.0
-            norms = oracle.bucket_norms(lay, g)
-            assert norms[0, j // 32] == 1.0
-            codes, frac, u = oracle.quantize(lay, g, norms, 2, seed, step, want_frac_u=True)
-            assert frac[0, j] == np.float32(val)
-            assert codes[0, j] == want_level
+def test_rounding_boundaries():
+    # With s = 1 and a norm of exactly 1 the position on the grid is the input itself,
+    # and the drawn v of every element is known.  The level goes up (away from zero)
+    # exactly when p_r + v >= 1 for positive inputs and v < p_r for negative ones.
+    lay = oracle.Layout([32], 32)
+    one = np.ones((1, 1), np.float32)
+    zeros = np.zeros((1, 32), np.float32)
+    _, _, v = oracle.quantize(lay, zeros, one, 2, 77, 5, want_x_v=True)
+    v = v[0]
+    assert np.all((v > 0) & (v < 1))
+    s = 1
+    cases = [
+        (np.float32(1.0) - v, s + 1),                              # p_r + v = 1: up
+        (np.nextafter(np.float32(1.0) - v, np.float32(0)), s),     # just below: stays
+        (-v, s),                                                   # v = p_r: stays at 0
+        (np.nextafter(-v, np.float32(-1)), s - 1),                 # v < p_r: goes to -1
+        (zeros[0], s), (np.full(32, 1.0, np.float32), s + 1), (np.full(32, -1.0, np.float32), s - 1),
+    ]
+    for g, want in cases:
+        g = np.ascontiguousarray(g.astype(np.float32).reshape(1, 32))
+        codes, x, v2 = oracle.quantize(lay, g, one, 2, 77, 5, want_x_v=True)
+        assert np.array_equal(x, g) and np.array_equal(v2[0], v)
+        assert np.all(codes[0] == want)
 
 
 def test_ratio_one_ulp_above_s_is_clamped():
     # a single-element bucket has |g|/norm = 1, but fp32 a * (s/a) can land one
-    # ulp above s; the level must still be s (never s+1, which would reach the sign bit)
+    # ulp above s; the level must still be s, or the code would leave 0 .. 2s
     for b in (3, 4, 7):
         s = np.float32((1 << (b - 1)) - 1)
         a = np.random.default_rng(b).uniform(0.5, 2.0, 200000).astype(np.float32)
@@ -323,10 +334,11 @@ def test_ratio_one_ulp_above_s_is_clamped():
         for val in over[:8]:
             lay = oracle.Layout([1], 32)
             g = np.zeros((1, 32), np.float32)
-            g[0, 0] = -val
-            norms = oracle.bucket_norms(lay, g)
-            assert norms[0, 0] == val
-            for seed in range(4):
-                codes, frac, _ = oracle.quantize(lay, g, norms, b, seed, 0, want_frac_u=True)
-                assert frac[0, 0] == 0.0
-                assert codes[0, 0] == (1 << (b - 1)) | int(s)
+            for sign in (1.0, -1.0):
+                g[0, 0] = sign * val
+                norms = oracle.bucket_norms(lay, g)
+                assert norms[0, 0] == val
+                for seed in range(4):
+                    codes, x, _ = oracle.quantize(lay, g, norms, b, seed, 0, want_x_v=True)
+                    assert x[0, 0] == sign * s
+                    assert codes[0, 0] == int(s) + int(sign) * int(s)
