@@ -28,11 +28,14 @@
  *    buffer holds D32 = sum_i roundup32(n_i) elements.  Buckets of `bucket`
  *    elements tile each tensor separately; the last bucket of a tensor may be
  *    short.  Elements between a tensor's end and the next multiple of 32 are
- *    padding: ignored on input, code 0 in the packed stream, +0 in the output.
+ *    padding: ignored on input, the code of 0 in the packed stream, +0 in the
+ *    output.
+ *  - Codes: s = 2^(b-1) - 1 levels per sign (Sec. IV-A).  A b-bit code holds
+ *    s + sgn * level, a number in 0 .. 2s: the paper's sign bit and b-1 bits of
+ *    zeta folded into one field (0 has a single code, s).
  *  - Packed stream of one worker: group q (padded elements 32q .. 32q+31) owns
  *    words b*q .. b*q+b-1; element e of the group owns bits [e*b, e*b+b) of
- *    that little-endian bit string.  A code is sign << (b-1) | level
- *    (Sec. IV-A: one sign bit and b-1 bits for zeta), s = 2^(b-1) - 1.
+ *    that little-endian bit string.
  */
 #ifndef DQ_H
 #define DQ_H
@@ -58,6 +61,7 @@ extern "C" {
 #define DQ_STAT_BAD_BITS    2  /* device b outside 1..16                               */
 #define DQ_STAT_CAPACITY    4  /* b * D32/32 words exceed packed_stride_words          */
 #define DQ_STAT_WAIT        8  /* a bounded wait on an asynchronous copy ran out       */
+#define DQ_STAT_INTERNAL   16  /* a kernel found its shared memory misaligned and left  */
 
 #define DQ_MAX_BITS       16
 #define DQ_MAX_BUCKET   4096
@@ -134,20 +138,23 @@ int dq_choose_bits(const dq_layout_t* layout, const float* dev_norms, int32_t M,
 
 /* ----------------------------------------------------- quantizer, Eq. 5 and 6
  * For every valid element j of worker m, with norm the norm of its bucket and
- * s = 2^(b-1) - 1, all in fp32 with each operation rounded on its own:
- *   inv = norm >= 2^-100 ? s / norm : 0      r = min(|g_j| * inv, s)
- *   l = floor(r)   p_r = r - l   level = l + [u <= p_r]   code = sign(g_j) << (b-1) | level
- * u = 1 - (2k + 1) / 2^24 in (0, 1), k = w >> 9, where w is word (j & 3) of
- * Philox4x32-10 with counter (j >> 2, 0, m, step) and key (seed low word, seed
- * high word); j is the element's index in the padded layout.  The level goes
- * up with probability p_r (within 2^-24) as Eq. 6 asks, and values that lie
- * on a level are reproduced for every draw.  b = 1 stores the sign bit only.
+ * s = 2^(b-1) - 1, in fp32 with each operation rounded on its own:
+ *   inv = norm >= 2^-100 ? s / norm : 0
+ *   x   = sgn(g_j) * min(|g_j| * inv, s)        position on the level grid
+ *   code = floor(x + v) + s                      (x + v evaluated exactly)
+ * v = (2k + 1) / 2^17 in (0, 1) is the element's uniform draw: k is half (j & 1)
+ * (0 = low 16 bits) of word ((j >> 1) & 3) of Philox4x32-10 with counter
+ * (j >> 3, 0, m, step) and key (seed low word, seed high word); j is the
+ * element's index in the padded layout.  floor(x + v) is the neighbour of x
+ * away from zero with probability p_r = frac(|x|) and the one toward zero
+ * otherwise, which is Eq. 6 (to within 2^-17); values that lie on a level are
+ * reproduced for every draw.  b = 1 (s = 0) stores zeros.
  * The codes are packed as described at the top of this file.
  * in : dev_grads, dev_norms [M][nb], dev_b (written by dq_choose_bits)
  * out: dev_packed uint32, worker m at dev_packed + m*packed_stride_words; the
  *      first b*D32/32 words are written, the rest left untouched.
  * Device conditions: DQ_STAT_BAD_BITS, DQ_STAT_CAPACITY (nothing is written),
- * DQ_STAT_WAIT. */
+ * DQ_STAT_WAIT, DQ_STAT_INTERNAL. */
 int dq_quantize_pack(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
                      int32_t M, const float* dev_norms, const int32_t* dev_b,
                      uint64_t seed, uint32_t step,
@@ -155,7 +162,7 @@ int dq_quantize_pack(const dq_layout_t* layout, const float* dev_grads, int64_t 
                      int32_t* dev_status, void* stream);
 
 /* ----------------------------------- Algorithm 1, server side: "Average"
- * dev_out[j] = (1/M) sum_m sgn * level * norm_m / s   (Eq. 5 inverted, then
+ * dev_out[j] = (1/M) sum_m (code_m - s) * norm_m / s   (Eq. 5 inverted, then
  * the mean over workers); 0 for padding and when s = 0.  fp32 accumulation in
  * worker order: deterministic, within 1e-6 relative L2 of an fp64 evaluation.
  * in : dev_packed, dev_norms [M][nb], dev_b

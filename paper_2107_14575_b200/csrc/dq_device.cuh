@@ -1,7 +1,8 @@
 // Device-side arithmetic of the quantizer: the Philox4x32-10 block function,
-// the per-element encoder of Eq. 5/6 and the register bit packer.  All of it
-// is written for a thread that owns one 32-element group, so that every shift
-// and word index is a compile-time constant once B (bits per code) is known.
+// the per-element encoder of Eq. 5/6, the register bit packer and the in-place
+// decoder of the average.  All of it is written for a thread that owns one
+// 32-element group, so that every shift and word index is a compile-time
+// constant once B (bits per code) is known.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -49,27 +50,29 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
-// Eq. 5/6 for one element: r = min(|g| * inv, s); l = floor(r); p_r = r - l;
-// level = l + [u <= p_r] with u = 1 - v, v = (2k + 1) / 2^24, k the top 23 bits of
-// the element's Philox word; code = sign << (B-1) | level.
+// Eq. 5/6 for one element.  With x = sgn(g) * min(|g| * inv, s) the element's
+// position on the level grid and v = (2k + 1) / 2^17 its uniform draw (k a 16-bit
+// half of a Philox word), the code is floor(x + v) + s: for either sign the
+// neighbour of x away from zero is taken with probability frac(|x|), Eq. 6.
 // Every fp32 operation rounds on its own (no fused multiply-add).
-//  * v: the bits 0x3F800000 | k are the float 1 + k / 2^23; subtracting
-//    1 - 2^-24 from it is exact and leaves (2k + 1) / 2^24.
-//  * level = floor(r + v): u <= p_r  <=>  p_r + v >= 1.  An add rounded toward
-//    -inf never crosses an integer downwards, so floor(fl(r + v)) is the floor
-//    of the exact sum; adding 2^23, again toward -inf, leaves that integer in
-//    the low mantissa bits (0 <= r + v < 32768).  No conversion instruction.
-template <int B>
+//  * HALF selects the low (0) or high (1) 16 bits of w.  The bits
+//    0x3F800040 | k << 7 are the float 1 + v.
+//  * An add rounded toward -inf never crosses an integer downwards, so
+//    floor(fl(x + (1 + v))) is the floor of the exact sum; adding 2^23 + s - 1,
+//    again toward -inf, leaves floor(x + v) + s in the low mantissa bits.  No
+//    conversion instruction, no separate sign handling.
+// The result carries the code in its low B bits and the exponent bits of 2^23
+// above them; the packer drops everything above bit B-1.
+template <int B, int HALF>
 __device__ __forceinline__ uint32_t encode(const float g, const float inv, const float sf, const uint32_t w)
 {
-    const uint32_t gb = __float_as_uint(g);
-    if constexpr (B == 1) return gb >> 31;
+    constexpr int s = (1 << (B - 1)) - 1;
     const float r = fminf(__fmul_rn(fabsf(g), inv), sf);
-    const float x = __uint_as_float(__funnelshift_r(w, 0x7Fu, 9));      // 1 + k 2^-23
-    const float v = __fsub_rn(x, 0.99999994f);                          // (2k + 1) 2^-24, exact
-    const float t = __fadd_rd(__fadd_rd(r, v), 8388608.0f);
-    constexpr uint32_t kLow = (1u << (B - 1)) - 1u;
-    return (__float_as_uint(t) & kLow) | ((gb >> (32 - B)) & ~kLow);    // bits >= B are zero
+    const float x = __uint_as_float(__float_as_uint(r) | (__float_as_uint(g) & 0x80000000u));
+    const uint32_t kbits = HALF ? (w >> 9) : (w << 7);
+    const float one_plus_v = __uint_as_float((kbits & 0x007FFF80u) | 0x3F800040u);
+    const float t = __fadd_rd(__fadd_rd(x, one_plus_v), 8388608.0f + (float)(s - 1));
+    return __float_as_uint(t);
 }
 
 // Appends code number E of a group to the group's little-endian bit string.
@@ -77,7 +80,7 @@ __device__ __forceinline__ uint32_t encode(const float g, const float inv, const
 // top, so after 32 bits the first code sits at bit 0 and the word is complete.
 // A code that straddles two words finishes the current word with its low bits
 // and seeds the next one with itself at the top; the surplus low bits fall off
-// as that word fills up.
+// as that word fills up.  Bits of `code` above B-1 never reach a word.
 template <int B, int E>
 __device__ __forceinline__ void push_code(uint32_t (&acc)[B], uint32_t& cur, const uint32_t code)
 {
@@ -89,58 +92,62 @@ __device__ __forceinline__ void push_code(uint32_t (&acc)[B], uint32_t& cur, con
         if constexpr (sh == 0) cur = code << (32 - B);
         else cur = __funnelshift_r(cur, code, B);
     } else if constexpr (end == 32) {
-        if constexpr (sh == 0) acc[w] = code;                    // B == 32 never happens; kept for completeness
-        else acc[w] = __funnelshift_r(cur, code, B);
+        acc[w] = __funnelshift_r(cur, code, B);
     } else {
         acc[w] = __funnelshift_r(cur, code, 32 - sh);
         cur = code << (32 - B);
     }
 }
 
-// Decoding for the average.  The level bits of a code are masked out of the
-// word where they stand and OR-ed under the exponent of 2^23: the float
-// 2^23 + level * 2^k minus 2^23 is level * 2^k exactly, one logic operation and
-// one add with no shift and no int-to-float conversion.  The sign bit is shifted
-// to bit 31 and OR-ed into that float.  k depends only on the code's position
-// E, so the caller removes 2^k once after all workers have been accumulated
-// (decoded_shift).  Codes whose level bits reach above bit 22 of their word are
-// decoded from the word's upper half (shifted down by 16 once per word) or,
-// when they straddle two words, from a funnel shift.
+// (a & mask) | c as one three-input logic operation.  `c` must come from a register the
+// compiler cannot fold (callers pass the exponent pattern of 2^23 from a kernel
+// argument), otherwise two immediates would cost two instructions.
+__device__ __forceinline__ uint32_t and_or(const uint32_t a, const uint32_t mask, const uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(c));
+    return d;
+}
+
+// Decoding for the average.  A code holds s + sgn * level.  Its B bits are
+// masked out of the word where they stand and OR-ed under the exponent of 2^23:
+// that float is 2^23 + code * 2^k, and subtracting 2^23 + s * 2^k leaves
+// sgn * level * 2^k exactly -- one logic operation and one add, no shift, no
+// int-to-float conversion, no sign handling.  k depends only on the code's
+// position E, so the caller removes 2^k once after all workers have been
+// accumulated.  Codes that reach above bit 22 of their word are decoded from the
+// word's upper half (shifted down by 16 once per word) or, when they straddle
+// two words, from a funnel shift.
 template <int B, int E>
 struct CodePos {
     static constexpr int bit = E * B;
     static constexpr int w = bit >> 5;
     static constexpr int sh = bit & 31;
-    static constexpr int end = sh + B;            // one past the sign bit, counted in word w
+    static constexpr int end = sh + B;            // one past the code's last bit, counted in word w
     static constexpr bool straddles = end > 32;
-    static constexpr bool in_place = !straddles && (end - 1) <= 23;
+    static constexpr bool in_place = !straddles && end <= 23;
     static constexpr bool in_upper = !straddles && !in_place && sh >= 16;
-    // power of two the decoded magnitude carries
+    // power of two the decoded value carries
     static constexpr int k = in_place ? sh : (in_upper ? sh - 16 : 0);
 };
 
 template <int B, int E>
-__device__ __forceinline__ float decode_code(const uint32_t (&wd)[B], const uint32_t (&hi)[B])
+__device__ __forceinline__ float decode_code(const uint32_t (&wd)[B], const uint32_t (&hi)[B], const uint32_t magic)
 {
     using P = CodePos<B, E>;
-    constexpr uint32_t kLevel = (1u << (B - 1)) - 1u;
-    constexpr uint32_t kMagic = 0x4B000000u;     // 2^23
-    uint32_t m, t;
+    constexpr uint32_t kCode = (1u << B) - 1u;
+    constexpr int s = (1 << (B - 1)) - 1;
+    uint32_t m;                                  // magic = 0x4B000000, the bits of 2^23
     if constexpr (P::in_place) {
-        m = (wd[P::w] & (kLevel << P::k)) | kMagic;
-        t = (P::end == 32) ? wd[P::w] : (wd[P::w] << (32 - P::end));
+        m = and_or(wd[P::w], kCode << P::k, magic);
     } else if constexpr (P::in_upper) {
-        m = (hi[P::w] & (kLevel << P::k)) | kMagic;
-        t = (P::end == 32) ? wd[P::w] : (wd[P::w] << (32 - P::end));
+        m = and_or(hi[P::w], kCode << P::k, magic);
     } else if constexpr (!P::straddles) {
-        m = ((wd[P::w] >> P::sh) & kLevel) | kMagic;
-        t = (P::end == 32) ? wd[P::w] : (wd[P::w] << (32 - P::end));
+        m = and_or(wd[P::w] >> P::sh, kCode, magic);
     } else {
-        m = (__funnelshift_r(wd[P::w], wd[P::w + 1], P::sh) & kLevel) | kMagic;
-        t = wd[P::w + 1] << (64 - P::end);
+        m = and_or(__funnelshift_r(wd[P::w], wd[P::w + 1], P::sh), kCode, magic);
     }
-    const float d = __uint_as_float(m) - 8388608.0f;                  // level * 2^k, exact
-    return __uint_as_float(__float_as_uint(d) | (t & 0x80000000u));
+    return __uint_as_float(m) - (8388608.0f + (float)(s << P::k));      // sgn * level * 2^k, exact
 }
 
 // does any code of word W need the word's upper half?

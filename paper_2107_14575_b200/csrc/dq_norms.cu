@@ -8,6 +8,7 @@
 // searched once per run and then followed; neighbouring warps read neighbouring
 // memory.  HBM-bound: 4 bytes read per element, 4/bucket bytes written.
 #include "dq_common.cuh"
+#include "dq_tma.cuh"
 
 namespace {
 
@@ -210,6 +211,171 @@ bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, co
     if (bad) atomicOr(status, DQ_STAT_NONFINITE);
 }
 
+// Bulk-copy variant for bucket sizes that are 32 times a power of two (every size in
+// common use).  Persistent CTAs each take a contiguous range of tiles of
+// R = 4096 / bucket consecutive buckets of one worker; in the padded layout such
+// a run is one contiguous span of at most 128 groups, fetched by a single TMA
+// tensor copy into a ring of swizzled shared-memory stages, so the bytes in
+// flight are set by the ring and not by how many loads the warps manage to
+// issue.  Thread t of a tile owns group (t % gpb) of bucket (t / gpb): it squares
+// its 128-byte row, the gpb threads of a bucket combine by shuffles (and through
+// shared memory when a bucket spans several warps).
+constexpr int kTmaThreads = 128;
+constexpr int kTmaStages = 4;
+constexpr int kTmaTileBytes = kTmaThreads * 128;
+constexpr int kTmaMaxSmemSegs = 1023;
+
+extern __shared__ __align__(1024) unsigned char smem[];
+constexpr int kPartOffset = kTmaStages * kTmaTileBytes;          // 4 floats: per-warp partial sums
+constexpr int kBarOffset = kPartOffset + 16;
+constexpr int kTblOffset = kBarOffset + kTmaStages * 8;
+
+__device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
+
+struct NormsArgs {
+    LayoutView v;
+    const float* grads;
+    float* norms;
+    int32_t* status;
+    int32_t M;
+    int32_t map_has_worker_dim;
+    int32_t gpb_shift;           // log2(groups per bucket)
+};
+
+__global__ void __launch_bounds__(kTmaThreads)
+bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_constant__ CUtensorMap map)
+{
+    const int tid = threadIdx.x;
+    if (tma::smem_addr(smem) & 1023u) {
+        if (tid == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
+        return;
+    }
+    const int n1 = a.v.n_seg + 1;
+    const bool tbl_in_smem = a.v.n_seg > 1 && a.v.n_seg <= kTmaMaxSmemSegs;
+    int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
+    if (tbl_in_smem)
+        for (int i = tid; i < 3 * n1; i += kTmaThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
+    if (tid == 0) {
+        tma::prefetch_tensor_map(&map);
+#pragma unroll
+        for (int st = 0; st < kTmaStages; ++st) tma::mbar_init(full_bar(st), 1);
+        tma::fence_barrier_init();
+    }
+    __syncthreads();
+    auto tbl = [&](int i) -> int { return tbl_in_smem ? tbl_s[i] : __ldg(a.v.seg_group0 + i); };
+
+    const int gpb = 1 << a.gpb_shift;
+    const int R = kTmaThreads >> a.gpb_shift;                   // buckets per tile
+    const int nb = a.v.nb;
+    const int tiles_per_worker = (nb + R - 1) / R;
+    const int total_tiles = a.M * tiles_per_worker;
+    const int bsz = gpb * 32;
+    // every CTA takes one contiguous range of the worker-major tile list
+    const int tile_begin = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
+    const int tile_end = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
+
+    // first group and valid elements of bucket k; `seg` is a walking hint (buckets only move forward)
+    auto locate = [&](int k, int& seg, int& first_group, int& len) {
+        int local, n, g0;
+        if (a.v.n_seg == 1) {
+            local = k; n = a.v.seg0_elems; g0 = 0;
+        } else {
+            while (k >= tbl(n1 + seg + 1)) ++seg;
+            local = k - tbl(n1 + seg);
+            n = tbl(2 * n1 + seg);
+            g0 = tbl(seg);
+        }
+        first_group = g0 + (local << a.gpb_shift);
+        const int left = n - local * bsz;
+        len = left < bsz ? left : bsz;
+    };
+    auto advance = [&](int& mm, int& rr) {
+        if (++rr == tiles_per_worker) { rr = 0; ++mm; }
+    };
+
+    int m = tile_begin / tiles_per_worker, kt = tile_begin - m * tiles_per_worker;
+    int pm = m, pkt = kt, ptile = tile_begin, pseg = 0, pseg_m = m;
+    auto issue = [&](int st) {
+        if (pm != pseg_m) { pseg = 0; pseg_m = pm; }
+        int row0, len0;
+        locate(pkt * R, pseg, row0, len0);
+        tma::mbar_expect_tx(full_bar(st), kTmaTileBytes);
+        tma::load_tile_3d(smem + st * kTmaTileBytes, &map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0);
+    };
+#pragma unroll
+    for (int st = 0; st < kTmaStages; ++st) {
+        if (ptile < tile_end && tid == 0) issue(st);
+        ++ptile;
+        advance(pm, pkt);
+    }
+
+    const int r = tid >> a.gpb_shift;            // bucket of the tile this thread works on
+    const int l = tid & (gpb - 1);               // its group inside that bucket
+    const int lane = tid & 31, warp = tid >> 5;
+    float* part = reinterpret_cast<float*>(smem + kPartOffset);
+    int seg = 0, seg0 = 0, seg_m = -1;
+    int it = 0;
+    bool timed_out = false, bad = false;
+    for (int tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, kt)) {
+        const int st = it % kTmaStages;
+        if (m != seg_m) { seg = 0; seg0 = 0; seg_m = m; }
+        const int k0 = kt * R;
+        const int k = k0 + r;
+        int row0, len0, first = 0, len = 0;
+        locate(k0, seg0, row0, len0);
+        if (k < nb) locate(k, seg, first, len);
+        const int row = first - row0 + l;        // this thread's row of the tile
+        int valid = len - l * 32;                // elements of its group that count
+        valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
+
+        if (!tma::mbar_wait(full_bar(st), (it / kTmaStages) & 1)) { timed_out = true; break; }
+
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        if (valid > 0) {
+            const unsigned char* base = smem + st * kTmaTileBytes;
+            if (valid == 32) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
+                    a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                }
+            } else {                             // last group of a tensor: what follows is padding
+                for (int e = 0; e < valid; ++e) {
+                    const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
+                    a0 = fmaf(x, x, a0);
+                }
+            }
+        }
+        float sum = (a0 + a1) + (a2 + a3);
+        // combine the gpb threads of a bucket: inside a warp by shuffles ...
+        const int w = gpb < 32 ? gpb : 32;
+        for (int o = w >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (gpb > 32) {                          // ... and across the warps of a bucket through shared memory
+            if (lane == 0) part[warp] = sum;
+            __syncthreads();
+            if (l == 0) {
+                sum = 0.f;
+                for (int i = 0; i < (gpb >> 5); ++i) sum += part[(tid >> 5) + i];
+            }
+        }
+        if (l == 0 && k < nb) {
+            const float nrm = sqrtf(sum);
+            a.norms[(int64_t)m * nb + k] = nrm;
+            bad |= !isfinite(nrm);
+        }
+        __syncthreads();                         // everyone is done with this stage (and with part[])
+        if (ptile < tile_end && tid == 0) issue(st);
+        ++ptile;
+        advance(pm, pkt);
+    }
+    if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
+    if (timed_out) {
+        if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
+        for (int j = it + 1; j < it + kTmaStages; ++j)
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kTmaStages), (j / kTmaStages) & 1);
+    }
+}
+
 }  // namespace
 
 extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
@@ -224,6 +390,43 @@ extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int
     if (M > 1 && worker_stride_elems < L->padded && worker_stride_elems != 0) return DQ_ERR_RANGE;
 
     const LayoutView v = make_view(L);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t gpb = (uint32_t)v.groups_per_bucket;
+    if ((gpb & (gpb - 1)) == 0) {
+        // bucket = 32 * 2^k: bulk-copy kernel
+        NormsArgs a;
+        a.v = v;
+        a.grads = dev_grads;
+        a.norms = dev_norms;
+        a.status = dev_status;
+        a.M = M;
+        a.gpb_shift = 0;
+        while ((1u << a.gpb_shift) < gpb) ++a.gpb_shift;
+        const bool worker_dim = (M > 1 && worker_stride_elems != 0);
+        a.map_has_worker_dim = worker_dim ? 1 : 0;
+        CUtensorMap map;
+        const uint64_t dims[3] = {32, (uint64_t)v.total_groups, worker_dim ? (uint64_t)M : 1};
+        const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
+        const uint32_t box[3] = {32, (uint32_t)kTmaThreads, 1};
+        if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
+                                  CU_TENSOR_MAP_SWIZZLE_128B))
+            return DQ_ERR_CUDA;
+        size_t smem_need = (size_t)kTblOffset;
+        if (L->n_seg > 1 && L->n_seg <= kTmaMaxSmemSegs) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
+        if (cudaFuncSetAttribute(bucket_norms_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return DQ_ERR_CUDA;
+        }
+        const int R = kTmaThreads >> a.gpb_shift;
+        const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
+        int64_t blocks = (int64_t)dq_sm_count() * 3;    // three 65 KB CTAs per SM
+        if (blocks > tiles) blocks = tiles;
+        bucket_norms_tma_kernel<<<(unsigned)blocks, kTmaThreads, smem_need, st>>>(a, map);
+        if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+        return DQ_OK;
+    }
+
+    // other bucket sizes: plain-load kernels
     const int lanes = L->bucket >= 128 ? 32 : (L->bucket >= 64 ? 16 : 8);
     const int64_t chunk = (int64_t)kRun * (32 / lanes);
     const int64_t nchunks = (L->nb + chunk - 1) / chunk;
@@ -234,7 +437,6 @@ extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int
     if (bx > cap) bx = cap;
     if (bx < 1) bx = 1;
     const dim3 grid((unsigned)bx, (unsigned)M);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (lanes == 32) {
         const size_t smem = (L->n_seg > 1 && (size_t)3 * (L->n_seg + 1) * 4 <= 12 * 1024) ? (size_t)3 * (L->n_seg + 1) * 4 : 0;
         bucket_norms_warp_kernel<<<grid, kThreads, smem, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);

@@ -1,15 +1,16 @@
 // dq_quantize_pack: the EWU quantizer of Eq. 5/6 fused with the b-bit packer.
 //
-// Persistent CTAs walk tiles of 128 groups (one group = 32 consecutive padded
-// elements = one thread).  A tile's 16 KB of gradients arrive by one TMA tensor
-// copy into a ring of shared-memory stages written with the 128-byte
-// swizzle, so that a thread reading its own 128-byte row in 16-byte pieces
-// hits every bank group once per quarter warp.  The thread draws the eight
-// Philox blocks of its group, encodes the 32 codes and assembles the group's
-// b words in a register shift chain (all shifts are constants once b is
-// known).  Each warp transposes its 32*b words through shared memory and writes
-// them with 16-byte coalesced stores.  b is read from device memory and selects
-// one of sixteen specialisations with a grid-uniform switch.
+// Persistent CTAs each take a contiguous range of tiles of 128 groups (one
+// group = 32 consecutive padded elements = one thread).  A tile's 16 KB of
+// gradients arrive by one TMA tensor copy into a ring of shared-memory stages
+// written with the 128-byte swizzle, so that a thread reading its own 128-byte
+// row in 16-byte pieces hits every bank group once per quarter warp.  The
+// thread draws the four Philox blocks of its group (16 random bits per
+// element), encodes the 32 codes and assembles the group's b words in a
+// register shift chain (all shifts are constants once b is known).  Each warp
+// transposes its 32*b words through shared memory and writes them with 16-byte
+// coalesced stores.  b is read from device memory and selects one of sixteen
+// specialisations with a grid-uniform switch.
 // HBM traffic: 4 bytes read and b/8 bytes written per element.
 #include "dq_common.cuh"
 #include "dq_device.cuh"
@@ -22,6 +23,17 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kStages = 2;
 constexpr int kTileBytes = kThreads * 128;  // 16 KB of fp32 per tile
 constexpr int kMaxSmemSegs = 1023;          // layouts with more tensors read the table from global memory
+
+// Dynamic shared memory, addressed only through this symbol so that every access
+// compiles to a shared-memory instruction:
+//   [0, kStages * 16 KB)      input tiles (1024-byte aligned for the 128-byte swizzle)
+//   then kWarps * 32 * 16 words of output staging, the stage barriers, the tensor table
+extern __shared__ __align__(1024) unsigned char smem[];
+constexpr int kOutOffset = kStages * kTileBytes;
+constexpr int kBarOffset = kOutOffset + kWarps * 32 * DQ_MAX_BITS * 4;
+constexpr int kTblOffset = kBarOffset + kStages * 8;
+
+__device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
 
 struct QuantizeArgs {
     LayoutView v;
@@ -63,23 +75,29 @@ __device__ __forceinline__ void stage_words(uint32_t* __restrict__ dst, const ui
     }
 }
 
+// Encodes elements 8C .. 8C+7 of a group (one Philox block) and appends the codes.
 template <int B, int C>
-__device__ __forceinline__ void encode_chunk(uint32_t (&acc)[B], uint32_t& cur, const float4 x, const float inv,
-                                             const float sf, const uint32_t q, const uint32_t m, const uint32_t step,
-                                             const PhiloxKeys& keys)
+__device__ __forceinline__ void encode_block(uint32_t (&acc)[B], uint32_t& cur, const float4 lo, const float4 hi,
+                                             const float inv, const float sf, const uint32_t q, const uint32_t m,
+                                             const uint32_t step, const PhiloxKeys& keys)
 {
-    uint32_t w[4] = {0u, 0u, 0u, 0u};
-    if constexpr (B > 1) philox4x32_10(q, 0u, m, step, keys, w);
-    push_code<B, 4 * C + 0>(acc, cur, encode<B>(x.x, inv, sf, w[0]));
-    push_code<B, 4 * C + 1>(acc, cur, encode<B>(x.y, inv, sf, w[1]));
-    push_code<B, 4 * C + 2>(acc, cur, encode<B>(x.z, inv, sf, w[2]));
-    push_code<B, 4 * C + 3>(acc, cur, encode<B>(x.w, inv, sf, w[3]));
+    uint32_t w[4];
+    philox4x32_10(q, 0u, m, step, keys, w);
+    push_code<B, 8 * C + 0>(acc, cur, encode<B, 0>(lo.x, inv, sf, w[0]));
+    push_code<B, 8 * C + 1>(acc, cur, encode<B, 1>(lo.y, inv, sf, w[0]));
+    push_code<B, 8 * C + 2>(acc, cur, encode<B, 0>(lo.z, inv, sf, w[1]));
+    push_code<B, 8 * C + 3>(acc, cur, encode<B, 1>(lo.w, inv, sf, w[1]));
+    push_code<B, 8 * C + 4>(acc, cur, encode<B, 0>(hi.x, inv, sf, w[2]));
+    push_code<B, 8 * C + 5>(acc, cur, encode<B, 1>(hi.y, inv, sf, w[2]));
+    push_code<B, 8 * C + 6>(acc, cur, encode<B, 0>(hi.z, inv, sf, w[3]));
+    push_code<B, 8 * C + 7>(acc, cur, encode<B, 1>(hi.w, inv, sf, w[3]));
 }
 
 template <int B>
-__device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUtensorMap* map, unsigned char* tiles,
-                                               uint32_t* out_stage, uint64_t* full, const int32_t* tbl)
+__device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUtensorMap* map, const bool tbl_in_smem)
 {
+    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kTblOffset);
+    auto tbl = [&](int i) -> int { return tbl_in_smem ? tbl_s[i] : __ldg(a.v.seg_group0 + i); };
     constexpr int s = (1 << (B - 1)) - 1;
     const float sf = (float)s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -87,30 +105,38 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
     const int tiles_per_worker = (G + kThreads - 1) / kThreads;
     const int total_tiles = a.M * tiles_per_worker;
     const int n1 = a.v.n_seg + 1;
-    uint32_t* my_out = out_stage + warp * (32 * B);
+    uint32_t* my_out = reinterpret_cast<uint32_t*>(smem + kOutOffset) + warp * (32 * B);
+
+    // Tiles are numbered worker-major and every CTA takes one contiguous range of them, so
+    // the walk through the tensor table below advances by at most a few entries per tile.
+    // (m, rt) = worker and tile-within-worker of the tile being consumed, (pm, prt) of the
+    // next tile to prefetch.
+    const int tile_begin = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
+    const int tile_end = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
+    int m = tile_begin / tiles_per_worker, rt = tile_begin - m * tiles_per_worker;
+    int pm = m, prt = rt, ptile = tile_begin;
+    auto advance = [&](int& mm, int& rr) {
+        if (++rr == tiles_per_worker) { rr = 0; ++mm; }
+    };
 
     // prologue: fill the ring
-    if (tid == 0) {
 #pragma unroll
-        for (int st = 0; st < kStages; ++st) {
-            const int tile = blockIdx.x + st * gridDim.x;
-            if (tile < total_tiles) {
-                const int m = tile / tiles_per_worker;
-                const int row0 = (tile - m * tiles_per_worker) * kThreads;
-                tma::mbar_expect_tx(&full[st], kTileBytes);
-                tma::load_tile_3d(tiles + st * kTileBytes, map, &full[st], 0, row0, a.map_has_worker_dim ? m : 0);
-            }
+    for (int st = 0; st < kStages; ++st) {
+        if (ptile < tile_end && tid == 0) {
+            tma::mbar_expect_tx(full_bar(st), kTileBytes);
+            tma::load_tile_3d(smem + st * kTileBytes, map, full_bar(st), 0, prt * kThreads, a.map_has_worker_dim ? pm : 0);
         }
+        ++ptile;
+        advance(pm, prt);
     }
 
     int seg = 0, seg_m = -1;
     int it = 0;
     bool timed_out = false;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x, ++it) {
+    for (int tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, rt)) {
         const int st = it % kStages;
         const uint32_t parity = (it / kStages) & 1;
-        const int m = tile / tiles_per_worker;
-        const int row0 = (tile - m * tiles_per_worker) * kThreads;
+        const int row0 = rt * kThreads;
         const int g = row0 + tid;
         const bool active = g < G;
 
@@ -122,10 +148,10 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
                 local = g; n = a.v.seg0_elems; b0 = 0;
             } else {
                 if (m != seg_m) { seg = 0; seg_m = m; }
-                while (g >= tbl[seg + 1]) ++seg;                 // groups only move forward within a worker
-                local = g - tbl[seg];
-                b0 = tbl[n1 + seg];
-                n = tbl[2 * n1 + seg];
+                while (g >= tbl(seg + 1)) ++seg;                 // groups only move forward within a worker
+                local = g - tbl(seg);
+                b0 = tbl(n1 + seg);
+                n = tbl(2 * n1 + seg);
             }
             bucket = b0 + (int)div_gpb(a, (uint32_t)local);
             const int left = n - local * 32;
@@ -134,23 +160,29 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
         const float norm = active ? __ldg(a.norms + (int64_t)m * a.v.nb + bucket) : 0.0f;
         const float inv = (norm >= 0x1p-100f) ? __fdiv_rn(sf, norm) : 0.0f;
 
-        if (!tma::mbar_wait(&full[st], parity)) { timed_out = true; break; }
+        if (!tma::mbar_wait(full_bar(st), parity)) { timed_out = true; break; }
 
-        unsigned char* row = tiles + st * kTileBytes + tid * 128;
-        if (valid < 32) {                       // padding after a tensor's end encodes as +0
+        unsigned char* row = smem + st * kTileBytes + tid * 128;
+        if (valid < 32) {                       // padding after a tensor's end encodes as 0
             for (int e = valid; e < 32; ++e)
                 *reinterpret_cast<float*>(row + ((((e >> 2) ^ (tid & 7)) << 4) | ((e & 3) << 2))) = 0.0f;
             tma::fence_proxy_async();           // these stores precede the next bulk copy into this stage
         }
         uint32_t acc[B];
-        uint32_t cur = 0;
-        const uint32_t q0 = (uint32_t)g * 8u;
-        const uint32_t sw = (uint32_t)(tid & 7);
-#define DQ_CHUNK(C)                                                                                        \
-        encode_chunk<B, C>(acc, cur, *reinterpret_cast<const float4*>(row + (((uint32_t)(C) ^ sw) << 4)), \
-                           inv, sf, q0 + (C), (uint32_t)m, a.step, a.keys);
-        DQ_CHUNK(0) DQ_CHUNK(1) DQ_CHUNK(2) DQ_CHUNK(3) DQ_CHUNK(4) DQ_CHUNK(5) DQ_CHUNK(6) DQ_CHUNK(7)
-#undef DQ_CHUNK
+        if constexpr (B == 1) {
+            acc[0] = 0u;                        // s = 0: every code is 0
+        } else {
+            uint32_t cur = 0;
+            const uint32_t q0 = (uint32_t)g * 4u;
+            const uint32_t sw = (uint32_t)(tid & 7);
+#define DQ_BLOCK(C)                                                                                             \
+            encode_block<B, C>(acc, cur,                                                                        \
+                               *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C)) ^ sw) << 4)),      \
+                               *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)),  \
+                               inv, sf, q0 + (C), (uint32_t)m, a.step, a.keys);
+            DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
+#undef DQ_BLOCK
+        }
 
         // transpose the warp's 32*B words through shared memory, then coalesced 16-byte stores
         stage_words<B>(my_out + lane * B, acc);
@@ -167,16 +199,13 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
 
         // everyone is done with this stage (and with the staging area): refill it
         __syncthreads();
-        if (tid == 0) {
-            const int next = tile + kStages * gridDim.x;
-            if (next < total_tiles) {
-                const int nm = next / tiles_per_worker;
-                const int nrow0 = (next - nm * tiles_per_worker) * kThreads;
-                tma::fence_proxy_async();
-                tma::mbar_expect_tx(&full[st], kTileBytes);
-                tma::load_tile_3d(tiles + st * kTileBytes, map, &full[st], 0, nrow0, a.map_has_worker_dim ? nm : 0);
-            }
+        if (ptile < tile_end && tid == 0) {
+            tma::fence_proxy_async();
+            tma::mbar_expect_tx(full_bar(st), kTileBytes);
+            tma::load_tile_3d(smem + st * kTileBytes, map, full_bar(st), 0, prt * kThreads, a.map_has_worker_dim ? pm : 0);
         }
+        ++ptile;
+        advance(pm, prt);
     }
 
     if (timed_out) {
@@ -184,7 +213,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
         // give copies still in flight a bounded chance to land before the CTA's shared memory is released
         for (int k = 1; k < kStages; ++k) {
             const int j = it + k;
-            if (blockIdx.x + (int64_t)j * gridDim.x < total_tiles) (void)tma::mbar_wait(&full[j % kStages], (j / kStages) & 1);
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kStages), (j / kStages) & 1);
         }
     }
 }
@@ -192,13 +221,6 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
 __global__ void __launch_bounds__(kThreads, 5)
 quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_constant__ CUtensorMap map)
 {
-    extern __shared__ unsigned char smem_raw[];
-    // [tiles: kStages * 16 KB, 1024-byte aligned][output staging: kWarps * 32 * 16 words][barriers][table]
-    unsigned char* tiles = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint32_t* out_stage = reinterpret_cast<uint32_t*>(tiles + kStages * kTileBytes);
-    uint64_t* full = reinterpret_cast<uint64_t*>(out_stage + kWarps * 32 * DQ_MAX_BITS);
-    int32_t* tbl_s = reinterpret_cast<int32_t*>(full + kStages);
-
     const int b = __ldg(a.dev_b);
     if (b < 1 || b > DQ_MAX_BITS) {
         if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
@@ -208,22 +230,25 @@ quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_consta
         if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
         return;
     }
-
-    const int32_t* tbl = a.v.seg_group0;
-    if (a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs) {
+    if (tma::smem_addr(smem) & 1023u) {           // the swizzled tiles need a 1024-byte aligned base
+        if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
+        return;
+    }
+    const bool tbl_in_smem = a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs;
+    if (tbl_in_smem) {
+        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
         for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
-        tbl = tbl_s;
     }
     if (threadIdx.x == 0) {
         tma::prefetch_tensor_map(&map);
 #pragma unroll
-        for (int st = 0; st < kStages; ++st) tma::mbar_init(&full[st], 1);
+        for (int st = 0; st < kStages; ++st) tma::mbar_init(full_bar(st), 1);
         tma::fence_barrier_init();
     }
     __syncthreads();
 
     switch (b) {
-#define DQ_CASE(BB) case BB: quantize_tiles<BB>(a, &map, tiles, out_stage, full, tbl); break;
+#define DQ_CASE(BB) case BB: quantize_tiles<BB>(a, &map, tbl_in_smem); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -233,7 +258,7 @@ quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_consta
 
 size_t smem_bytes(int n_seg)
 {
-    size_t n = 1024 + (size_t)kStages * kTileBytes + (size_t)kWarps * 32 * DQ_MAX_BITS * 4 + kStages * 8;
+    size_t n = (size_t)kTblOffset;
     if (n_seg > 1 && n_seg <= kMaxSmemSegs) n += (size_t)3 * (n_seg + 1) * 4;
     return n;
 }
@@ -287,16 +312,16 @@ extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, in
                               CU_TENSOR_MAP_SWIZZLE_128B))
         return DQ_ERR_CUDA;
 
-    const size_t smem = smem_bytes(L->n_seg);
+    const size_t smem_need = smem_bytes(L->n_seg);
     // raising the dynamic shared-memory limit is per device and idempotent
-    if (cudaFuncSetAttribute(quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    if (cudaFuncSetAttribute(quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
         (void)cudaGetLastError();
         return DQ_ERR_CUDA;
     }
     const int64_t tiles = (int64_t)M * ((a.v.total_groups + kThreads - 1) / kThreads);
     int64_t blocks = (int64_t)dq_sm_count() * 5;       // five 42 KB CTAs fit one SM
     if (blocks > tiles) blocks = tiles;
-    quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem, static_cast<cudaStream_t>(stream)>>>(a, map);
+    quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }

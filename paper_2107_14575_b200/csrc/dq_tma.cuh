@@ -102,6 +102,26 @@ __device__ __forceinline__ void load_bulk(void* dst, const void* src, uint32_t b
                  : "memory");
 }
 
+// 2-D tiled tensor copy shared -> global (rows outside the tensor are clipped), tracked
+// by the thread's bulk-async group.
+__device__ __forceinline__ void store_tile_2d(const CUtensorMap* map, const void* src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(smem_addr(src)), "r"(c0), "r"(c1)
+                 : "memory");
+}
+
+__device__ __forceinline__ void store_commit()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+// Blocks until every committed bulk store of this thread has finished reading shared memory.
+__device__ __forceinline__ void store_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+
 __device__ __forceinline__ void prefetch_tensor_map(const CUtensorMap* map)
 {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");

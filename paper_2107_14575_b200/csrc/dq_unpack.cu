@@ -1,15 +1,17 @@
 // dq_unpack_dequant_average: the server's "Average" step of Algorithm 1 on
-// packed codes: out_j = (1/M) sum_m sgn * level * norm_m / s  (Eq. 5 inverted).
+// packed codes: out_j = (1/M) sum_m (code_m - s) * norm_m / s  (Eq. 5 inverted;
+// a code holds s + sgn * level).
 //
-// Persistent CTAs walk tiles of 128 groups (one group = 32 padded elements = one
-// thread, which keeps its 32 fp32 sums in registers).  The M workers' words of
-// a tile are fetched in chunks of a few workers by linear bulk copies (TMA) into
-// a ring of shared-memory stages, so the copies of the next chunks overlap the
-// decoding of the current one.  A code is decoded where it stands in its word
-// (mask under the exponent of 2^23, subtract 2^23, OR the sign in: see
-// decode_code) and accumulated with one FMA; the power of two its position
-// carries is removed once per element after the last worker.  Each thread
-// stores its 32 results as eight 16-byte pieces of its own 128-byte line.
+// Persistent CTAs each take a contiguous range of tiles of 128 groups (one
+// group = 32 padded elements = one thread, which keeps its 32 fp32 sums in
+// registers).  The M workers' words of a tile are fetched in chunks of a few
+// workers by linear bulk copies (TMA) into a ring of shared-memory stages, so
+// the copies of the next chunks overlap the decoding of the current one.  A
+// code is decoded where it stands in its word (mask under the exponent of 2^23,
+// subtract 2^23 + s: see decode_code) and accumulated with one FMA; the power
+// of two its position carries is removed once per element after the last
+// worker.  The 128 x 32 results of a tile go through a swizzled shared-memory
+// tile and leave with one bulk tensor store.
 // HBM traffic per output element: M*b/8 bytes read, 4 written.
 #include "dq_common.cuh"
 #include "dq_device.cuh"
@@ -20,7 +22,22 @@ namespace {
 constexpr int kThreads = 128;                 // groups per tile
 constexpr int kStages = 2;
 constexpr int kStageWords = 4096;             // 16 KB per stage
+constexpr int kMaxChunk = 8;                  // workers per stage at most
 constexpr int kMaxSmemSegs = 1023;
+
+// Dynamic shared memory, addressed only through this symbol so that every access
+// compiles to a shared-memory instruction:
+//   [0, 16 KB)                 output tile, 128-byte swizzle (1024-byte aligned)
+//   then kStages * 16 KB of input stages, 8 * 128 scales, the stage barriers, the tensor table
+extern __shared__ __align__(1024) unsigned char smem[];
+constexpr int kOutBytes = kThreads * 128;
+constexpr int kStageOffset = kOutBytes;
+constexpr int kScaleOffset = kStageOffset + kStages * kStageWords * 4;
+constexpr int kBarOffset = kScaleOffset + kMaxChunk * kThreads * 4;
+constexpr int kTblOffset = kBarOffset + kStages * 8;
+
+__device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
+__device__ __forceinline__ uint32_t* stage_words(int st) { return reinterpret_cast<uint32_t*>(smem + kStageOffset) + st * kStageWords; }
 
 struct AverageArgs {
     LayoutView v;
@@ -33,6 +50,7 @@ struct AverageArgs {
     int32_t M;
     uint32_t div_magic;
     int32_t div_shift;
+    uint32_t magic;               // 0x4B000000, kept out of the compiler's sight (see and_or)
 };
 
 __device__ __forceinline__ uint32_t div_gpb(const AverageArgs& a, uint32_t n)
@@ -41,12 +59,11 @@ __device__ __forceinline__ uint32_t div_gpb(const AverageArgs& a, uint32_t n)
     return (uint32_t)(((uint64_t)n * a.div_magic) >> 33);     // exact for n < 2^26, divisor <= 128
 }
 
-// workers per stage: as many as fit 16 KB with 128 groups of B words each, at most 8
-// (their scales sit in registers while the chunk is decoded)
+// workers per stage: as many as fit 16 KB with 128 groups of B words each, at most kMaxChunk
 template <int B>
 struct ChunkOf {
     static constexpr int fit = kStageWords / (kThreads * B);
-    static constexpr int value = fit < 1 ? 1 : (fit > 8 ? 8 : fit);
+    static constexpr int value = fit < 1 ? 1 : (fit > kMaxChunk ? kMaxChunk : fit);
 };
 
 template <int B>
@@ -73,15 +90,16 @@ __device__ __forceinline__ void load_words(const uint32_t* __restrict__ src, uin
 template <int B, int E>
 struct AccumulateAll {
     static __device__ __forceinline__ void run(float (&acc)[32], const uint32_t (&wd)[B], const uint32_t (&hi)[B],
-                                               const float scale)
+                                               const float scale, const uint32_t magic)
     {
-        acc[E] = fmaf(decode_code<B, E>(wd, hi), scale, acc[E]);
-        AccumulateAll<B, E + 1>::run(acc, wd, hi, scale);
+        acc[E] = fmaf(decode_code<B, E>(wd, hi, magic), scale, acc[E]);
+        AccumulateAll<B, E + 1>::run(acc, wd, hi, scale, magic);
     }
 };
 template <int B>
 struct AccumulateAll<B, 32> {
-    static __device__ __forceinline__ void run(float (&)[32], const uint32_t (&)[B], const uint32_t (&)[B], const float) {}
+    static __device__ __forceinline__ void run(float (&)[32], const uint32_t (&)[B], const uint32_t (&)[B], const float,
+                                               const uint32_t) {}
 };
 
 template <int B, int W>
@@ -98,7 +116,7 @@ struct UpperHalves<B, B> {
     static __device__ __forceinline__ void run(const uint32_t (&)[B], uint32_t (&)[B]) {}
 };
 
-// removes the power of two each element's decoded magnitude carried
+// removes the power of two each element's decoded value carried
 template <int B, int E>
 struct Normalise {
     static __device__ __forceinline__ void run(float (&acc)[32])
@@ -115,23 +133,24 @@ struct Normalise<B, 32> {
 
 // Issues the bulk copies of one pipeline unit: workers [m0, m0 + mc) of the tile at row0.
 template <int B>
-__device__ __forceinline__ void issue_unit(const AverageArgs& a, uint32_t* stage, uint64_t* bar, int row0, int m0, int mc)
+__device__ __forceinline__ void issue_unit(const AverageArgs& a, int st, int row0, int m0, int mc)
 {
     int rows = a.v.total_groups - row0;
     rows = rows > kThreads ? kThreads : rows;
     const uint32_t bytes = ((uint32_t)(rows * B * 4) + 15u) & ~15u;   // the stream's stride is a multiple of 16 bytes
-    tma::mbar_expect_tx(bar, bytes * (uint32_t)mc);
+    tma::mbar_expect_tx(full_bar(st), bytes * (uint32_t)mc);
     for (int j = 0; j < mc; ++j)
-        tma::load_bulk(stage + j * (kThreads * B), a.packed + (int64_t)(m0 + j) * a.packed_stride + (int64_t)row0 * B,
-                       bytes, bar);
+        tma::load_bulk(stage_words(st) + j * (kThreads * B),
+                       a.packed + (int64_t)(m0 + j) * a.packed_stride + (int64_t)row0 * B, bytes, full_bar(st));
 }
 
 template <int B>
-__device__ __forceinline__ void average_tiles(const AverageArgs& a, uint32_t* stages, float* scales,
-                                              uint64_t* full, const int32_t* tbl)
+__device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtensorMap* out_map, const bool tbl_in_smem)
 {
     constexpr int s = (1 << (B - 1)) - 1;
     constexpr int MC = ChunkOf<B>::value;
+    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kTblOffset);
+    auto tbl = [&](int i) -> int { return tbl_in_smem ? tbl_s[i] : __ldg(a.v.seg_group0 + i); };
     const int tid = threadIdx.x;
     const int G = a.v.total_groups;
     const int M = a.M;
@@ -139,23 +158,25 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, uint32_t* st
     const int nchunk = (M + MC - 1) / MC;
     const int n1 = a.v.n_seg + 1;
     const float unit = (B == 1) ? 0.0f : __fdiv_rn(1.0f, (float)s * (float)M);      // 1 / (s * M)
-    float* my_scales = scales + tid;              // column tid of a [kMaxChunk][kThreads] array
+    float* my_scales = reinterpret_cast<float*>(smem + kScaleOffset) + tid;         // column tid of [kMaxChunk][kThreads]
+    const uint32_t magic = a.magic;
 
-    // number of pipeline units this CTA will consume, and the prologue that fills the ring
-    const int my_tiles = (total_tiles > (int)blockIdx.x) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int my_units = (B == 1) ? 0 : my_tiles * nchunk;
+    // every CTA takes one contiguous range of tiles; its pipeline units are (tile, chunk) pairs
+    const int tile_begin = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
+    const int tile_end = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
+    const int my_units = (B == 1) ? 0 : (tile_end - tile_begin) * nchunk;
     if (tid == 0) {
         for (int u = 0; u < kStages && u < my_units; ++u) {
-            const int tile = blockIdx.x + (u / nchunk) * gridDim.x;
+            const int tile = tile_begin + u / nchunk;
             const int m0 = (u % nchunk) * MC;
-            issue_unit<B>(a, stages + u * kStageWords, &full[u], tile * kThreads, m0, (M - m0) < MC ? (M - m0) : MC);
+            issue_unit<B>(a, u, tile * kThreads, m0, (M - m0) < MC ? (M - m0) : MC);
         }
     }
 
     int seg = 0;
     int u = 0;                                    // pipeline unit counter
     bool timed_out = false;
-    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+    for (int tile = tile_begin; tile < tile_end; ++tile) {
         const int row0 = tile * kThreads;
         const int g = row0 + tid;
         const bool active = g < G;
@@ -165,10 +186,10 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, uint32_t* st
             if (a.v.n_seg == 1) {
                 local = g; n = a.v.seg0_elems; b0 = 0;
             } else {
-                while (g >= tbl[seg + 1]) ++seg;
-                local = g - tbl[seg];
-                b0 = tbl[n1 + seg];
-                n = tbl[2 * n1 + seg];
+                while (g >= tbl(seg + 1)) ++seg;
+                local = g - tbl(seg);
+                b0 = tbl(n1 + seg);
+                n = tbl(2 * n1 + seg);
             }
             bucket = b0 + (int)div_gpb(a, (uint32_t)local);
             const int left = n - local * 32;
@@ -188,29 +209,33 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, uint32_t* st
                     my_scales[j * kThreads] = active ? __ldg(nrm + (int64_t)j * a.v.nb) * unit : 0.0f;
 
                 const int st = u % kStages;
-                if (!tma::mbar_wait(&full[st], (u / kStages) & 1)) { timed_out = true; break; }
-                const uint32_t* base = stages + st * kStageWords + tid * B;
+                if (!tma::mbar_wait(full_bar(st), (u / kStages) & 1)) { timed_out = true; break; }
+                const uint32_t* base = stage_words(st) + tid * B;
 #pragma unroll 2
                 for (int j = 0; j < mc; ++j) {
                     uint32_t wd[B], hi[B];
                     load_words<B>(base + j * (kThreads * B), wd);
                     UpperHalves<B, 0>::run(wd, hi);
-                    AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads]);
+                    AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
                 }
+                // the previous tile's bulk store must have drained the output tile before it is rewritten below
+                if (c == nchunk - 1 && tid == 0) tma::store_wait_read();
                 __syncthreads();                  // the stage is free again
                 if (tid == 0) {
                     const int nu = u + kStages;
                     if (nu < my_units) {
                         tma::fence_proxy_async();
-                        const int ntile = blockIdx.x + (nu / nchunk) * gridDim.x;
+                        const int ntile = tile_begin + nu / nchunk;
                         const int nm0 = (nu % nchunk) * MC;
-                        issue_unit<B>(a, stages + st * kStageWords, &full[st], ntile * kThreads, nm0,
-                                      (M - nm0) < MC ? (M - nm0) : MC);
+                        issue_unit<B>(a, st, ntile * kThreads, nm0, (M - nm0) < MC ? (M - nm0) : MC);
                     }
                 }
             }
             if (timed_out) break;
             Normalise<B, 0>::run(acc);
+        } else {
+            if (tid == 0) tma::store_wait_read();
+            __syncthreads();
         }
 
         if (valid < 32) {
@@ -218,32 +243,30 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, uint32_t* st
             for (int e = 0; e < 32; ++e)
                 if (e >= valid) acc[e] = 0.0f;
         }
-        if (active) {
-            float4* dst = reinterpret_cast<float4*>(a.out + (int64_t)g * 32);
+        // own row of the swizzled output tile (conflict-free), then one bulk tensor store per tile
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                dst[c] = make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+        for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) =
+                make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+        tma::fence_proxy_async();
+        __syncthreads();
+        if (tid == 0) {
+            tma::store_tile_2d(out_map, smem, 0, row0);
+            tma::store_commit();
         }
     }
 
+    if (tid == 0) tma::store_wait_read();         // shared memory must outlive the last store's reads
     if (timed_out) {
         if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
         for (int k = 1; k < kStages; ++k)
-            if (u + k < my_units) (void)tma::mbar_wait(&full[(u + k) % kStages], ((u + k) / kStages) & 1);
+            if (u + k < my_units) (void)tma::mbar_wait(full_bar((u + k) % kStages), ((u + k) / kStages) & 1);
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 5)
-unpack_average_kernel(const __grid_constant__ AverageArgs a)
+__global__ void __launch_bounds__(kThreads, 4)
+unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_constant__ CUtensorMap out_map)
 {
-    extern __shared__ unsigned char smem_raw[];
-    // [stages: kStages * 16 KB][scales: 8 * 128 floats][barriers][table]
-    unsigned char* p = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~uintptr_t(127));
-    uint32_t* stages = reinterpret_cast<uint32_t*>(p);
-    float* scales = reinterpret_cast<float*>(p + kStages * kStageWords * 4);
-    uint64_t* full = reinterpret_cast<uint64_t*>(scales + 8 * kThreads);
-    int32_t* tbl_s = reinterpret_cast<int32_t*>(full + kStages);
-
     const int b = __ldg(a.dev_b);
     if (b < 1 || b > DQ_MAX_BITS) {
         if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
@@ -253,20 +276,25 @@ unpack_average_kernel(const __grid_constant__ AverageArgs a)
         if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
         return;
     }
-    const int32_t* tbl = a.v.seg_group0;
-    if (a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs) {
+    if (tma::smem_addr(smem) & 1023u) {           // the swizzled tile needs a 1024-byte aligned base
+        if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
+        return;
+    }
+    const bool tbl_in_smem = a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs;
+    if (tbl_in_smem) {
+        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
         for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
-        tbl = tbl_s;
     }
     if (threadIdx.x == 0) {
+        tma::prefetch_tensor_map(&out_map);
 #pragma unroll
-        for (int st = 0; st < kStages; ++st) tma::mbar_init(&full[st], 1);
+        for (int st = 0; st < kStages; ++st) tma::mbar_init(full_bar(st), 1);
         tma::fence_barrier_init();
     }
     __syncthreads();
 
     switch (b) {
-#define DQ_CASE(BB) case BB: average_tiles<BB>(a, stages, scales, full, tbl); break;
+#define DQ_CASE(BB) case BB: average_tiles<BB>(a, &out_map, tbl_in_smem); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -276,7 +304,7 @@ unpack_average_kernel(const __grid_constant__ AverageArgs a)
 
 size_t smem_bytes(int n_seg)
 {
-    size_t n = 128 + (size_t)kStages * kStageWords * 4 + (size_t)8 * kThreads * 4 + kStages * 8;
+    size_t n = (size_t)kTblOffset;
     if (n_seg > 1 && n_seg <= kMaxSmemSegs) n += (size_t)3 * (n_seg + 1) * 4;
     return n;
 }
@@ -305,6 +333,7 @@ extern "C" int dq_unpack_dequant_average(const dq_layout_t* L, const uint32_t* d
     a.out = dev_out;
     a.status = dev_status;
     a.M = M;
+    a.magic = 0x4B000000u;
     const uint32_t gpb = (uint32_t)a.v.groups_per_bucket;
     if ((gpb & (gpb - 1)) == 0) {
         a.div_shift = 0;
@@ -315,15 +344,24 @@ extern "C" int dq_unpack_dequant_average(const dq_layout_t* L, const uint32_t* d
         a.div_magic = (uint32_t)(((uint64_t(1) << 33) + gpb - 1) / gpb);
     }
 
-    const size_t smem = smem_bytes(L->n_seg);
-    if (cudaFuncSetAttribute(unpack_average_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+    // tensor map over the output: [group][32 floats], box = one tile of 128 groups, 128-byte swizzle
+    CUtensorMap out_map;
+    const uint64_t dims[2] = {32, (uint64_t)a.v.total_groups};
+    const uint64_t strides[1] = {128};
+    const uint32_t box[2] = {32, (uint32_t)kThreads};
+    if (!dq_encode_tensor_map(&out_map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, dev_out, dims, strides, box,
+                              CU_TENSOR_MAP_SWIZZLE_128B))
+        return DQ_ERR_CUDA;
+
+    const size_t smem_need = smem_bytes(L->n_seg);
+    if (cudaFuncSetAttribute(unpack_average_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
         (void)cudaGetLastError();
         return DQ_ERR_CUDA;
     }
     const int64_t tiles = ((int64_t)a.v.total_groups + kThreads - 1) / kThreads;
-    int64_t blocks = (int64_t)dq_sm_count() * 5;       // five 37 KB CTAs per SM
+    int64_t blocks = (int64_t)dq_sm_count() * 4;       // four 53 KB CTAs per SM
     if (blocks > tiles) blocks = tiles;
-    unpack_average_kernel<<<(unsigned)blocks, kThreads, smem, static_cast<cudaStream_t>(stream)>>>(a);
+    unpack_average_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, out_map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }

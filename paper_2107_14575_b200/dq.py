@@ -15,7 +15,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdq.so")
 
 OK, ERR_ARG, ERR_ALIGN, ERR_RANGE, ERR_CUDA, ERR_STATE = 0, -1, -2, -3, -4, -5
-STAT_NONFINITE, STAT_BAD_BITS, STAT_CAPACITY, STAT_WAIT = 1, 2, 4, 8
+STAT_NONFINITE, STAT_BAD_BITS, STAT_CAPACITY, STAT_WAIT, STAT_INTERNAL = 1, 2, 4, 8, 16
 
 # every symbol include/dq.h declares
 SYMBOLS = [

@@ -3,9 +3,10 @@
 Acceptance (stated once, used throughout):
   * packed words are bit-exact when the quantizer is driven with the oracle's norms;
   * bucket norms agree to 1e-6 relative;
-  * with the GPU's own norms a code may differ by one level only where
-    |p_r - u| < 1e-6 + r * delta, r = s|g|/norm and delta the relative difference of
-    the two norms of that bucket (<= 1e-6): the window by which r itself moves;
+  * with the GPU's own norms a code may differ by one only where x + v lies within
+    1e-6 + |x| * delta + 2 ulp(x) of an integer, x = sgn*s|g|/norm the position on the
+    level grid (an fp32 product), v the uniform draw and delta the relative difference
+    of the two norms of that bucket (<= 1e-6): the window by which x itself moves;
   * the bit width b is identical when the rule is driven with the oracle's norms;
   * the averaged gradient agrees to 1e-6 relative L2.
 """
@@ -173,22 +174,22 @@ def test_quantize_with_gpu_norms_differs_only_at_ties(G, name, b):
     assert np.all(np.abs(norms_gpu - norms) <= NORM_RTOL * norms)
     r.set_b(b)
     got = r.quantize(SEED, 9)
-    codes_ref, frac, u = oracle.quantize(ref, g, norms, b, SEED, 9, want_frac_u=True)
-    s = (1 << (b - 1)) - 1
+    codes_ref, x, v = oracle.quantize(ref, g, norms, b, SEED, 9, want_x_v=True)
     for m in range(w.M):
         codes = oracle.unpack(got[m], ref.D32, b)
         diff = np.nonzero(codes != codes_ref[m])[0]
         if diff.size:
-            assert np.all((codes[diff] >> (b - 1)) == (codes_ref[m][diff] >> (b - 1)))          # same sign
-            dl = (codes[diff] & s).astype(np.int64) - (codes_ref[m][diff] & s).astype(np.int64)
+            dl = codes[diff].astype(np.int64) - codes_ref[m][diff].astype(np.int64)
             assert np.all(np.abs(dl) == 1)
-            # a relative norm difference delta moves r = s|g|/norm by r*delta, so a
-            # decision can flip only where |p_r - u| <= r*delta (+ rounding); for small r
-            # this is the plain 1e-6 window
+            # a relative norm difference delta moves x = sgn*s|g|/norm by |x|*delta, so
+            # floor(x + v) can change only where x + v lies within |x|*delta (+ the fp32
+            # spacing of x) of an integer; for small |x| this is the plain 1e-6 window
             k = np.searchsorted(ref.bucket_start, diff, side="right") - 1
             delta = np.abs(norms_gpu[m][k].astype(np.float64) - norms[m][k]) / norms[m][k]
-            r_val = (codes_ref[m][diff] & s).astype(np.float64) + 1.0
-            assert np.all(np.abs(frac[m][diff].astype(np.float64) - u[m][diff]) < 1e-6 + 1.001 * r_val * delta)
+            z = x[m][diff].astype(np.float64) + v[m][diff].astype(np.float64)
+            margin = np.abs(z - np.round(z))
+            ulp = np.spacing(np.abs(x[m][diff])).astype(np.float64)     # x itself is an fp32 product
+            assert np.all(margin < 1e-6 + 1.001 * np.abs(x[m][diff]) * delta + 2 * ulp)
         assert diff.size <= 1e-4 * ref.D32 + 2
     # and driven with its own norms the GPU reproduces the oracle driven with those same norms
     want = oracle.quantize_pack(ref, g, norms_gpu, b, SEED, 9)
