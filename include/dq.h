@@ -55,6 +55,7 @@ extern "C" {
 #define DQ_ERR_RANGE  (-3)  /* size, bucket, rule field or capacity out of range       */
 #define DQ_ERR_CUDA   (-4)  /* a CUDA call (launch, copy, descriptor encode) failed    */
 #define DQ_ERR_STATE  (-5)  /* multi-tensor layout used before its device table was bound */
+#define DQ_ERR_TOO_LARGE (-6) /* more data than an allocation-free entry point's built-in scratch covers */
 
 /* ---- device status bits (OR-ed into *dev_status) ---- */
 #define DQ_STAT_NONFINITE   1  /* a bucket norm or G-bar is NaN/Inf                    */
@@ -135,6 +136,37 @@ size_t dq_choose_bits_scratch_bytes(const dq_layout_t* layout, int32_t M);
 int dq_choose_bits(const dq_layout_t* layout, const float* dev_norms, int32_t M, const dq_rule_t* rule,
                    int32_t* dev_b, void* dev_scratch, size_t scratch_bytes,
                    int32_t* dev_status, void* stream);
+
+/* ------------------------------------------- bit rule without any allocation
+ * (The paper has no counterpart: this entry point exists for the library's
+ * users, not for the method.)
+ *
+ * Same computation and same result as dq_choose_bits, for callers that have no
+ * scratch buffer to give and no way to get one: code that runs after start-up
+ * in a process whose device memory was handed out once and for all (a
+ * framework's caching allocator owns it, or the job runs against a fixed
+ * memory budget), and code on a latency-critical path where cudaMalloc is off
+ * limits because it synchronises the device and takes an unpredictable time.
+ * The chunk sums of the norm reduction live in a 64 KB array inside the
+ * library image instead; every GPU that loads the library holds those 64 KB
+ * until the process exits.  The call itself allocates and frees nothing.
+ *
+ *  - Limit: M * nb <= dq_choose_bits_noalloc_max_norms() (8192 * 8192 = 67,108,864
+ *    norms).  Beyond it the call returns DQ_ERR_TOO_LARGE and launches nothing;
+ *    use dq_choose_bits with caller scratch for larger problems.
+ *  - The first call on each device looks up the array's device address (that
+ *    device must be current, as for every call).  Make that first call before
+ *    any stream capture begins.
+ *  - All calls on a device share the one array, and it keeps what the last call
+ *    wrote.  Nothing in it needs clearing between calls (each call overwrites
+ *    every entry it later reads), but two calls whose kernels overlap on the
+ *    GPU -- different streams without an ordering between them -- race on it
+ *    and may both produce a wrong b.  Calls on one stream are safe.
+ * Arguments, outputs, status bits and the other error codes are those of
+ * dq_choose_bits without the scratch pair. */
+int64_t dq_choose_bits_noalloc_max_norms(void);
+int dq_choose_bits_noalloc(const dq_layout_t* layout, const float* dev_norms, int32_t M, const dq_rule_t* rule,
+                           int32_t* dev_b, int32_t* dev_status, void* stream);
 
 /* ----------------------------------------------------- quantizer, Eq. 5 and 6
  * For every valid element j of worker m, with norm the norm of its bucket and

@@ -11,6 +11,7 @@
 #include "dq_common.cuh"
 
 #include <cmath>
+#include <mutex>
 
 namespace {
 
@@ -115,6 +116,90 @@ extern "C" int dq_choose_bits(const dq_layout_t* L, const float* dev_norms, int3
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partial = static_cast<double*>(dev_scratch);
+    if (rule->fixed_b == 0) {
+        norm_square_partials<<<(unsigned)chunks, kThreads, 0, st>>>(dev_norms, n, partial);
+        if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    }
+    apply_rule<<<1, kThreads, 0, st>>>(partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
+                                      rule->b_min, rule->b_max, rule->fixed_b, dev_b, dev_status);
+    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+// ---------------------------------------------------------------------------
+// dq_choose_bits_noalloc: the same rule with the chunk sums kept in memory that
+// belongs to the library image instead of memory the caller hands in.
+//
+// The array below is part of the loaded module: every GPU that loads the library
+// holds these 64 KB from load until the process exits.  Its name is a device
+// symbol; in host code the name is only a stand-in and not an address a kernel
+// could use, so the address is asked for once per device with
+// cudaGetSymbolAddress while that device is current, and the kernels get that.
+namespace {
+
+constexpr int kNoAllocMaxChunks = 8192;                        // 8192 doubles = 64 KB
+static __device__ __align__(256) double g_noalloc_partials[kNoAllocMaxChunks];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mu;
+double* g_noalloc_ptr[kMaxDevices] = {};
+
+// Address of the array on the current device (looked up on the first call per device).
+int noalloc_scratch(double** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        (void)cudaGetLastError();
+        return DQ_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_noalloc_mu);
+    if (!g_noalloc_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_noalloc_partials) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return DQ_ERR_CUDA;
+        }
+        g_noalloc_ptr[dev] = static_cast<double*>(p);
+    }
+    *out = g_noalloc_ptr[dev];
+    return DQ_OK;
+}
+
+}  // namespace
+
+extern "C" int64_t dq_choose_bits_noalloc_max_norms(void) { return (int64_t)kNoAllocMaxChunks * kChunk; }
+
+extern "C" int dq_choose_bits_noalloc(const dq_layout_t* L, const float* dev_norms, int32_t M, const dq_rule_t* rule,
+                                      int32_t* dev_b, int32_t* dev_status, void* stream)
+{
+    if (!L || !rule) return DQ_ERR_ARG;
+    if (M < 1) return DQ_ERR_ARG;
+    if (M > DQ_MAX_WORKERS) return DQ_ERR_RANGE;
+    if (!dev_norms || !dev_b || !dev_status) return DQ_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(dev_norms) & 3u) || (reinterpret_cast<uintptr_t>(dev_b) & 3u) ||
+        (reinterpret_cast<uintptr_t>(dev_status) & 3u))
+        return DQ_ERR_ALIGN;
+    if (rule->fixed_b < 0 || rule->fixed_b > DQ_MAX_BITS) return DQ_ERR_RANGE;
+    if (rule->b_min < 1 || rule->b_max > DQ_MAX_BITS || rule->b_min > rule->b_max) return DQ_ERR_RANGE;
+    if (rule->fixed_b == 0 &&
+        (rule->T < 1 || rule->t < 0 || rule->t >= rule->T || !(rule->eps_hat > 0.0) || !(rule->alpha > 0.0) ||
+         !std::isfinite(rule->eps_hat) || !std::isfinite(rule->alpha)))
+        return DQ_ERR_RANGE;
+    const int64_t n = (int64_t)M * L->nb;
+    const int64_t chunks = num_chunks(n);
+    if (chunks > kNoAllocMaxChunks) return DQ_ERR_TOO_LARGE;     // more norms than the built-in array covers
+
+    double* partial = nullptr;
+    const int rc = noalloc_scratch(&partial);
+    if (rc != DQ_OK) return rc;
+
+    double coef = 0.0;
+    if (rule->fixed_b == 0)
+        coef = std::sqrt((double)rule->T / rule->eps_hat) *
+               std::pow(rule->alpha, (double)(rule->T - 1 - rule->t) / 2.0);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Nothing in the array has to start at zero: the first kernel writes every entry the
+    // second one reads, so whatever an earlier call left behind is overwritten, never used.
     if (rule->fixed_b == 0) {
         norm_square_partials<<<(unsigned)chunks, kThreads, 0, st>>>(dev_norms, n, partial);
         if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;

@@ -141,6 +141,7 @@ extern "C" const char* dq_status_string(int code)
         case DQ_ERR_RANGE: return "value out of range";
         case DQ_ERR_CUDA:  return "CUDA call failed";
         case DQ_ERR_STATE: return "layout has several tensors but no device table is bound";
+        case DQ_ERR_TOO_LARGE: return "problem larger than the built-in scratch of an allocation-free entry point";
         default:           return "unknown status";
     }
 }

@@ -14,7 +14,7 @@ from typing import Optional, Sequence
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libdq.so")
 
-OK, ERR_ARG, ERR_ALIGN, ERR_RANGE, ERR_CUDA, ERR_STATE = 0, -1, -2, -3, -4, -5
+OK, ERR_ARG, ERR_ALIGN, ERR_RANGE, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
 STAT_NONFINITE, STAT_BAD_BITS, STAT_CAPACITY, STAT_WAIT, STAT_INTERNAL = 1, 2, 4, 8, 16
 
 # every symbol include/dq.h declares
@@ -23,6 +23,7 @@ SYMBOLS = [
     "dq_layout_seg_offset", "dq_layout_num_buckets", "dq_layout_packed_words", "dq_layout_bucket",
     "dq_layout_table_bytes", "dq_layout_bind_device_table",
     "dq_bucket_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
+    "dq_choose_bits_noalloc_max_norms", "dq_choose_bits_noalloc",
     "dq_quantize_pack", "dq_unpack_dequant_average", "dq_status_string",
 ]
 
@@ -86,6 +87,10 @@ def lib():
         L.dq_choose_bits_scratch_bytes.argtypes = [vp, i32]
         L.dq_choose_bits.restype = C.c_int
         L.dq_choose_bits.argtypes = [vp, vp, i32, C.POINTER(Rule), vp, vp, sz, vp, vp]
+        L.dq_choose_bits_noalloc_max_norms.restype = i64
+        L.dq_choose_bits_noalloc_max_norms.argtypes = []
+        L.dq_choose_bits_noalloc.restype = C.c_int
+        L.dq_choose_bits_noalloc.argtypes = [vp, vp, i32, C.POINTER(Rule), vp, vp, vp]
         L.dq_quantize_pack.restype = C.c_int
         L.dq_quantize_pack.argtypes = [vp, vp, i64, i32, vp, vp, u64, u32, vp, i64, vp, vp]
         L.dq_unpack_dequant_average.restype = C.c_int
@@ -188,6 +193,14 @@ def choose_bits(layout: Layout, norms, M: int, rule: Rule, dev_b, scratch, scrat
                 stream=None) -> None:
     _check(lib().dq_choose_bits(layout.handle, _ptr(norms), int(M), C.byref(rule), _ptr(dev_b), _ptr(scratch),
                                 int(scratch_bytes), _ptr(status), _stream(stream)), "dq_choose_bits")
+
+
+def choose_bits_noalloc(layout: Layout, norms, M: int, rule: Rule, dev_b, status, stream=None) -> None:
+    """``dq_choose_bits`` for callers that cannot provide scratch memory: the reduction's
+    scratch is a 64 KB array inside the library (see ``include/dq.h`` for the limit and
+    the sharing rules)."""
+    _check(lib().dq_choose_bits_noalloc(layout.handle, _ptr(norms), int(M), C.byref(rule), _ptr(dev_b),
+                                        _ptr(status), _stream(stream)), "dq_choose_bits_noalloc")
 
 
 def quantize_pack(layout: Layout, grads, worker_stride_elems: int, M: int, norms, dev_b, seed: int, step: int,
