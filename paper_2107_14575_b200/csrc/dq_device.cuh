@@ -50,13 +50,24 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
 }
 
+// (a & mask) | c as one three-input logic operation.  `c` must come from a register the
+// compiler cannot fold (callers pass the exponent pattern of 2^23 from a kernel
+// argument), otherwise two immediates would cost two instructions.
+__device__ __forceinline__ uint32_t and_or(const uint32_t a, const uint32_t mask, const uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(c));
+    return d;
+}
+
 // Eq. 5/6 for one element.  With x = sgn(g) * min(|g| * inv, s) the element's
 // position on the level grid and v = (2k + 1) / 2^17 its uniform draw (k a 16-bit
 // half of a Philox word), the code is floor(x + v) + s: for either sign the
 // neighbour of x away from zero is taken with probability frac(|x|), Eq. 6.
 // Every fp32 operation rounds on its own (no fused multiply-add).
 //  * HALF selects the low (0) or high (1) 16 bits of w.  The bits
-//    0x3F800040 | k << 7 are the float 1 + v.
+//    0x3F800040 | k << 7 are the float 1 + v (the constant comes in a register the
+//    compiler cannot fold, see and_or).
 //  * An add rounded toward -inf never crosses an integer downwards, so
 //    floor(fl(x + (1 + v))) is the floor of the exact sum; adding 2^23 + s - 1,
 //    again toward -inf, leaves floor(x + v) + s in the low mantissa bits.  No
@@ -64,13 +75,16 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 // The result carries the code in its low B bits and the exponent bits of 2^23
 // above them; the packer drops everything above bit B-1.
 template <int B, int HALF>
-__device__ __forceinline__ uint32_t encode(const float g, const float inv, const float sf, const uint32_t w)
+__device__ __forceinline__ uint32_t encode(const float g, const float inv, const float sf, const uint32_t w,
+                                           const uint32_t one_bits)
 {
     constexpr int s = (1 << (B - 1)) - 1;
     const float r = fminf(__fmul_rn(fabsf(g), inv), sf);
     const float x = __uint_as_float(__float_as_uint(r) | (__float_as_uint(g) & 0x80000000u));
-    const uint32_t kbits = HALF ? (w >> 9) : (w << 7);
-    const float one_plus_v = __uint_as_float((kbits & 0x007FFF80u) | 0x3F800040u);
+    // k << 7 in place: the high half comes down by a multiply-high (w * 2^23 >> 32 = w >> 9),
+    // which runs on the multiplier and leaves the logic pipe to the generator
+    const uint32_t kbits = HALF ? __umulhi(w, 0x00800000u) : (w << 7);
+    const float one_plus_v = __uint_as_float(and_or(kbits, 0x007FFF80u, one_bits));   // one_bits = 0x3F800040
     const float t = __fadd_rd(__fadd_rd(x, one_plus_v), 8388608.0f + (float)(s - 1));
     return __float_as_uint(t);
 }
@@ -97,16 +111,6 @@ __device__ __forceinline__ void push_code(uint32_t (&acc)[B], uint32_t& cur, con
         acc[w] = __funnelshift_r(cur, code, 32 - sh);
         cur = code << (32 - B);
     }
-}
-
-// (a & mask) | c as one three-input logic operation.  `c` must come from a register the
-// compiler cannot fold (callers pass the exponent pattern of 2^23 from a kernel
-// argument), otherwise two immediates would cost two instructions.
-__device__ __forceinline__ uint32_t and_or(const uint32_t a, const uint32_t mask, const uint32_t c)
-{
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(mask), "r"(c));
-    return d;
 }
 
 // Decoding for the average.  A code holds s + sgn * level.  Its B bits are

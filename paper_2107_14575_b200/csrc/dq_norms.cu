@@ -240,6 +240,7 @@ struct NormsArgs {
     int32_t M;
     int32_t map_has_worker_dim;
     int32_t gpb_shift;           // log2(groups per bucket)
+    int32_t stream_reads;        // 1: the gradients exceed the L2, read them with the evict-first policy
 };
 
 __global__ void __launch_bounds__(kTmaThreads)
@@ -295,12 +296,16 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
 
     int m = tile_begin / tiles_per_worker, kt = tile_begin - m * tiles_per_worker;
     int pm = m, pkt = kt, ptile = tile_begin, pseg = 0, pseg_m = m;
+    const uint64_t policy = tma::policy_evict_first();
     auto issue = [&](int st) {
         if (pm != pseg_m) { pseg = 0; pseg_m = pm; }
         int row0, len0;
         locate(pkt * R, pseg, row0, len0);
         tma::mbar_expect_tx(full_bar(st), kTmaTileBytes);
-        tma::load_tile_3d(smem + st * kTmaTileBytes, &map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0);
+        if (a.stream_reads)
+            tma::load_tile_3d_hint(smem + st * kTmaTileBytes, &map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0, policy);
+        else
+            tma::load_tile_3d(smem + st * kTmaTileBytes, &map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0);
     };
 #pragma unroll
     for (int st = 0; st < kTmaStages; ++st) {
@@ -402,6 +407,7 @@ extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int
         a.M = M;
         a.gpb_shift = 0;
         while ((1u << a.gpb_shift) < gpb) ++a.gpb_shift;
+        a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
         const bool worker_dim = (M > 1 && worker_stride_elems != 0);
         a.map_has_worker_dim = worker_dim ? 1 : 0;
         CUtensorMap map;

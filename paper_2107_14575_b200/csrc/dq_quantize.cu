@@ -1,15 +1,17 @@
 // dq_quantize_pack: the EWU quantizer of Eq. 5/6 fused with the b-bit packer.
 //
-// Persistent CTAs each take a contiguous range of tiles of 128 groups (one
-// group = 32 consecutive padded elements = one thread).  A tile's 16 KB of
-// gradients arrive by one TMA tensor copy into a ring of shared-memory stages
-// written with the 128-byte swizzle, so that a thread reading its own 128-byte
-// row in 16-byte pieces hits every bank group once per quarter warp.  The
-// thread draws the four Philox blocks of its group (16 random bits per
-// element), encodes the 32 codes and assembles the group's b words in a
-// register shift chain (all shifts are constants once b is known).  Each warp
-// transposes its 32*b words through shared memory and writes them with 16-byte
-// coalesced stores.  b is read from device memory and selects one of sixteen
+// Every warp is an independent pipeline over a contiguous range of warp tiles
+// (32 groups; one group = 32 consecutive padded elements = one thread).  A warp
+// tile's 4 KB of gradients arrive by one TMA tensor copy into the warp's own
+// ring of shared-memory stages written with the 128-byte swizzle, so that a
+// thread reading its own 128-byte row in 16-byte pieces hits every bank group
+// once per quarter warp.  The thread draws the four Philox blocks of its group
+// (16 random bits per element), encodes the 32 codes and assembles the group's
+// b words in a register shift chain (all shifts are constants once b is
+// known).  The warp then transposes its 32*b words through the stage it has just
+// consumed and writes them with 16-byte coalesced stores, and one lane refills
+// the stage.  Warps never wait for each other: there is no CTA barrier in the
+// loop.  b is read from device memory and selects one of sixteen
 // specialisations with a grid-uniform switch.
 // HBM traffic: 4 bytes read and b/8 bytes written per element.
 #include "dq_common.cuh"
@@ -18,22 +20,28 @@
 
 namespace {
 
-constexpr int kThreads = 128;               // groups per tile
+constexpr int kThreads = 128;
 constexpr int kWarps = kThreads / 32;
-constexpr int kStages = 2;
-constexpr int kTileBytes = kThreads * 128;  // 16 KB of fp32 per tile
+constexpr int kStages = 2;                  // per warp
+constexpr int kTileBytes = 32 * 128;        // 4 KB of fp32 per warp tile
 constexpr int kMaxSmemSegs = 1023;          // layouts with more tensors read the table from global memory
 
 // Dynamic shared memory, addressed only through this symbol so that every access
 // compiles to a shared-memory instruction:
-//   [0, kStages * 16 KB)      input tiles (1024-byte aligned for the 128-byte swizzle)
-//   then kWarps * 32 * 16 words of output staging, the stage barriers, the tensor table
+//   [0, kWarps * kStages * 4 KB)   input tiles, warp-major (each 1024-byte aligned for the swizzle)
+//   then the stage barriers and the tensor table
 extern __shared__ __align__(1024) unsigned char smem[];
-constexpr int kOutOffset = kStages * kTileBytes;
-constexpr int kBarOffset = kOutOffset + kWarps * 32 * DQ_MAX_BITS * 4;
-constexpr int kTblOffset = kBarOffset + kStages * 8;
+constexpr int kBarOffset = kWarps * kStages * kTileBytes;
+constexpr int kTblOffset = kBarOffset + kWarps * kStages * 8;
 
-__device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
+__device__ __forceinline__ uint64_t* full_bar(int warp, int st)
+{
+    return reinterpret_cast<uint64_t*>(smem + kBarOffset) + warp * kStages + st;
+}
+__device__ __forceinline__ unsigned char* stage_ptr(int warp, int st)
+{
+    return smem + (warp * kStages + st) * kTileBytes;
+}
 
 struct QuantizeArgs {
     LayoutView v;
@@ -48,6 +56,8 @@ struct QuantizeArgs {
     int32_t map_has_worker_dim;   // 0 when all workers read the same buffer (stride 0)
     uint32_t div_magic;           // groups_per_bucket: division by multiply-shift, or by shift if a power of two
     int32_t div_shift;            // >= 0: power of two, shift; < 0: use div_magic with a 33-bit shift
+    int32_t stream_reads;         // 1: the gradients exceed the L2, read them with the evict-first policy
+    uint32_t one_bits;            // 0x3F800040 = bits of 1 + 2^-17, kept out of the compiler's sight (see and_or)
 };
 
 __device__ __forceinline__ uint32_t div_gpb(const QuantizeArgs& a, uint32_t n)
@@ -79,18 +89,18 @@ __device__ __forceinline__ void stage_words(uint32_t* __restrict__ dst, const ui
 template <int B, int C>
 __device__ __forceinline__ void encode_block(uint32_t (&acc)[B], uint32_t& cur, const float4 lo, const float4 hi,
                                              const float inv, const float sf, const uint32_t q, const uint32_t m,
-                                             const uint32_t step, const PhiloxKeys& keys)
+                                             const uint32_t step, const PhiloxKeys& keys, const uint32_t ob)
 {
     uint32_t w[4];
     philox4x32_10(q, 0u, m, step, keys, w);
-    push_code<B, 8 * C + 0>(acc, cur, encode<B, 0>(lo.x, inv, sf, w[0]));
-    push_code<B, 8 * C + 1>(acc, cur, encode<B, 1>(lo.y, inv, sf, w[0]));
-    push_code<B, 8 * C + 2>(acc, cur, encode<B, 0>(lo.z, inv, sf, w[1]));
-    push_code<B, 8 * C + 3>(acc, cur, encode<B, 1>(lo.w, inv, sf, w[1]));
-    push_code<B, 8 * C + 4>(acc, cur, encode<B, 0>(hi.x, inv, sf, w[2]));
-    push_code<B, 8 * C + 5>(acc, cur, encode<B, 1>(hi.y, inv, sf, w[2]));
-    push_code<B, 8 * C + 6>(acc, cur, encode<B, 0>(hi.z, inv, sf, w[3]));
-    push_code<B, 8 * C + 7>(acc, cur, encode<B, 1>(hi.w, inv, sf, w[3]));
+    push_code<B, 8 * C + 0>(acc, cur, encode<B, 0>(lo.x, inv, sf, w[0], ob));
+    push_code<B, 8 * C + 1>(acc, cur, encode<B, 1>(lo.y, inv, sf, w[0], ob));
+    push_code<B, 8 * C + 2>(acc, cur, encode<B, 0>(lo.z, inv, sf, w[1], ob));
+    push_code<B, 8 * C + 3>(acc, cur, encode<B, 1>(lo.w, inv, sf, w[1], ob));
+    push_code<B, 8 * C + 4>(acc, cur, encode<B, 0>(hi.x, inv, sf, w[2], ob));
+    push_code<B, 8 * C + 5>(acc, cur, encode<B, 1>(hi.y, inv, sf, w[2], ob));
+    push_code<B, 8 * C + 6>(acc, cur, encode<B, 0>(hi.z, inv, sf, w[3], ob));
+    push_code<B, 8 * C + 7>(acc, cur, encode<B, 1>(hi.w, inv, sf, w[3], ob));
 }
 
 template <int B>
@@ -100,32 +110,39 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
     auto tbl = [&](int i) -> int { return tbl_in_smem ? tbl_s[i] : __ldg(a.v.seg_group0 + i); };
     constexpr int s = (1 << (B - 1)) - 1;
     const float sf = (float)s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = a.v.total_groups;
-    const int tiles_per_worker = (G + kThreads - 1) / kThreads;
-    const int total_tiles = a.M * tiles_per_worker;
+    const int tiles_per_worker = (G + 31) / 32;
+    const int64_t total_tiles = (int64_t)a.M * tiles_per_worker;
     const int n1 = a.v.n_seg + 1;
-    uint32_t* my_out = reinterpret_cast<uint32_t*>(smem + kOutOffset) + warp * (32 * B);
 
-    // Tiles are numbered worker-major and every CTA takes one contiguous range of them, so
-    // the walk through the tensor table below advances by at most a few entries per tile.
+    // Warp tiles are numbered worker-major and every warp takes one contiguous range of them,
+    // so the walk through the tensor table below advances by at most a few entries per tile.
     // (m, rt) = worker and tile-within-worker of the tile being consumed, (pm, prt) of the
     // next tile to prefetch.
-    const int tile_begin = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
-    const int tile_end = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
-    int m = tile_begin / tiles_per_worker, rt = tile_begin - m * tiles_per_worker;
-    int pm = m, prt = rt, ptile = tile_begin;
+    const int64_t nwarps = (int64_t)gridDim.x * kWarps;
+    const int64_t gw = (int64_t)blockIdx.x * kWarps + warp;
+    const int64_t tile_begin = gw * total_tiles / nwarps;
+    const int64_t tile_end = (gw + 1) * total_tiles / nwarps;
+    int m = (int)(tile_begin / tiles_per_worker), rt = (int)(tile_begin - (int64_t)m * tiles_per_worker);
+    int pm = m, prt = rt;
+    int64_t ptile = tile_begin;
     auto advance = [&](int& mm, int& rr) {
         if (++rr == tiles_per_worker) { rr = 0; ++mm; }
     };
+    const uint64_t policy = tma::policy_evict_first();
+    auto fetch = [&](int st) {
+        tma::mbar_expect_tx(full_bar(warp, st), kTileBytes);
+        if (a.stream_reads)
+            tma::load_tile_3d_hint(stage_ptr(warp, st), map, full_bar(warp, st), 0, prt * 32, a.map_has_worker_dim ? pm : 0, policy);
+        else
+            tma::load_tile_3d(stage_ptr(warp, st), map, full_bar(warp, st), 0, prt * 32, a.map_has_worker_dim ? pm : 0);
+    };
 
-    // prologue: fill the ring
+    // prologue: fill the warp's ring
 #pragma unroll
     for (int st = 0; st < kStages; ++st) {
-        if (ptile < tile_end && tid == 0) {
-            tma::mbar_expect_tx(full_bar(st), kTileBytes);
-            tma::load_tile_3d(smem + st * kTileBytes, map, full_bar(st), 0, prt * kThreads, a.map_has_worker_dim ? pm : 0);
-        }
+        if (ptile < tile_end && lane == 0) fetch(st);
         ++ptile;
         advance(pm, prt);
     }
@@ -133,11 +150,11 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
     int seg = 0, seg_m = -1;
     int it = 0;
     bool timed_out = false;
-    for (int tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, rt)) {
+    for (int64_t tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, rt)) {
         const int st = it % kStages;
         const uint32_t parity = (it / kStages) & 1;
-        const int row0 = rt * kThreads;
-        const int g = row0 + tid;
+        const int row0 = rt * 32;
+        const int g = row0 + lane;
         const bool active = g < G;
 
         // where this group lives: tensor, bucket, valid elements (independent of the tile's data)
@@ -160,13 +177,15 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
         const float norm = active ? __ldg(a.norms + (int64_t)m * a.v.nb + bucket) : 0.0f;
         const float inv = (norm >= 0x1p-100f) ? __fdiv_rn(sf, norm) : 0.0f;
 
-        if (!tma::mbar_wait(full_bar(st), parity)) { timed_out = true; break; }
+        // every lane polls the barrier itself; the verdict is made warp-uniform so that the
+        // warp-level synchronisations below are always reached by all lanes or by none
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(full_bar(warp, st), parity))) { timed_out = true; break; }
 
-        unsigned char* row = smem + st * kTileBytes + tid * 128;
+        unsigned char* tile_base = stage_ptr(warp, st);
+        unsigned char* row = tile_base + lane * 128;
         if (valid < 32) {                       // padding after a tensor's end encodes as 0
             for (int e = valid; e < 32; ++e)
-                *reinterpret_cast<float*>(row + ((((e >> 2) ^ (tid & 7)) << 4) | ((e & 3) << 2))) = 0.0f;
-            tma::fence_proxy_async();           // these stores precede the next bulk copy into this stage
+                *reinterpret_cast<float*>(row + ((((e >> 2) ^ (lane & 7)) << 4) | ((e & 3) << 2))) = 0.0f;
         }
         uint32_t acc[B];
         if constexpr (B == 1) {
@@ -174,51 +193,50 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
         } else {
             uint32_t cur = 0;
             const uint32_t q0 = (uint32_t)g * 4u;
-            const uint32_t sw = (uint32_t)(tid & 7);
+            const uint32_t sw = (uint32_t)(lane & 7);
 #define DQ_BLOCK(C)                                                                                             \
             encode_block<B, C>(acc, cur,                                                                        \
                                *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C)) ^ sw) << 4)),      \
                                *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)),  \
-                               inv, sf, q0 + (C), (uint32_t)m, a.step, a.keys);
+                               inv, sf, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
             DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
 #undef DQ_BLOCK
         }
 
-        // transpose the warp's 32*B words through shared memory, then coalesced 16-byte stores
-        stage_words<B>(my_out + lane * B, acc);
+        // The warp has read all of its rows: reuse the stage to transpose the 32*B words,
+        // then store them 16 bytes per lane.
         __syncwarp();
-        const int g_warp = row0 + warp * 32;
-        int ng = G - g_warp;
-        ng = ng < 0 ? 0 : (ng > 32 ? 32 : ng);
+        uint32_t* out_words = reinterpret_cast<uint32_t*>(tile_base);
+        stage_words<B>(out_words + lane * B, acc);
+        tma::fence_proxy_async();               // these stores precede the bulk copy that refills the stage
+        __syncwarp();
+        int ng = G - row0;
+        ng = ng > 32 ? 32 : ng;
         const int nwords = ng * B;
-        uint32_t* dst = a.packed + (int64_t)m * a.packed_stride + (int64_t)g_warp * B;
+        uint32_t* dst = a.packed + (int64_t)m * a.packed_stride + (int64_t)row0 * B;
         const int n4 = nwords >> 2;
         for (int i = lane; i < n4; i += 32)
-            reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(my_out)[i];
-        if (lane < (nwords & 3)) dst[n4 * 4 + lane] = my_out[n4 * 4 + lane];
+            reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(out_words)[i];
+        if (lane < (nwords & 3)) dst[n4 * 4 + lane] = out_words[n4 * 4 + lane];
+        __syncwarp();
 
-        // everyone is done with this stage (and with the staging area): refill it
-        __syncthreads();
-        if (ptile < tile_end && tid == 0) {
-            tma::fence_proxy_async();
-            tma::mbar_expect_tx(full_bar(st), kTileBytes);
-            tma::load_tile_3d(smem + st * kTileBytes, map, full_bar(st), 0, prt * kThreads, a.map_has_worker_dim ? pm : 0);
-        }
+        // refill the stage
+        if (ptile < tile_end && lane == 0) fetch(st);
         ++ptile;
         advance(pm, prt);
     }
 
     if (timed_out) {
-        if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
+        if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
         // give copies still in flight a bounded chance to land before the CTA's shared memory is released
         for (int k = 1; k < kStages; ++k) {
             const int j = it + k;
-            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kStages), (j / kStages) & 1);
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(warp, j % kStages), (j / kStages) & 1);
         }
     }
 }
 
-__global__ void __launch_bounds__(kThreads, 5)
+__global__ void __launch_bounds__(kThreads, 6)
 quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_constant__ CUtensorMap map)
 {
     const int b = __ldg(a.dev_b);
@@ -241,8 +259,7 @@ quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_consta
     }
     if (threadIdx.x == 0) {
         tma::prefetch_tensor_map(&map);
-#pragma unroll
-        for (int st = 0; st < kStages; ++st) tma::mbar_init(full_bar(st), 1);
+        for (int i = 0; i < kWarps * kStages; ++i) tma::mbar_init(full_bar(0, i), 1);
         tma::fence_barrier_init();
     }
     __syncthreads();
@@ -291,6 +308,8 @@ extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, in
     a.keys = make_philox_keys(seed);
     a.step = step;
     a.M = M;
+    a.one_bits = 0x3F800040u;
+    a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
     const bool worker_dim = (M > 1 && worker_stride_elems != 0);
     a.map_has_worker_dim = worker_dim ? 1 : 0;
     const uint32_t gpb = (uint32_t)a.v.groups_per_bucket;
@@ -303,11 +322,11 @@ extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, in
         a.div_magic = (uint32_t)(((uint64_t(1) << 33) + gpb - 1) / gpb);
     }
 
-    // tensor map over the gradients: [worker][group][32 floats], box = one tile of 128 groups
+    // tensor map over the gradients: [worker][group][32 floats], box = one warp tile of 32 groups
     CUtensorMap map;
     const uint64_t dims[3] = {32, (uint64_t)a.v.total_groups, worker_dim ? (uint64_t)M : 1};
     const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
-    const uint32_t box[3] = {32, (uint32_t)kThreads, 1};
+    const uint32_t box[3] = {32, 32, 1};                 // one warp tile
     if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
                               CU_TENSOR_MAP_SWIZZLE_128B))
         return DQ_ERR_CUDA;
@@ -318,9 +337,9 @@ extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, in
         (void)cudaGetLastError();
         return DQ_ERR_CUDA;
     }
-    const int64_t tiles = (int64_t)M * ((a.v.total_groups + kThreads - 1) / kThreads);
-    int64_t blocks = (int64_t)dq_sm_count() * 5;       // five 42 KB CTAs fit one SM
-    if (blocks > tiles) blocks = tiles;
+    const int64_t warp_tiles = (int64_t)M * ((a.v.total_groups + 31) / 32);
+    int64_t blocks = (int64_t)dq_sm_count() * 6;       // six 33 KB CTAs fit one SM
+    if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
     quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;

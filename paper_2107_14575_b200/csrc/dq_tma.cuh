@@ -94,6 +94,24 @@ __device__ __forceinline__ void load_tile_3d(void* dst, const CUtensorMap* map, 
         : "memory");
 }
 
+// L2 policy for data that is read once and should be the first to leave the cache.
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+
+// Same copy as load_tile_3d with an L2 cache policy attached to the global reads.
+__device__ __forceinline__ void load_tile_3d_hint(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2,
+                                                  uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+        ::"r"(smem_addr(dst)), "l"(map), "r"(smem_addr(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(policy)
+        : "memory");
+}
+
 // Linear bulk copy global -> shared; addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void load_bulk(void* dst, const void* src, uint32_t bytes, uint64_t* bar)
 {
