@@ -20,7 +20,7 @@ _SO = os.path.join(_HERE, "libdq_oracle.so")
 _lock = threading.Lock()
 _lib = None
 
-CFLAGS = ["-O2", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-Wall"]
+CFLAGS = ["-O2", "-ffp-contract=off", "-frounding-math", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-Wall"]
 
 
 def build(force: bool = False) -> str:

@@ -2,11 +2,13 @@
  * dq_oracle.c -- plain CPU oracle of the DQ-SGD quantizer hot path.
  * TEST INFRASTRUCTURE ONLY; see dq_oracle.h.  Build with
  *   gcc -O2 -ffp-contract=off -fopenmp -shared -fPIC
- * (-ffp-contract=off: every fp32 operation below rounds on its own, in the
- * order written; that order is part of the definition of the codes).
+ * (-ffp-contract=off -frounding-math: every fp32 operation below rounds on its
+ * own, in the order written and in the rounding mode set around it; both are
+ * part of the definition of the codes).
  */
 #include "dq_oracle.h"
 
+#include <fenv.h>
 #include <math.h>
 #include <stdlib.h>
 #include <string.h>
@@ -191,13 +193,22 @@ void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
     for (int64_t w = 0; w < total; ++w) {
         const int64_t m = w / tb.nb, k = w % tb.nb;
         const float norm = norms[w];
-        const float inv = (norm >= ORACLE_TINY_NORM) ? sf / norm : 0.0f;
+        /* s / norm and g * inv are both rounded toward zero: then |x| <= s for every
+         * element with |g| <= norm (the norm of a bucket dominates its entries), so the
+         * code stays in 0 .. 2s without a clamp, and inputs on a level stay exact. */
+        float xs[4096];                      /* a bucket has at most 4096 elements */
+        fesetround(FE_TOWARDZERO);
+        {
+            const volatile float inv = (norm >= ORACLE_TINY_NORM) ? sf / norm : 0.0f;
+            for (int64_t e = 0; e < tb.len[k]; ++e) {
+                const volatile float g = grads[m * worker_stride + tb.start[k] + e];
+                xs[e] = g * inv;             /* s * g_j / ||g||: signed position on the level grid (Eq. 6) */
+            }
+        }
+        fesetround(FE_TONEAREST);
         for (int64_t e = 0; e < tb.len[k]; ++e) {
             const int64_t j = tb.start[k] + e;
-            const float g = grads[m * worker_stride + j];
-            float r = fabsf(g) * inv;        /* s * |g_j| / ||g||  (Eq. 6), fp32 */
-            r = fminf(r, sf);                /* an ulp above s must stay inside the code range */
-            const float x = copysignf(r, g); /* signed position on the level grid */
+            const float x = xs[e];
             const float v = uniform16(seed, step, (uint32_t)m, j);
             /* Eq. 6 on the signed grid: floor(x + v) is the neighbour of x away
              * from zero with probability p_r = frac(|x|) and the one toward zero

@@ -65,7 +65,7 @@ void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t
 
 /* ---- Eq. 5/6: codes s + sgn * level, one uint32 per padded element (s for
  *      padding).  x_out / v_out (optional, may be NULL) receive the signed
- *      position x = sgn * s|g|/norm on the level grid and the uniform v drawn
+ *      position x = RZ(g * RZ(s/norm)) on the level grid and the uniform v drawn
  *      for every element; the code is floor(x + v) + s. ---- */
 void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
                      const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
