@@ -170,10 +170,14 @@ int dq_choose_bits_noalloc(const dq_layout_t* layout, const float* dev_norms, in
 
 /* ----------------------------------------------------- quantizer, Eq. 5 and 6
  * For every valid element j of worker m, with norm the norm of its bucket and
- * s = 2^(b-1) - 1, in fp32 with each operation rounded on its own:
- *   inv = norm >= 2^-100 ? s / norm : 0
- *   x   = sgn(g_j) * min(|g_j| * inv, s)        position on the level grid
+ * s = 2^(b-1) - 1, in fp32 with both operations rounded toward zero (RZ):
+ *   inv = norm >= 2^-100 ? RZ(s / norm) : 0
+ *   x   = RZ(g_j * inv)                          position on the level grid
  *   code = floor(x + v) + s                      (x + v evaluated exactly)
+ * Rounding toward zero keeps |x| <= s for every element with |g_j| <= norm, which
+ * holds for the norms dq_bucket_norms computes (a bucket's norm dominates its
+ * entries).  The codes of a bucket whose norm is smaller than one of its entries
+ * are unspecified (nothing outside the packed stream is touched).
  * v = (2k + 1) / 2^17 in (0, 1) is the element's uniform draw: k is half (j & 1)
  * (0 = low 16 bits) of word ((j >> 1) & 3) of Philox4x32-10 with counter
  * (j >> 3, 0, m, step) and key (seed low word, seed high word); j is the

@@ -60,27 +60,26 @@ __device__ __forceinline__ uint32_t and_or(const uint32_t a, const uint32_t mask
     return d;
 }
 
-// Eq. 5/6 for one element.  With x = sgn(g) * min(|g| * inv, s) the element's
+// Eq. 5/6 for one element.  With x = RZ(g * inv), inv = RZ(s / norm), the element's
 // position on the level grid and v = (2k + 1) / 2^17 its uniform draw (k a 16-bit
 // half of a Philox word), the code is floor(x + v) + s: for either sign the
 // neighbour of x away from zero is taken with probability frac(|x|), Eq. 6.
-// Every fp32 operation rounds on its own (no fused multiply-add).
+//  * Both roundings are toward zero, so |x| <= s whenever |g| <= norm (a bucket's
+//    norm dominates its entries): no clamp, no absolute value, no sign handling.
 //  * HALF selects the low (0) or high (1) 16 bits of w.  The bits
 //    0x3F800040 | k << 7 are the float 1 + v (the constant comes in a register the
 //    compiler cannot fold, see and_or).
 //  * An add rounded toward -inf never crosses an integer downwards, so
 //    floor(fl(x + (1 + v))) is the floor of the exact sum; adding 2^23 + s - 1,
 //    again toward -inf, leaves floor(x + v) + s in the low mantissa bits.  No
-//    conversion instruction, no separate sign handling.
+//    conversion instruction.
 // The result carries the code in its low B bits and the exponent bits of 2^23
 // above them; the packer drops everything above bit B-1.
 template <int B, int HALF>
-__device__ __forceinline__ uint32_t encode(const float g, const float inv, const float sf, const uint32_t w,
-                                           const uint32_t one_bits)
+__device__ __forceinline__ uint32_t encode(const float g, const float inv, const uint32_t w, const uint32_t one_bits)
 {
     constexpr int s = (1 << (B - 1)) - 1;
-    const float r = fminf(__fmul_rn(fabsf(g), inv), sf);
-    const float x = __uint_as_float(__float_as_uint(r) | (__float_as_uint(g) & 0x80000000u));
+    const float x = __fmul_rz(g, inv);
     // k << 7 in place: the high half comes down by a multiply-high (w * 2^23 >> 32 = w >> 9),
     // which runs on the multiplier and leaves the logic pipe to the generator
     const uint32_t kbits = HALF ? __umulhi(w, 0x00800000u) : (w << 7);

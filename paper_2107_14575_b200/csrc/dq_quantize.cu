@@ -88,19 +88,19 @@ __device__ __forceinline__ void stage_words(uint32_t* __restrict__ dst, const ui
 // Encodes elements 8C .. 8C+7 of a group (one Philox block) and appends the codes.
 template <int B, int C>
 __device__ __forceinline__ void encode_block(uint32_t (&acc)[B], uint32_t& cur, const float4 lo, const float4 hi,
-                                             const float inv, const float sf, const uint32_t q, const uint32_t m,
+                                             const float inv, const uint32_t q, const uint32_t m,
                                              const uint32_t step, const PhiloxKeys& keys, const uint32_t ob)
 {
     uint32_t w[4];
     philox4x32_10(q, 0u, m, step, keys, w);
-    push_code<B, 8 * C + 0>(acc, cur, encode<B, 0>(lo.x, inv, sf, w[0], ob));
-    push_code<B, 8 * C + 1>(acc, cur, encode<B, 1>(lo.y, inv, sf, w[0], ob));
-    push_code<B, 8 * C + 2>(acc, cur, encode<B, 0>(lo.z, inv, sf, w[1], ob));
-    push_code<B, 8 * C + 3>(acc, cur, encode<B, 1>(lo.w, inv, sf, w[1], ob));
-    push_code<B, 8 * C + 4>(acc, cur, encode<B, 0>(hi.x, inv, sf, w[2], ob));
-    push_code<B, 8 * C + 5>(acc, cur, encode<B, 1>(hi.y, inv, sf, w[2], ob));
-    push_code<B, 8 * C + 6>(acc, cur, encode<B, 0>(hi.z, inv, sf, w[3], ob));
-    push_code<B, 8 * C + 7>(acc, cur, encode<B, 1>(hi.w, inv, sf, w[3], ob));
+    push_code<B, 8 * C + 0>(acc, cur, encode<B, 0>(lo.x, inv, w[0], ob));
+    push_code<B, 8 * C + 1>(acc, cur, encode<B, 1>(lo.y, inv, w[0], ob));
+    push_code<B, 8 * C + 2>(acc, cur, encode<B, 0>(lo.z, inv, w[1], ob));
+    push_code<B, 8 * C + 3>(acc, cur, encode<B, 1>(lo.w, inv, w[1], ob));
+    push_code<B, 8 * C + 4>(acc, cur, encode<B, 0>(hi.x, inv, w[2], ob));
+    push_code<B, 8 * C + 5>(acc, cur, encode<B, 1>(hi.y, inv, w[2], ob));
+    push_code<B, 8 * C + 6>(acc, cur, encode<B, 0>(hi.z, inv, w[3], ob));
+    push_code<B, 8 * C + 7>(acc, cur, encode<B, 1>(hi.w, inv, w[3], ob));
 }
 
 template <int B>
@@ -175,7 +175,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
             valid = left < 32 ? left : 32;
         }
         const float norm = active ? __ldg(a.norms + (int64_t)m * a.v.nb + bucket) : 0.0f;
-        const float inv = (norm >= 0x1p-100f) ? __fdiv_rn(sf, norm) : 0.0f;
+        const float inv = (norm >= 0x1p-100f) ? __fdiv_rz(sf, norm) : 0.0f;
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
         // warp-level synchronisations below are always reached by all lanes or by none
@@ -198,7 +198,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
             encode_block<B, C>(acc, cur,                                                                        \
                                *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C)) ^ sw) << 4)),      \
                                *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)),  \
-                               inv, sf, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+                               inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
             DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
 #undef DQ_BLOCK
         }
