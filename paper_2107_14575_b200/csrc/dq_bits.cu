@@ -15,36 +15,46 @@
 
 namespace {
 
-constexpr int kThreads = 256;
-constexpr int kChunk = 8192;     // norms per CTA of the first kernel
+constexpr int kThreads = 256;       // threads of the second kernel
+constexpr int kChunk = 8192;        // norms per CTA of the first kernel
+constexpr int kSumThreads = 512;    // threads of the first kernel: 16 norms each, all loads in flight at once
 
+// Sum over the CTA in a fixed order: shuffle tree inside each warp, then the warp sums
+// added in warp order by thread 0.  Returns the total in thread 0.
+template <int NT>
 __device__ __forceinline__ double block_sum(double v, double* sh)
 {
-    sh[threadIdx.x] = v;
-    __syncthreads();
 #pragma unroll
-    for (int o = kThreads / 2; o > 0; o >>= 1) {
-        if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
-        __syncthreads();
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double total = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < NT / 32; ++w) total += sh[w];
     }
-    return sh[0];
+    return total;
 }
 
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kSumThreads)
 norm_square_partials(const float* __restrict__ norms, const int64_t n, double* __restrict__ partial)
 {
-    __shared__ double sh[kThreads];
-    const int64_t base = (int64_t)blockIdx.x * kChunk;
-    double acc = 0.0;
-#pragma unroll 4
-    for (int i = threadIdx.x; i < kChunk; i += kThreads) {
-        const int64_t j = base + i;
-        if (j < n) {
-            const double x = (double)__ldg(norms + j);
-            acc = fma(x, x, acc);
-        }
+    __shared__ double sh[kSumThreads / 32];
+    constexpr int kPer = kChunk / kSumThreads;
+    const int64_t base = (int64_t)blockIdx.x * kChunk + threadIdx.x;
+    float x[kPer];
+#pragma unroll
+    for (int i = 0; i < kPer; ++i) {
+        const int64_t j = base + (int64_t)i * kSumThreads;
+        x[i] = (j < n) ? __ldg(norms + j) : 0.0f;
     }
-    const double s = block_sum(acc, sh);
+    double a0 = 0.0, a1 = 0.0;
+#pragma unroll
+    for (int i = 0; i < kPer; i += 2) {
+        a0 = fma((double)x[i], (double)x[i], a0);
+        a1 = fma((double)x[i + 1], (double)x[i + 1], a1);
+    }
+    const double s = block_sum<kSumThreads>(a0 + a1, sh);
     if (threadIdx.x == 0) partial[blockIdx.x] = s;
 }
 
@@ -53,10 +63,10 @@ apply_rule(const double* __restrict__ partial, const int npartial, const int M, 
            const int b_min, const int b_max, const int fixed_b,
            int32_t* __restrict__ dev_b, int32_t* __restrict__ status)
 {
-    __shared__ double sh[kThreads];
+    __shared__ double sh[kThreads / 32];
     double acc = 0.0;
     for (int i = threadIdx.x; i < npartial; i += kThreads) acc += partial[i];
-    const double sum = block_sum(acc, sh);
+    const double sum = block_sum<kThreads>(acc, sh);
     if (threadIdx.x != 0) return;
 
     int b;
@@ -117,7 +127,7 @@ extern "C" int dq_choose_bits(const dq_layout_t* L, const float* dev_norms, int3
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partial = static_cast<double*>(dev_scratch);
     if (rule->fixed_b == 0) {
-        norm_square_partials<<<(unsigned)chunks, kThreads, 0, st>>>(dev_norms, n, partial);
+        norm_square_partials<<<(unsigned)chunks, kSumThreads, 0, st>>>(dev_norms, n, partial);
         if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     }
     apply_rule<<<1, kThreads, 0, st>>>(partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
@@ -201,7 +211,7 @@ extern "C" int dq_choose_bits_noalloc(const dq_layout_t* L, const float* dev_nor
     // Nothing in the array has to start at zero: the first kernel writes every entry the
     // second one reads, so whatever an earlier call left behind is overwritten, never used.
     if (rule->fixed_b == 0) {
-        norm_square_partials<<<(unsigned)chunks, kThreads, 0, st>>>(dev_norms, n, partial);
+        norm_square_partials<<<(unsigned)chunks, kSumThreads, 0, st>>>(dev_norms, n, partial);
         if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     }
     apply_rule<<<1, kThreads, 0, st>>>(partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,

@@ -32,7 +32,7 @@ constexpr int kMaxSmemSegs = 1023;
 extern __shared__ __align__(1024) unsigned char smem[];
 constexpr int kOutBytes = kThreads * 128;
 constexpr int kStageOffset = kOutBytes;
-constexpr int kScaleOffset = kStageOffset + kStages * kStageWords * 4;
+constexpr int kScaleOffset = kStageOffset + kStages * kStageWords * 4;            // [kMaxChunk][kThreads] floats
 constexpr int kBarOffset = kScaleOffset + kMaxChunk * kThreads * 4;
 constexpr int kTblOffset = kBarOffset + kStages * 8;
 
@@ -158,7 +158,8 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
     const int nchunk = (M + MC - 1) / MC;
     const int n1 = a.v.n_seg + 1;
     const float unit = (B == 1) ? 0.0f : __fdiv_rn(1.0f, (float)s * (float)M);      // 1 / (s * M)
-    float* my_scales = reinterpret_cast<float*>(smem + kScaleOffset) + tid;         // column tid of [kMaxChunk][kThreads]
+    // this thread's column of the [kMaxChunk][kThreads] scale buffer (only this thread touches it)
+    float* my_scales = reinterpret_cast<float*>(smem + kScaleOffset) + tid;
     const uint32_t magic = a.magic;
 
     // every CTA takes one contiguous range of tiles; its pipeline units are (tile, chunk) pairs
@@ -173,40 +174,101 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         }
     }
 
+    // Bucket and valid elements of this thread's group in a tile.  The first lookup of a CTA
+    // is a binary search, later ones walk on from the previous tile's tensor.
     int seg = 0;
-    int u = 0;                                    // pipeline unit counter
-    bool timed_out = false;
-    for (int tile = tile_begin; tile < tile_end; ++tile) {
-        const int row0 = tile * kThreads;
-        const int g = row0 + tid;
-        const bool active = g < G;
-        int bucket = 0, valid = 32;
-        if (active) {
-            int local, n, b0;
-            if (a.v.n_seg == 1) {
-                local = g; n = a.v.seg0_elems; b0 = 0;
-            } else {
-                while (g >= tbl(seg + 1)) ++seg;
-                local = g - tbl(seg);
-                b0 = tbl(n1 + seg);
-                n = tbl(2 * n1 + seg);
+    bool seg_known = false;
+    auto lookup = [&](int tile, int& bucket, int& valid) {
+        const int g = tile * kThreads + tid;
+        bucket = 0;
+        valid = 0;                                 // 0: the group lies beyond the layout
+        if (g >= G) return;
+        int local, n, b0;
+        if (a.v.n_seg == 1) {
+            local = g; n = a.v.seg0_elems; b0 = 0;
+        } else {
+            if (!seg_known) {
+                int lo = 0, hi = a.v.n_seg;
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (tbl(mid) <= g) lo = mid; else hi = mid;
+                }
+                seg = lo;
+                seg_known = true;
             }
-            bucket = b0 + (int)div_gpb(a, (uint32_t)local);
-            const int left = n - local * 32;
-            valid = left < 32 ? left : 32;
+            while (g >= tbl(seg + 1)) ++seg;
+            local = g - tbl(seg);
+            b0 = tbl(n1 + seg);
+            n = tbl(2 * n1 + seg);
         }
-        float acc[32];
-#pragma unroll
-        for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
+        bucket = b0 + (int)div_gpb(a, (uint32_t)local);
+        const int left = n - local * 32;
+        valid = left < 32 ? left : 32;
+    };
 
-        if constexpr (B > 1) {
+    if constexpr (B == 1) {
+        // s = 0: every value is 0
+        for (int tile = tile_begin; tile < tile_end; ++tile) {
+            if (tid == 0) tma::store_wait_read();
+            __syncthreads();
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) = make_float4(0.f, 0.f, 0.f, 0.f);
+            tma::fence_proxy_async();
+            __syncthreads();
+            if (tid == 0) {
+                tma::store_tile_2d(out_map, smem, 0, tile * kThreads);
+                tma::store_commit();
+            }
+        }
+        if (tid == 0) tma::store_wait_read();
+        return;
+    } else {
+        // Software pipeline over the units: while unit u is decoded, the scales of unit u + 1
+        // (norm * 1/(s M) per worker of the chunk, for this thread's bucket) are already on
+        // their way in registers; they replace the current ones in the scale buffer once the
+        // decode is done.
+        int bucket, valid, nbucket = 0, nvalid = 0;
+        lookup(tile_begin, bucket, valid);
+        float nxt[MC];
+        {
+            const int mc0 = M < MC ? M : MC;
+            const float* nrm = a.norms + bucket;
+#pragma unroll
+            for (int j = 0; j < MC; ++j)
+                nxt[j] = (j < mc0 && valid > 0 && my_units > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) * unit : 0.0f;
+#pragma unroll
+            for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j];
+        }
+
+        float acc[32];
+        bool timed_out = false;
+        int u = 0;
+        for (int tile = tile_begin; tile < tile_end && !timed_out; ++tile) {
+#pragma unroll
+            for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
             for (int c = 0; c < nchunk; ++c, ++u) {
                 const int m0 = c * MC;
                 const int mc = (M - m0) < MC ? (M - m0) : MC;
-                // this thread's per-worker scales of the chunk, parked in its shared-memory column
-                const float* nrm = a.norms + (int64_t)m0 * a.v.nb + bucket;
-                for (int j = 0; j < mc; ++j)
-                    my_scales[j * kThreads] = active ? __ldg(nrm + (int64_t)j * a.v.nb) * unit : 0.0f;
+
+                // next unit: same tile and the next chunk of workers, or the first chunk of the next tile
+                const bool last_chunk = (c == nchunk - 1);
+                const bool has_next = (u + 1 < my_units);
+                int nm0 = m0 + MC;
+                if (last_chunk) {
+                    nm0 = 0;
+                    if (has_next) lookup(tile + 1, nbucket, nvalid);
+                } else {
+                    nbucket = bucket;
+                    nvalid = valid;
+                }
+                {
+                    const int nmc = (M - nm0) < MC ? (M - nm0) : MC;
+                    const float* nrm = a.norms + (int64_t)nm0 * a.v.nb + nbucket;
+#pragma unroll
+                    for (int j = 0; j < MC; ++j)
+                        nxt[j] = (has_next && j < nmc && nvalid > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) * unit : 0.0f;
+                }
 
                 const int st = u % kStages;
                 if (!tma::mbar_wait(full_bar(st), (u / kStages) & 1)) { timed_out = true; break; }
@@ -218,49 +280,50 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                     UpperHalves<B, 0>::run(wd, hi);
                     AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
                 }
+#pragma unroll
+                for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j];
+
                 // the previous tile's bulk store must have drained the output tile before it is rewritten below
-                if (c == nchunk - 1 && tid == 0) tma::store_wait_read();
+                if (last_chunk && tid == 0) tma::store_wait_read();
                 __syncthreads();                  // the stage is free again
                 if (tid == 0) {
                     const int nu = u + kStages;
                     if (nu < my_units) {
                         tma::fence_proxy_async();
                         const int ntile = tile_begin + nu / nchunk;
-                        const int nm0 = (nu % nchunk) * MC;
-                        issue_unit<B>(a, st, ntile * kThreads, nm0, (M - nm0) < MC ? (M - nm0) : MC);
+                        const int um0 = (nu % nchunk) * MC;
+                        issue_unit<B>(a, st, ntile * kThreads, um0, (M - um0) < MC ? (M - um0) : MC);
                     }
                 }
             }
             if (timed_out) break;
             Normalise<B, 0>::run(acc);
-        } else {
-            if (tid == 0) tma::store_wait_read();
+            if (valid < 32) {
+#pragma unroll
+                for (int e = 0; e < 32; ++e)
+                    if (e >= valid) acc[e] = 0.0f;
+            }
+            // own row of the swizzled output tile (conflict-free), then one bulk tensor store per tile
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) =
+                    make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+            tma::fence_proxy_async();
             __syncthreads();
+            if (tid == 0) {
+                tma::store_tile_2d(out_map, smem, 0, tile * kThreads);
+                tma::store_commit();
+            }
+            bucket = nbucket;
+            valid = nvalid;
         }
 
-        if (valid < 32) {
-#pragma unroll
-            for (int e = 0; e < 32; ++e)
-                if (e >= valid) acc[e] = 0.0f;
+        if (tid == 0) tma::store_wait_read();         // shared memory must outlive the last store's reads
+        if (timed_out) {
+            if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
+            for (int k = 1; k < kStages; ++k)
+                if (u + k < my_units) (void)tma::mbar_wait(full_bar((u + k) % kStages), ((u + k) / kStages) & 1);
         }
-        // own row of the swizzled output tile (conflict-free), then one bulk tensor store per tile
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) =
-                make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
-        tma::fence_proxy_async();
-        __syncthreads();
-        if (tid == 0) {
-            tma::store_tile_2d(out_map, smem, 0, row0);
-            tma::store_commit();
-        }
-    }
-
-    if (tid == 0) tma::store_wait_read();         // shared memory must outlive the last store's reads
-    if (timed_out) {
-        if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
-        for (int k = 1; k < kStages; ++k)
-            if (u + k < my_units) (void)tma::mbar_wait(full_bar((u + k) % kStages), ((u + k) / kStages) & 1);
     }
 }
 
