@@ -218,75 +218,103 @@ def run_cuda(args) -> dict:
     def rule_for(i):
         return dq.Rule.dynamic(T, i % T, eps_hat, alpha)
 
-    # untimed pass: the b each step will choose (needed for the byte model); also warms up
-    bits = []
-    for i in range(K):
-        rnd.norms_(pool[i % npool])
-        rnd.bits_(rule_for(i))
-        bits.append(rnd.bits())
-    for i in range(max(W, 3)):
-        rnd.step(pool[i % npool], rule_for(i), SEED, i)
-    torch.cuda.synchronize()
-    assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
-
-    names = ["bucket_norms", "choose_bits", "quantize_pack", "unpack_dequant_average"]
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(K)]
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", ""))
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    start.record()
-    for i in range(K):
-        g = pool[i % npool]
-        rule = rule_for(i)
-        e = ev[i]
-        e[0].record()
-        rnd.norms_(g)
-        e[1].record()
-        rnd.bits_(rule)
-        e[2].record()
-        rnd.quantize_(g, SEED, i)
-        e[3].record()
-        rnd.average_()
-        e[4].record()
-    end.record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    ms = start.elapsed_time(end)
-    assert rnd.read_status() == 0
-    if world > 1:
-        tmax = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
-
-    per_kernel_ms = {n: [ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)] for j, n in enumerate(names)}
-    totals = {n: sum(v) for n, v in per_kernel_ms.items()}
-    dominant = max(totals, key=totals.get)
-    elems = M * D32
-    mean_b = sum(bits) / len(bits)
-    alg_bytes = {
-        "bucket_norms": 4.0 * elems,
-        "choose_bits": 4.0 * M * L.nb,
-        "quantize_pack": (4.0 + mean_b / 8.0) * elems,
-        "unpack_dequant_average": (M * mean_b / 8.0 + 4.0) * D32,
-    }
     peak, peak_src = _peaks()
-    kernels = {}
-    for n in names:
-        avg_ms = totals[n] / K
-        gbs = alg_bytes[n] / (avg_ms * 1e-3) / 1e9
-        kernels[n] = {"avg_ms": round(avg_ms, 5), "achieved_gbs": round(gbs, 1), "frac": round(gbs / peak, 4),
-                      "share": round(totals[n] / sum(totals.values()), 4)}
+    elems = M * D32
+
+    def b_of(norm_set, t):
+        """b the rule gives at schedule step t for the norms of input set `norm_set` (synchronises)."""
+        rnd.norms_(pool[norm_set % npool])
+        rnd.bits_(dq.Rule.dynamic(T, t % T, eps_hat, alpha))
+        return rnd.bits()
+
+    # Two orders of the same four steps (both supported by the library):
+    #  "algorithm1": as Algorithm 1 of the paper runs -- quantize with b_t, which was chosen from the
+    #     previous step's norms, in ONE pass together with the norms (dq_norms_quantize_pack), average,
+    #     then choose b_{t+1} from this step's norms.  This is the timed headline.
+    #  "four_call": norms, bit rule on this step's own norms, quantize (second pass), average.
+    def run_order(order, sampler=None):
+        if order == "algorithm1":
+            names = ["norms_quantize_pack", "unpack_dequant_average", "choose_bits"]
+            bits = [b_of(0, 0)] + [b_of(i - 1, i) for i in range(1, K)]          # untimed: b of every step
+        else:
+            names = ["bucket_norms", "choose_bits", "quantize_pack", "unpack_dequant_average"]
+            bits = [b_of(i, i) for i in range(K)]
+
+        def one_step(i, e):
+            g = pool[i % npool]
+            if order == "algorithm1":
+                e[0].record(); rnd.norms_quantize_(g, SEED, i)
+                e[1].record(); rnd.average_()
+                e[2].record(); rnd.bits_(rule_for(i + 1))
+                e[3].record()
+            else:
+                e[0].record(); rnd.norms_(g)
+                e[1].record(); rnd.bits_(rule_for(i))
+                e[2].record(); rnd.quantize_(g, SEED, i)
+                e[3].record(); rnd.average_()
+                e[4].record()
+
+        nev = len(names) + 1
+        b_of(0, 0)                                  # dev_b holds b_0 before the first step
+        dummy = [torch.cuda.Event(enable_timing=True) for _ in range(nev)]
+        for i in range(max(W, 3)):
+            one_step(i, dummy)
+        b_of(0, 0)
+        torch.cuda.synchronize()
+        assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(K)]
+        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+        if sampler:
+            sampler.start()
+        start.record()
+        for i in range(K):
+            one_step(i, ev[i])
+        end.record()
+        torch.cuda.synchronize()
+        clk = sampler.stop() if sampler else None
+        t_ms = start.elapsed_time(end)
+        assert rnd.read_status() == 0
+        if world > 1:
+            tmax = torch.tensor([t_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            t_ms = float(tmax.item())
+        totals = {n: sum(ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)) for j, n in enumerate(names)}
+        mean_b = sum(bits) / len(bits)
+        alg_bytes = {
+            "bucket_norms": 4.0 * elems,
+            "choose_bits": 4.0 * M * L.nb,
+            "quantize_pack": (4.0 + mean_b / 8.0) * elems,
+            "norms_quantize_pack": (4.0 + mean_b / 8.0) * elems,
+            "unpack_dequant_average": (M * mean_b / 8.0 + 4.0) * D32,
+        }
+        kernels = {}
+        for n in names:
+            avg_ms = totals[n] / K
+            gbs = alg_bytes[n] / (avg_ms * 1e-3) / 1e9
+            kernels[n] = {"avg_ms": round(avg_ms, 5), "achieved_gbs": round(gbs, 1), "frac": round(gbs / peak, 4),
+                          "share": round(totals[n] / sum(totals.values()), 4),
+                          "algorithmic_bytes_per_launch": alg_bytes[n]}
+        return t_ms, bits, mean_b, kernels, clk, len(names) + (1 if "choose_bits" in names else 0)
+
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", ""))
+    ms, bits, mean_b, kernels, clocks, launches_per_step = run_order("algorithm1", sampler)
+    dominant = max(kernels, key=lambda n: kernels[n]["avg_ms"])
     tr = _traffic(dominant)
     roofline = {
         "kernel": dominant, "bound": "hbm", "achieved": kernels[dominant]["achieved_gbs"], "peak": peak,
         "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": (tr or {}).get("bytes_per_launch"),
         "peak_source": peak_src + "; of measured" if peak_src.startswith("measured") else peak_src + "; of fallback",
-        "algorithmic_bytes_per_launch": alg_bytes[dominant], "mean_b": round(mean_b, 3),
+        "algorithmic_bytes_per_launch": kernels[dominant]["algorithmic_bytes_per_launch"], "mean_b": round(mean_b, 3),
         "kernels": kernels,
     }
+    four = None
+    if not args.no_four_call:
+        ms4, bits4, mean_b4, kernels4, _, _ = run_order("four_call")
+        four = {"ms_per_step": ms4 / K, "value": world * 4.0 * M * w.d * K / (ms4 * 1e-3) / 1e9,
+                "mean_bits": round(mean_b4, 3), "kernels": kernels4}
 
     value = world * 4.0 * M * w.d * K / (ms * 1e-3) / 1e9
 
@@ -299,9 +327,11 @@ def run_cuda(args) -> dict:
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "bits_first_last": [bits[0], bits[-1]], "mean_bits": round(mean_b, 3),
+                   "order": "Algorithm 1: norms+quantize+pack in one pass with b_t, average, b_{t+1} from this step's norms",
                    "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": 5 * K, "roofline": roofline,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "roofline": roofline,
+        "four_call_order": four,
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -316,14 +346,14 @@ def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> d
     Ke = min(K, 10)
     host = [pool[p].cpu().pin_memory() for p in range(2)]
     for i in range(2):
-        rnd.step_host(host[i % 2], rule_for(i), SEED, i)
+        rnd.step_host(host[i % 2], rule_for(i + 1), SEED, i)
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
     s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s2.record()
     for i in range(Ke):
-        res = rnd.step_host(host[i % 2], rule_for(i), SEED, i)
+        res = rnd.step_host(host[i % 2], rule_for(i + 1), SEED, i)
     e2.record()
     torch.cuda.synchronize()
     checksum = float(res[:1024].double().abs().sum())        # the result is read on the host
@@ -361,6 +391,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-four-call", action="store_true", help="skip the secondary timing of the four separate calls")
     args = ap.parse_args()
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:

@@ -197,6 +197,23 @@ int dq_quantize_pack(const dq_layout_t* layout, const float* dev_grads, int64_t 
                      uint32_t* dev_packed, int64_t packed_stride_words,
                      int32_t* dev_status, void* stream);
 
+/* --------------------------- norms and quantizer in one pass, Eq. 5 and 6
+ * dq_bucket_norms followed by dq_quantize_pack on the same gradients, with every
+ * gradient byte read once: dev_norms receives exactly what dq_bucket_norms
+ * writes and dev_packed exactly what dq_quantize_pack writes for those norms.
+ * Algorithm 1 sets b_{t+1} from the gradients of iteration t ("Update the
+ * quantization bits b_{t+1} according to Eq. 17" follows the averaging of step
+ * t), so dev_b is known before this step's gradients are and the two steps
+ * need not be separate passes.  A step is then
+ *   dq_norms_quantize_pack (b_t) -> dq_unpack_dequant_average -> dq_choose_bits (b_{t+1}).
+ * in : dev_grads, dev_b
+ * out: dev_norms fp32 [M][nb], dev_packed (as for dq_quantize_pack)
+ * Device conditions: those of both calls. */
+int dq_norms_quantize_pack(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
+                           int32_t M, const int32_t* dev_b, uint64_t seed, uint32_t step,
+                           float* dev_norms, uint32_t* dev_packed, int64_t packed_stride_words,
+                           int32_t* dev_status, void* stream);
+
 /* ----------------------------------- Algorithm 1, server side: "Average"
  * dev_out[j] = (1/M) sum_m (code_m - s) * norm_m / s   (Eq. 5 inverted, then
  * the mean over workers); 0 for padding and when s = 0.  fp32 accumulation in

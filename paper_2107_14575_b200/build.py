@@ -17,7 +17,7 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libdq.so")
 
-SOURCES = ["dq_layout.cu", "dq_tma.cu", "dq_norms.cu", "dq_bits.cu", "dq_quantize.cu", "dq_unpack.cu"]
+SOURCES = ["dq_layout.cu", "dq_tma.cu", "dq_norms.cu", "dq_bits.cu", "dq_quantize.cu", "dq_fused.cu", "dq_unpack.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -1,0 +1,332 @@
+// dq_norms_quantize_pack: bucket norms (Eq. 5) and quantize+pack (Eq. 5/6) in one
+// pass over the gradients.
+//
+// Algorithm 1 takes b_{t+1} from the gradients of iteration t, so the bit width of
+// a step is known before its gradients are: once a bucket sits in shared
+// memory its norm can be taken and its codes emitted at once, and every gradient
+// byte is read from HBM a single time.  The norms are written out as well: the
+// server needs them for the average and for the next bit width.
+//
+// Persistent CTAs each take a contiguous range of tiles of R = 4096 / bucket
+// consecutive buckets of one worker (bucket = 32 * 2^k).  In the padded layout
+// such a run is one contiguous span of at most 128 groups, fetched by a single
+// TMA tensor copy into a ring of swizzled shared-memory stages.  Thread t of a
+// tile owns group (t % gpb) of bucket (t / gpb): it squares its 128-byte row, the
+// gpb threads of a bucket combine by shuffles (through shared memory when a
+// bucket spans several warps) exactly as dq_bucket_norms does, then the thread
+// encodes its row against that norm and the tile's words leave with 16-byte
+// coalesced stores.  HBM traffic: 4 + b/8 bytes per element.
+#include "dq_common.cuh"
+#include "dq_device.cuh"
+#include "dq_tma.cuh"
+
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kStages = 2;
+constexpr int kTileBytes = kThreads * 128;          // 16 KB
+constexpr int kMaxSmemSegs = 1023;
+
+// Dynamic shared memory, addressed only through this symbol:
+//   [0, kStages * 16 KB)   input tiles (1024-byte aligned for the 128-byte swizzle)
+//   then 128 * 16 + 4 words of output staging, 4 partial sums, the stage barriers, the tensor table
+extern __shared__ __align__(1024) unsigned char smem[];
+constexpr int kOutOffset = kStages * kTileBytes;
+constexpr int kPartOffset = kOutOffset + (kThreads * DQ_MAX_BITS + 4) * 4;
+constexpr int kBarOffset = kPartOffset + 16;
+constexpr int kTblOffset = kBarOffset + kStages * 8;
+
+__device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
+
+struct FusedArgs {
+    LayoutView v;
+    float* norms;
+    const int32_t* dev_b;
+    uint32_t* packed;
+    int64_t packed_stride;
+    int32_t* status;
+    PhiloxKeys keys;
+    uint32_t step;
+    int32_t M;
+    int32_t map_has_worker_dim;
+    int32_t gpb_shift;            // log2(groups per bucket)
+    int32_t stream_reads;         // 1: the gradients exceed the L2, read them with the evict-first policy
+    uint32_t one_bits;            // 0x3F800040, kept out of the compiler's sight (see and_or)
+};
+
+template <int B>
+__device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMap* map, const bool tbl_in_smem)
+{
+    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kTblOffset);
+    auto tbl = [&](int i) -> int { return tbl_in_smem ? tbl_s[i] : __ldg(a.v.seg_group0 + i); };
+    constexpr int s = (1 << (B - 1)) - 1;
+    const float sf = (float)s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n1 = a.v.n_seg + 1;
+    const int gpb = 1 << a.gpb_shift;
+    const int R = kThreads >> a.gpb_shift;                    // buckets per tile
+    const int nb = a.v.nb;
+    const int tiles_per_worker = (nb + R - 1) / R;
+    const int total_tiles = a.M * tiles_per_worker;
+    const int bsz = gpb * 32;
+    const int tile_begin = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
+    const int tile_end = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
+
+    // first group and valid elements of bucket k; `seg` is a walking hint (buckets only move forward)
+    auto locate = [&](int k, int& seg, int& first_group, int& len) {
+        int local, n, g0;
+        if (a.v.n_seg == 1) {
+            local = k; n = a.v.seg0_elems; g0 = 0;
+        } else {
+            while (k >= tbl(n1 + seg + 1)) ++seg;
+            local = k - tbl(n1 + seg);
+            n = tbl(2 * n1 + seg);
+            g0 = tbl(seg);
+        }
+        first_group = g0 + (local << a.gpb_shift);
+        const int left = n - local * bsz;
+        len = left < bsz ? left : bsz;
+    };
+    auto advance = [&](int& mm, int& rr) {
+        if (++rr == tiles_per_worker) { rr = 0; ++mm; }
+    };
+
+    int m = tile_begin / tiles_per_worker, kt = tile_begin - m * tiles_per_worker;
+    int pm = m, pkt = kt, ptile = tile_begin, pseg = 0, pseg_m = m;
+    const uint64_t policy = tma::policy_evict_first();
+    auto issue = [&](int st) {
+        if (pm != pseg_m) { pseg = 0; pseg_m = pm; }
+        int row0, len0;
+        locate(pkt * R, pseg, row0, len0);
+        tma::mbar_expect_tx(full_bar(st), kTileBytes);
+        if (a.stream_reads)
+            tma::load_tile_3d_hint(smem + st * kTileBytes, map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0, policy);
+        else
+            tma::load_tile_3d(smem + st * kTileBytes, map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0);
+    };
+#pragma unroll
+    for (int st = 0; st < kStages; ++st) {
+        if (ptile < tile_end && tid == 0) issue(st);
+        ++ptile;
+        advance(pm, pkt);
+    }
+
+    const int r = tid >> a.gpb_shift;            // bucket of the tile this thread works on
+    const int l = tid & (gpb - 1);               // its group inside that bucket
+    float* part = reinterpret_cast<float*>(smem + kPartOffset);
+    uint32_t* out_words = reinterpret_cast<uint32_t*>(smem + kOutOffset);
+    int seg = 0, seg0 = 0, seg1 = 0, seg_m = -1;
+    int it = 0;
+    bool timed_out = false, bad = false;
+    for (int tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, kt)) {
+        const int st = it % kStages;
+        if (m != seg_m) { seg = 0; seg0 = 0; seg1 = 0; seg_m = m; }
+        const int k0 = kt * R;
+        const int k = k0 + r;
+        const int k_last = (k0 + R < nb ? k0 + R : nb) - 1;
+        int row0, len0, first = 0, len = 0, first_last, len_last;
+        locate(k0, seg0, row0, len0);
+        locate(k_last, seg1, first_last, len_last);
+        if (k < nb) locate(k, seg, first, len);
+        const int span = first_last + ((len_last + 31) >> 5) - row0;       // groups this tile covers
+        const int row = first - row0 + l;        // this thread's row of the tile
+        int valid = len - l * 32;                // elements of its group that count
+        valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
+
+        if (!tma::mbar_wait(full_bar(st), (it / kStages) & 1)) { timed_out = true; break; }
+
+        // ---- norm of the bucket (same operations, same order as dq_bucket_norms)
+        unsigned char* base = smem + st * kTileBytes;
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        if (valid > 0) {
+            if (valid == 32) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
+                    a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                }
+            } else {                             // last group of a tensor: what follows is padding
+                for (int e = 0; e < valid; ++e) {
+                    const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
+                    a0 = fmaf(x, x, a0);
+                }
+            }
+        }
+        float sum = (a0 + a1) + (a2 + a3);
+        const int w = gpb < 32 ? gpb : 32;
+        for (int o = w >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (gpb > 32) {
+            if (lane == 0) part[warp] = sum;
+            __syncthreads();
+            sum = 0.f;
+            const int w0 = (tid >> a.gpb_shift << a.gpb_shift) >> 5;        // first warp of this bucket
+            for (int i = 0; i < (gpb >> 5); ++i) sum += part[w0 + i];
+        }
+        const float nrm = sqrtf(sum);
+        if (l == 0 && k < nb) {
+            a.norms[(int64_t)m * nb + k] = nrm;
+            bad |= !isfinite(nrm);
+        }
+
+        // ---- codes of this thread's group against that norm
+        const int off = (int)(((int64_t)row0 * B) & 3);      // staging keeps the stream's 16-byte phase
+        if (valid > 0) {
+            const float inv = (nrm >= 0x1p-100f) ? __fdiv_rz(sf, nrm) : 0.0f;
+            unsigned char* rowp = base + row * 128;
+            const uint32_t sw = (uint32_t)(row & 7);
+            if (valid < 32) {                    // padding after a tensor's end encodes as 0
+                for (int e = valid; e < 32; ++e)
+                    *reinterpret_cast<float*>(rowp + ((((e >> 2) ^ sw) << 4) | ((e & 3) << 2))) = 0.0f;
+                tma::fence_proxy_async();        // these stores precede the next bulk copy into this stage
+            }
+            uint32_t acc[B];
+            if constexpr (B == 1) {
+                acc[0] = 0u;
+            } else {
+                uint32_t cur = 0;
+                const uint32_t q0 = (uint32_t)(row0 + row) * 4u;
+#define DQ_BLOCK(C)                                                                                             \
+                encode_block<B, C>(acc, cur,                                                                    \
+                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)), \
+                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
+                                   inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+                DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
+#undef DQ_BLOCK
+            }
+#pragma unroll
+            for (int i = 0; i < B; ++i) out_words[off + row * B + i] = acc[i];
+        }
+        __syncthreads();
+
+        // ---- the tile's span * B words.  Word i of the tile sits at out_words[off + i] and goes to
+        //      aligned_dst[off + i]; whole quads move 16 bytes at a time, the ragged ends word by word.
+        {
+            const int jend = off + span * B;
+            uint32_t* aligned_dst = a.packed + (int64_t)m * a.packed_stride + ((int64_t)row0 * B - off);
+            const int q0 = off ? 1 : 0, q1 = jend >> 2;          // full quads [q0, q1)
+            for (int q = q0 + tid; q < q1; q += kThreads)
+                reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
+            if (off && tid >= off && tid < 4 && tid < jend) aligned_dst[tid] = out_words[tid];       // head
+            int ts = q1 * 4;                                                                         // tail
+            if (off && ts < 4) ts = 4;
+            if (tid < jend - ts) aligned_dst[ts + tid] = out_words[ts + tid];
+        }
+        __syncthreads();                         // everyone is done with this stage and with the staging area
+        if (ptile < tile_end && tid == 0) {
+            tma::fence_proxy_async();
+            issue(st);
+        }
+        ++ptile;
+        advance(pm, pkt);
+    }
+    if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
+    if (timed_out) {
+        if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
+        for (int j = it + 1; j < it + kStages; ++j)
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kStages), (j / kStages) & 1);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 5)
+norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
+{
+    const int b = __ldg(a.dev_b);
+    if (b < 1 || b > DQ_MAX_BITS) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
+        return;
+    }
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
+        return;
+    }
+    if (tma::smem_addr(smem) & 1023u) {
+        if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
+        return;
+    }
+    const bool tbl_in_smem = a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs;
+    if (tbl_in_smem) {
+        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
+        for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
+    }
+    if (threadIdx.x == 0) {
+        tma::prefetch_tensor_map(&map);
+#pragma unroll
+        for (int st = 0; st < kStages; ++st) tma::mbar_init(full_bar(st), 1);
+        tma::fence_barrier_init();
+    }
+    __syncthreads();
+
+    switch (b) {
+#define DQ_CASE(BB) case BB: fused_tiles<BB>(a, &map, tbl_in_smem); break;
+        DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
+        DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
+#undef DQ_CASE
+        default: break;
+    }
+}
+
+}  // namespace
+
+extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
+                                      int32_t M, const int32_t* dev_b, uint64_t seed, uint32_t step,
+                                      float* dev_norms, uint32_t* dev_packed, int64_t packed_stride_words,
+                                      int32_t* dev_status, void* stream)
+{
+    const int rc = dq_check_common(L, M);
+    if (rc != DQ_OK) return rc;
+    if (!dev_grads || !dev_norms || !dev_b || !dev_packed || !dev_status) return DQ_ERR_ARG;
+    if (!aligned16(dev_grads) || !aligned16(dev_packed) || (worker_stride_elems % 32) != 0 ||
+        (packed_stride_words % 4) != 0 || (reinterpret_cast<uintptr_t>(dev_norms) & 3u) ||
+        (reinterpret_cast<uintptr_t>(dev_b) & 3u) || (reinterpret_cast<uintptr_t>(dev_status) & 3u))
+        return DQ_ERR_ALIGN;
+    if (M > 1 && worker_stride_elems < L->padded && worker_stride_elems != 0) return DQ_ERR_RANGE;
+    if (packed_stride_words < L->padded / 32) return DQ_ERR_RANGE;
+
+    const uint32_t gpb = (uint32_t)(L->bucket / 32);
+    if ((gpb & (gpb - 1)) != 0) {
+        // bucket sizes that are not 32 * 2^k: the two separate passes give the same result
+        const int r1 = dq_bucket_norms(L, dev_grads, worker_stride_elems, M, dev_norms, dev_status, stream);
+        if (r1 != DQ_OK) return r1;
+        return dq_quantize_pack(L, dev_grads, worker_stride_elems, M, dev_norms, dev_b, seed, step, dev_packed,
+                                packed_stride_words, dev_status, stream);
+    }
+
+    FusedArgs a;
+    a.v = make_view(L);
+    a.norms = dev_norms;
+    a.dev_b = dev_b;
+    a.packed = dev_packed;
+    a.packed_stride = packed_stride_words;
+    a.status = dev_status;
+    a.keys = make_philox_keys(seed);
+    a.step = step;
+    a.M = M;
+    a.one_bits = 0x3F800040u;
+    a.gpb_shift = 0;
+    while ((1u << a.gpb_shift) < gpb) ++a.gpb_shift;
+    a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
+    const bool worker_dim = (M > 1 && worker_stride_elems != 0);
+    a.map_has_worker_dim = worker_dim ? 1 : 0;
+
+    CUtensorMap map;
+    const uint64_t dims[3] = {32, (uint64_t)a.v.total_groups, worker_dim ? (uint64_t)M : 1};
+    const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
+    const uint32_t box[3] = {32, (uint32_t)kThreads, 1};
+    if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
+                              CU_TENSOR_MAP_SWIZZLE_128B))
+        return DQ_ERR_CUDA;
+
+    size_t smem_need = (size_t)kTblOffset;
+    if (L->n_seg > 1 && L->n_seg <= kMaxSmemSegs) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
+    if (cudaFuncSetAttribute(norms_quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DQ_ERR_CUDA;
+    }
+    const int R = kThreads >> a.gpb_shift;
+    const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
+    int64_t blocks = (int64_t)dq_sm_count() * 5;       // five 42 KB CTAs per SM
+    if (blocks > tiles) blocks = tiles;
+    norms_quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
+    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}

@@ -66,43 +66,6 @@ __device__ __forceinline__ uint32_t div_gpb(const QuantizeArgs& a, uint32_t n)
     return (uint32_t)(((uint64_t)n * a.div_magic) >> 33);     // exact for n < 2^26, divisor <= 128
 }
 
-// Stores the B words of one group into the warp's staging area (stride B words
-// between lanes; the widest access the alignment allows keeps bank conflicts low).
-template <int B>
-__device__ __forceinline__ void stage_words(uint32_t* __restrict__ dst, const uint32_t (&acc)[B])
-{
-    if constexpr (B % 4 == 0) {
-#pragma unroll
-        for (int i = 0; i < B / 4; ++i)
-            reinterpret_cast<uint4*>(dst)[i] = make_uint4(acc[4 * i], acc[4 * i + 1], acc[4 * i + 2], acc[4 * i + 3]);
-    } else if constexpr (B % 2 == 0) {
-#pragma unroll
-        for (int i = 0; i < B / 2; ++i)
-            reinterpret_cast<uint2*>(dst)[i] = make_uint2(acc[2 * i], acc[2 * i + 1]);
-    } else {
-#pragma unroll
-        for (int i = 0; i < B; ++i) dst[i] = acc[i];
-    }
-}
-
-// Encodes elements 8C .. 8C+7 of a group (one Philox block) and appends the codes.
-template <int B, int C>
-__device__ __forceinline__ void encode_block(uint32_t (&acc)[B], uint32_t& cur, const float4 lo, const float4 hi,
-                                             const float inv, const uint32_t q, const uint32_t m,
-                                             const uint32_t step, const PhiloxKeys& keys, const uint32_t ob)
-{
-    uint32_t w[4];
-    philox4x32_10(q, 0u, m, step, keys, w);
-    push_code<B, 8 * C + 0>(acc, cur, encode<B, 0>(lo.x, inv, w[0], ob));
-    push_code<B, 8 * C + 1>(acc, cur, encode<B, 1>(lo.y, inv, w[0], ob));
-    push_code<B, 8 * C + 2>(acc, cur, encode<B, 0>(lo.z, inv, w[1], ob));
-    push_code<B, 8 * C + 3>(acc, cur, encode<B, 1>(lo.w, inv, w[1], ob));
-    push_code<B, 8 * C + 4>(acc, cur, encode<B, 0>(hi.x, inv, w[2], ob));
-    push_code<B, 8 * C + 5>(acc, cur, encode<B, 1>(hi.y, inv, w[2], ob));
-    push_code<B, 8 * C + 6>(acc, cur, encode<B, 0>(hi.z, inv, w[3], ob));
-    push_code<B, 8 * C + 7>(acc, cur, encode<B, 1>(hi.w, inv, w[3], ob));
-}
-
 template <int B>
 __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUtensorMap* map, const bool tbl_in_smem)
 {

@@ -24,7 +24,7 @@ SYMBOLS = [
     "dq_layout_table_bytes", "dq_layout_bind_device_table",
     "dq_bucket_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
     "dq_choose_bits_noalloc_max_norms", "dq_choose_bits_noalloc",
-    "dq_quantize_pack", "dq_unpack_dequant_average", "dq_status_string",
+    "dq_quantize_pack", "dq_norms_quantize_pack", "dq_unpack_dequant_average", "dq_status_string",
 ]
 
 
@@ -93,6 +93,8 @@ def lib():
         L.dq_choose_bits_noalloc.argtypes = [vp, vp, i32, C.POINTER(Rule), vp, vp, vp]
         L.dq_quantize_pack.restype = C.c_int
         L.dq_quantize_pack.argtypes = [vp, vp, i64, i32, vp, vp, u64, u32, vp, i64, vp, vp]
+        L.dq_norms_quantize_pack.restype = C.c_int
+        L.dq_norms_quantize_pack.argtypes = [vp, vp, i64, i32, vp, u64, u32, vp, vp, i64, vp, vp]
         L.dq_unpack_dequant_average.restype = C.c_int
         L.dq_unpack_dequant_average.argtypes = [vp, vp, i64, vp, i32, vp, vp, vp, vp]
         L.dq_status_string.restype = C.c_char_p
@@ -208,6 +210,14 @@ def quantize_pack(layout: Layout, grads, worker_stride_elems: int, M: int, norms
     _check(lib().dq_quantize_pack(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(norms),
                                   _ptr(dev_b), int(seed) & (2 ** 64 - 1), int(step) & 0xFFFFFFFF, _ptr(packed),
                                   int(packed_stride_words), _ptr(status), _stream(stream)), "dq_quantize_pack")
+
+
+def norms_quantize_pack(layout: Layout, grads, worker_stride_elems: int, M: int, dev_b, seed: int, step: int,
+                        norms, packed, packed_stride_words: int, status, stream=None) -> None:
+    _check(lib().dq_norms_quantize_pack(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(dev_b),
+                                        int(seed) & (2 ** 64 - 1), int(step) & 0xFFFFFFFF, _ptr(norms), _ptr(packed),
+                                        int(packed_stride_words), _ptr(status), _stream(stream)),
+           "dq_norms_quantize_pack")
 
 
 def unpack_dequant_average(layout: Layout, packed, packed_stride_words: int, norms, M: int, dev_b, out, status,

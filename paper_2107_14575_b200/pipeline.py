@@ -46,6 +46,11 @@ class Round:
         dq.quantize_pack(self.layout, grads, self.stride, self.M, self.norms, self.dev_b, seed, step,
                          self.packed, self.packed_stride, self.status)
 
+    def norms_quantize_(self, grads, seed: int, step: int) -> None:
+        """Norms and quantize+pack in one pass, with the b already in ``dev_b``."""
+        dq.norms_quantize_pack(self.layout, grads, self.stride, self.M, self.dev_b, seed, step, self.norms,
+                               self.packed, self.packed_stride, self.status)
+
     def average_(self) -> None:
         dq.unpack_dequant_average(self.layout, self.packed, self.packed_stride, self.norms, self.M, self.dev_b,
                                   self.out, self.status)
@@ -58,8 +63,18 @@ class Round:
         self.average_()
         return self.out
 
-    def step_host(self, host_grads: torch.Tensor, rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
-        """Whole round on pinned host gradients [M, stride]; returns a pinned host tensor [D32].
+    def step_fused(self, grads, next_rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
+        """One round in the order of Algorithm 1: quantize with the b chosen after the
+        previous round (one pass over the gradients), average, then choose the next b from
+        this round's norms.  ``dev_b`` must hold a b (a first call to ``bits_`` with the
+        initial b_0 does that)."""
+        self.norms_quantize_(grads, seed, step)
+        self.average_()
+        self.bits_(next_rule)
+        return self.out
+
+    def step_host(self, host_grads: torch.Tensor, next_rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
+        """``step_fused`` on pinned host gradients [M, stride]; returns a pinned host tensor [D32].
 
         Copies the gradients to the device, runs the round and copies the
         average back, all on the current stream; the caller synchronises.
@@ -68,7 +83,7 @@ class Round:
             self._dev_in = torch.empty((self.M, self.stride), dtype=torch.float32, device=self.device)
             self._host_out = torch.empty(self.layout.D32, dtype=torch.float32).pin_memory()
         self._dev_in.copy_(host_grads, non_blocking=True)
-        self.step(self._dev_in, rule, seed, step)
+        self.step_fused(self._dev_in, next_rule, seed, step)
         self._host_out.copy_(self.out, non_blocking=True)
         return self._host_out
 

@@ -75,6 +75,15 @@ class GpuRound:
                          self.g_packed.view, self.pstride, self.status)
         return self.g_packed.view.cpu().numpy().view(np.uint32).reshape(self.M, self.pstride)
 
+    def norms_quantize(self, seed, step, fill=None):
+        """Fused call: returns (norms [M, nb], packed [M, pstride])."""
+        if fill is not None:
+            self.g_packed.view.fill_(fill)
+        dq.norms_quantize_pack(self.lay, self.grads, self.stride, self.M, self.g_b.view, seed, step,
+                               self.g_norms.view, self.g_packed.view, self.pstride, self.status)
+        return (self.g_norms.view.cpu().numpy().reshape(self.M, self.lay.nb),
+                self.g_packed.view.cpu().numpy().view(np.uint32).reshape(self.M, self.pstride))
+
     def average(self, fill=None) -> np.ndarray:
         if fill is not None:
             self.g_out.view.fill_(fill)

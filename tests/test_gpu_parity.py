@@ -196,6 +196,75 @@ def test_quantize_with_gpu_norms_differs_only_at_ties(G, name, b):
     assert np.array_equal(got[:, : ref.packed_words(b)], want)
 
 
+# ------------------------------------------- norms + quantize in one pass
+
+@pytest.mark.parametrize("name", sorted(CASES))
+def test_fused_norms_quantize_equals_the_two_passes(G, name):
+    """dq_norms_quantize_pack writes the norms of dq_bucket_norms and the words of
+    dq_quantize_pack for those norms, bit for bit; and the words are the oracle's for them."""
+    w = CASES[name]
+    ref, g = _make(w, pad_value=7e29)
+    r = G.GpuRound(w.segments, w.bucket, w.M)
+    r.set_grads(g)
+    norms_sep = r.norms().copy()
+    for b, step in ((4, 0), (1, 2), (7, 3), (16, 9)):
+        r.set_b(b)
+        packed_sep = r.quantize(SEED, step, fill=-1).copy()
+        r.g_norms.view.fill_(-1.0)
+        norms_fused, packed_fused = r.norms_quantize(SEED, step, fill=-1)
+        assert np.array_equal(norms_fused, norms_sep)
+        assert np.array_equal(packed_fused, packed_sep)
+        nw = ref.packed_words(b)
+        want = oracle.quantize_pack(ref, g, norms_fused, b, SEED, step)
+        assert np.array_equal(packed_fused[:, :nw], want)
+        assert np.all(packed_fused[:, nw:] == 0xFFFFFFFF)
+    assert np.all(np.abs(norms_sep - oracle.bucket_norms(ref, g)) <= NORM_RTOL * oracle.bucket_norms(ref, g))
+    assert r.read_status() == 0 and r.guards_intact()
+
+
+@pytest.mark.parametrize("bucket", [32, 64, 128, 256, 1024, 2048, 4096, 96, 160])
+def test_fused_bucket_sizes(G, bucket):
+    w = W.config_flat(d=3 * 4096 + 1234, M=3, bucket=bucket, sigma=2.0)
+    ref, g = _make(w)
+    r = G.GpuRound(w.segments, bucket, w.M)
+    r.set_grads(g)
+    for b in (3, 8):
+        r.set_b(b)
+        norms, packed = r.norms_quantize(5, 1, fill=-1)
+        ref_norms = oracle.bucket_norms(ref, g)
+        assert np.all(np.abs(norms - ref_norms) <= NORM_RTOL * ref_norms)
+        want = oracle.quantize_pack(ref, g, norms, b, 5, 1)
+        assert np.array_equal(packed[:, : ref.packed_words(b)], want)
+    assert r.read_status() == 0 and r.guards_intact()
+
+
+def test_fused_step_order_of_algorithm_1(G):
+    """quantize with b_t (one pass) -> average -> b_{t+1} from this step's norms."""
+    w = CASES["resnet/64"]
+    T = 10
+    alpha = (2.4e-3) ** (1.0 / T)
+    r = G.GpuRound(w.segments, w.bucket, w.M)
+    b = 4                                                      # b_0, an input of Algorithm 1
+    r.set_b(b)
+    eps_hat = None
+    for t in range(T):
+        ref, g = _make(w, step=t)
+        r.set_grads(g)
+        norms, packed = r.norms_quantize(SEED, t)
+        want = oracle.quantize_pack(ref, g, norms, b, SEED, t)
+        assert np.array_equal(packed[:, : ref.packed_words(b)], want)
+        out = r.average()
+        assert G.rel_l2(out, oracle.unpack_dequant_average(ref, want, norms, b)) <= AVG_RTOL
+        if eps_hat is None:
+            G2 = float((norms.astype(np.float64) ** 2).sum() / w.M)
+            eps_hat = T * alpha ** (T - 1) * G2 / 36.0
+        if t + 1 < T:
+            b_next = r.bits(G.dq.Rule.dynamic(T, t + 1, eps_hat, alpha))
+            assert b_next[0] == oracle.choose_bits(norms, T, t + 1, eps_hat, alpha)[0]
+            b = b_next[0]
+    assert b > 4 and r.read_status() == 0 and r.guards_intact()
+
+
 # ------------------------------------------------------------------ bit rule
 
 def test_choose_bits_matches_oracle(G):
