@@ -29,12 +29,14 @@ constexpr int kMaxSmemSegs = 1023;
 
 // Dynamic shared memory, addressed only through this symbol:
 //   [0, kStages * 16 KB)   input tiles (1024-byte aligned for the 128-byte swizzle)
-//   then 128 * 16 + 4 words of output staging, 4 partial sums, the stage barriers, the tensor table
+//   then 128 * 16 + 4 words of output staging, 4 partial sums, the stage barriers, per-stage tile
+//   geometry, the tensor table
 extern __shared__ __align__(1024) unsigned char smem[];
 constexpr int kOutOffset = kStages * kTileBytes;
 constexpr int kPartOffset = kOutOffset + (kThreads * DQ_MAX_BITS + 4) * 4;
 constexpr int kBarOffset = kPartOffset + 16;
-constexpr int kTblOffset = kBarOffset + kStages * 8;
+constexpr int kMetaOffset = kBarOffset + kStages * 8;        // per stage: first group and span of the tile
+constexpr int kTblOffset = kMetaOffset + kStages * 8;
 
 __device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
 
@@ -55,10 +57,12 @@ struct FusedArgs {
 };
 
 template <int B>
-__device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMap* map, const bool tbl_in_smem)
+__device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMap* map)
 {
+    // the tensor table of a multi-tensor layout always sits in shared memory here (the host
+    // takes the two-pass route for layouts too large for that)
     const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kTblOffset);
-    auto tbl = [&](int i) -> int { return tbl_in_smem ? tbl_s[i] : __ldg(a.v.seg_group0 + i); };
+    auto tbl = [&](int i) -> int { return tbl_s[i]; };
     constexpr int s = (1 << (B - 1)) - 1;
     const float sf = (float)s;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -94,10 +98,20 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
     int m = tile_begin / tiles_per_worker, kt = tile_begin - m * tiles_per_worker;
     int pm = m, pkt = kt, ptile = tile_begin, pseg = 0, pseg_m = m;
     const uint64_t policy = tma::policy_evict_first();
+    int* meta = reinterpret_cast<int*>(smem + kMetaOffset);
+    int pseg1 = 0;
+    // The issuing thread works out where the tile starts and how many groups it spans, and
+    // leaves both in shared memory for the consumers of that stage (they read them after the
+    // barrier that precedes the stage's next use, or after the prologue's barrier).
     auto issue = [&](int st) {
-        if (pm != pseg_m) { pseg = 0; pseg_m = pm; }
-        int row0, len0;
-        locate(pkt * R, pseg, row0, len0);
+        if (pm != pseg_m) { pseg = 0; pseg1 = 0; pseg_m = pm; }
+        const int k0 = pkt * R;
+        const int k_last = (k0 + R < nb ? k0 + R : nb) - 1;
+        int row0, len0, first_last, len_last;
+        locate(k0, pseg, row0, len0);
+        locate(k_last, pseg1, first_last, len_last);
+        meta[2 * st] = row0;
+        meta[2 * st + 1] = first_last + ((len_last + 31) >> 5) - row0;
         tma::mbar_expect_tx(full_bar(st), kTileBytes);
         if (a.stream_reads)
             tma::load_tile_3d_hint(smem + st * kTileBytes, map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0, policy);
@@ -110,25 +124,22 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
         ++ptile;
         advance(pm, pkt);
     }
+    __syncthreads();                             // the prologue's tile geometry is visible
 
     const int r = tid >> a.gpb_shift;            // bucket of the tile this thread works on
     const int l = tid & (gpb - 1);               // its group inside that bucket
     float* part = reinterpret_cast<float*>(smem + kPartOffset);
     uint32_t* out_words = reinterpret_cast<uint32_t*>(smem + kOutOffset);
-    int seg = 0, seg0 = 0, seg1 = 0, seg_m = -1;
+    int seg = 0, seg_m = -1;
     int it = 0;
     bool timed_out = false, bad = false;
     for (int tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, kt)) {
         const int st = it % kStages;
-        if (m != seg_m) { seg = 0; seg0 = 0; seg1 = 0; seg_m = m; }
-        const int k0 = kt * R;
-        const int k = k0 + r;
-        const int k_last = (k0 + R < nb ? k0 + R : nb) - 1;
-        int row0, len0, first = 0, len = 0, first_last, len_last;
-        locate(k0, seg0, row0, len0);
-        locate(k_last, seg1, first_last, len_last);
+        if (m != seg_m) { seg = 0; seg_m = m; }
+        const int k = kt * R + r;
+        const int row0 = meta[2 * st], span = meta[2 * st + 1];
+        int first = 0, len = 0;
         if (k < nb) locate(k, seg, first, len);
-        const int span = first_last + ((len_last + 31) >> 5) - row0;       // groups this tile covers
         const int row = first - row0 + l;        // this thread's row of the tile
         int valid = len - l * 32;                // elements of its group that count
         valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
@@ -153,8 +164,13 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
             }
         }
         float sum = (a0 + a1) + (a2 + a3);
-        const int w = gpb < 32 ? gpb : 32;
-        for (int o = w >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        // butterfly over the threads of the bucket: the steps up to its size, smallest distance last
+        // (the same order as in dq_bucket_norms)
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float other = __shfl_xor_sync(0xffffffffu, sum, o);
+            if (o < gpb) sum += other;
+        }
         if (gpb > 32) {
             if (lane == 0) part[warp] = sum;
             __syncthreads();
@@ -243,8 +259,7 @@ norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_con
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
         return;
     }
-    const bool tbl_in_smem = a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs;
-    if (tbl_in_smem) {
+    if (a.v.n_seg > 1) {
         int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
         for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
     }
@@ -257,7 +272,7 @@ norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_con
     __syncthreads();
 
     switch (b) {
-#define DQ_CASE(BB) case BB: fused_tiles<BB>(a, &map, tbl_in_smem); break;
+#define DQ_CASE(BB) case BB: fused_tiles<BB>(a, &map); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -283,8 +298,9 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
     if (packed_stride_words < L->padded / 32) return DQ_ERR_RANGE;
 
     const uint32_t gpb = (uint32_t)(L->bucket / 32);
-    if ((gpb & (gpb - 1)) != 0) {
-        // bucket sizes that are not 32 * 2^k: the two separate passes give the same result
+    if ((gpb & (gpb - 1)) != 0 || L->n_seg > kMaxSmemSegs) {
+        // bucket sizes that are not 32 * 2^k, or more tensors than the kernel's shared-memory table
+        // holds: the two separate passes give the same result
         const int r1 = dq_bucket_norms(L, dev_grads, worker_stride_elems, M, dev_norms, dev_status, stream);
         if (r1 != DQ_OK) return r1;
         return dq_quantize_pack(L, dev_grads, worker_stride_elems, M, dev_norms, dev_b, seed, step, dev_packed,
@@ -317,7 +333,7 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
         return DQ_ERR_CUDA;
 
     size_t smem_need = (size_t)kTblOffset;
-    if (L->n_seg > 1 && L->n_seg <= kMaxSmemSegs) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
+    if (L->n_seg > 1) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
     if (cudaFuncSetAttribute(norms_quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
         (void)cudaGetLastError();
         return DQ_ERR_CUDA;
