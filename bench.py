@@ -45,19 +45,34 @@ def _peaks():
     return 6650.0, "fallback (earlier measurement on this pool)"
 
 
+# Sources whose text decides what each timed call moves through DRAM: a counter capture
+# stays valid only while their digest is the one stored beside it.
+KERNEL_SOURCES = {
+    "norms_quantize_pack": ["dq_fused.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
+    "quantize_pack": ["dq_quantize.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
+    "bucket_norms": ["dq_norms.cu", "dq_tma.cuh", "dq_common.cuh"],
+    "unpack_dequant_average": ["dq_unpack.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
+    "choose_bits": ["dq_bits.cu", "dq_common.cuh"],
+}
+
+
+def _sources_digest(kernel_key: str) -> str:
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES[kernel_key]:
+        with open(os.path.join(ROOT, "paper_2107_14575_b200", "csrc", name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
 def _traffic(kernel_key: str):
-    """DRAM bytes per launch from the committed ncu capture, or None if the kernel
-    source changed since the capture."""
+    """DRAM bytes per launch from the committed ncu capture, or None if one of the
+    kernel's sources changed since the capture."""
     path = os.path.join(ROOT, "profiles", "dram_traffic.json")
     if not os.path.exists(path):
         return None
     with open(path) as fh:
         rec = json.load(fh).get(kernel_key)
-    if not rec:
-        return None
-    src = os.path.join(ROOT, rec["source"])
-    digest = hashlib.sha256(open(src, "rb").read()).hexdigest()
-    if digest != rec["sha256"]:
+    if not rec or rec.get("sha256") != _sources_digest(kernel_key):
         return None
     return rec
 
@@ -392,7 +407,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-four-call", action="store_true", help="skip the secondary timing of the four separate calls")
+    ap.add_argument("--source-digests", action="store_true",
+                    help="print the digest of each kernel's sources (stored beside a counter capture) and exit")
     args = ap.parse_args()
+    if args.source_digests:
+        print(json.dumps({k: _sources_digest(k) for k in KERNEL_SOURCES}, indent=1))
+        return
     if args.impl == "reference":
         if int(os.environ.get("RANK", "0")) != 0:
             return

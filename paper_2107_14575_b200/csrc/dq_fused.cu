@@ -7,15 +7,18 @@
 // byte is read from HBM a single time.  The norms are written out as well: the
 // server needs them for the average and for the next bit width.
 //
-// Persistent CTAs each take a contiguous range of tiles of R = 4096 / bucket
-// consecutive buckets of one worker (bucket = 32 * 2^k).  In the padded layout
-// such a run is one contiguous span of at most 128 groups, fetched by a single
-// TMA tensor copy into a ring of swizzled shared-memory stages.  Thread t of a
-// tile owns group (t % gpb) of bucket (t / gpb): it squares its 128-byte row, the
-// gpb threads of a bucket combine by shuffles (through shared memory when a
-// bucket spans several warps) exactly as dq_bucket_norms does, then the thread
-// encodes its row against that norm and the tile's words leave with 16-byte
-// coalesced stores.  HBM traffic: 4 + b/8 bytes per element.
+// Work is cut into tiles of R consecutive buckets of one worker (bucket = 32 * 2^k
+// elements = gpb groups).  In the padded layout such a run is one contiguous span
+// of at most R * gpb groups, fetched by a single TMA tensor copy into a ring of
+// swizzled shared-memory stages.  The thread that owns group l of bucket r of the
+// tile squares its 128-byte row, the gpb threads of a bucket combine by shuffles
+// exactly as dq_bucket_norms does, then the thread encodes its row against that
+// norm and the tile's words leave with 16-byte coalesced stores.
+//  * Buckets of up to 1024 elements (gpb <= 32): every WARP is a pipeline of its own
+//    over tiles of 32 / gpb buckets; no CTA barrier in the loop.
+//  * Larger buckets (up to 4096 elements): the CTA is the pipeline, tiles of
+//    128 / gpb buckets, partial sums of a bucket's warps meet in shared memory.
+// HBM traffic: 4 + b/8 bytes per element.
 #include "dq_common.cuh"
 #include "dq_device.cuh"
 #include "dq_tma.cuh"
@@ -37,6 +40,24 @@ constexpr int kPartOffset = kOutOffset + (kThreads * DQ_MAX_BITS + 4) * 4;
 constexpr int kBarOffset = kPartOffset + 16;
 constexpr int kMetaOffset = kBarOffset + kStages * 8;        // per stage: first group and span of the tile
 constexpr int kTblOffset = kMetaOffset + kStages * 8;
+
+// The per-warp pipelines use another carving of the same symbol:
+//   [0, kWarps * kWStages * 4 KB)   input tiles, warp-major; a consumed tile doubles as the staging
+//   area of its warp's output words; then the stage barriers and the tensor table
+constexpr int kWarps = kThreads / 32;
+constexpr int kWStages = 2;
+constexpr int kWTileBytes = 32 * 128;
+constexpr int kWBarOffset = kWarps * kWStages * kWTileBytes;
+constexpr int kWTblOffset = kWBarOffset + kWarps * kWStages * 8;
+
+__device__ __forceinline__ uint64_t* wbar(int warp, int st)
+{
+    return reinterpret_cast<uint64_t*>(smem + kWBarOffset) + warp * kWStages + st;
+}
+__device__ __forceinline__ unsigned char* wstage(int warp, int st)
+{
+    return smem + (warp * kWStages + st) * kWTileBytes;
+}
 
 __device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
 
@@ -243,6 +264,219 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
     }
 }
 
+// ---- buckets that fit one warp: per-warp pipelines ---------------------------------
+template <int B>
+__device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUtensorMap* map)
+{
+    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kWTblOffset);
+    auto tbl = [&](int i) -> int { return tbl_s[i]; };
+    constexpr int s = (1 << (B - 1)) - 1;
+    const float sf = (float)s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n1 = a.v.n_seg + 1;
+    const int gpb = 1 << a.gpb_shift;
+    const int R = 32 >> a.gpb_shift;                          // buckets per warp tile
+    const int nb = a.v.nb;
+    const int tiles_per_worker = (nb + R - 1) / R;
+    const int64_t total_tiles = (int64_t)a.M * tiles_per_worker;
+    const int bsz = gpb * 32;
+    const int64_t nwarps = (int64_t)gridDim.x * kWarps;
+    const int64_t gw = (int64_t)blockIdx.x * kWarps + warp;
+    const int64_t tile_begin = gw * total_tiles / nwarps;
+    const int64_t tile_end = (gw + 1) * total_tiles / nwarps;
+
+    // first group and valid elements of bucket k; `seg` is a walking hint (buckets only move forward)
+    auto locate = [&](int k, int& seg, int& first_group, int& len) {
+        int local, n, g0;
+        if (a.v.n_seg == 1) {
+            local = k; n = a.v.seg0_elems; g0 = 0;
+        } else {
+            while (k >= tbl(n1 + seg + 1)) ++seg;
+            local = k - tbl(n1 + seg);
+            n = tbl(2 * n1 + seg);
+            g0 = tbl(seg);
+        }
+        first_group = g0 + (local << a.gpb_shift);
+        const int left = n - local * bsz;
+        len = left < bsz ? left : bsz;
+    };
+    auto advance = [&](int& mm, int& rr) {
+        if (++rr == tiles_per_worker) { rr = 0; ++mm; }
+    };
+
+    int m = (int)(tile_begin / tiles_per_worker), kt = (int)(tile_begin - (int64_t)m * tiles_per_worker);
+    int pm = m, pkt = kt, pseg = 0, pseg_m = m;
+    int64_t ptile = tile_begin;
+    const uint64_t policy = tma::policy_evict_first();
+    // lane 0 fetches: a tile starts at the first group of its first bucket and is always 32 rows
+    // (rows past the tile's span belong to later tiles or lie outside the tensor map; nobody reads them)
+    auto issue = [&](int st) {
+        if (pm != pseg_m) { pseg = 0; pseg_m = pm; }
+        int row0, len0;
+        locate(pkt * R, pseg, row0, len0);
+        tma::mbar_expect_tx(wbar(warp, st), kWTileBytes);
+        if (a.stream_reads)
+            tma::load_tile_3d_hint(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? pm : 0, policy);
+        else
+            tma::load_tile_3d(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? pm : 0);
+    };
+#pragma unroll
+    for (int st = 0; st < kWStages; ++st) {
+        if (ptile < tile_end && lane == 0) issue(st);
+        ++ptile;
+        advance(pm, pkt);
+    }
+
+    const int r = lane >> a.gpb_shift;           // bucket of the tile this lane works on
+    const int l = lane & (gpb - 1);              // its group inside that bucket
+    int seg = 0, seg_m = -1;
+    int it = 0;
+    bool timed_out = false, bad = false;
+    for (int64_t tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, kt)) {
+        const int st = it % kWStages;
+        if (m != seg_m) { seg = 0; seg_m = m; }
+        const int k = kt * R + r;
+        int first = 0, len = 0;
+        if (k < nb) locate(k, seg, first, len);
+        const int row0 = __shfl_sync(0xffffffffu, first, 0);          // lane 0 owns the tile's first group
+        const int row = first - row0 + l;        // this lane's row of the tile
+        int valid = len - l * 32;                // elements of its group that count
+        valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
+        const int span = __reduce_max_sync(0xffffffffu, valid > 0 ? row + 1 : 0);   // groups the tile covers
+
+        // every lane polls the barrier itself; the verdict is made warp-uniform so that the
+        // warp-level synchronisations below are always reached by all lanes or by none
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, st), (it / kWStages) & 1))) { timed_out = true; break; }
+
+        // ---- norm of the bucket (same operations, same order as dq_bucket_norms)
+        unsigned char* base = wstage(warp, st);
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        if (valid > 0) {
+            if (valid == 32) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
+                    a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                }
+            } else {                             // last group of a tensor: what follows is padding
+                for (int e = 0; e < valid; ++e) {
+                    const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
+                    a0 = fmaf(x, x, a0);
+                }
+            }
+        }
+        float sum = (a0 + a1) + (a2 + a3);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float other = __shfl_xor_sync(0xffffffffu, sum, o);
+            if (o < gpb) sum += other;
+        }
+        const float nrm = sqrtf(sum);
+        if (l == 0 && k < nb) {
+            a.norms[(int64_t)m * nb + k] = nrm;
+            bad |= !isfinite(nrm);
+        }
+
+        // ---- codes of this lane's group against that norm
+        uint32_t acc[B];
+        if (valid > 0) {
+            const float inv = (nrm >= 0x1p-100f) ? __fdiv_rz(sf, nrm) : 0.0f;
+            unsigned char* rowp = base + row * 128;
+            const uint32_t sw = (uint32_t)(row & 7);
+            if (valid < 32) {                    // padding after a tensor's end encodes as 0
+                for (int e = valid; e < 32; ++e)
+                    *reinterpret_cast<float*>(rowp + ((((e >> 2) ^ sw) << 4) | ((e & 3) << 2))) = 0.0f;
+            }
+            if constexpr (B == 1) {
+                acc[0] = 0u;
+            } else {
+                uint32_t cur = 0;
+                const uint32_t q0 = (uint32_t)(row0 + row) * 4u;
+#define DQ_BLOCK(C)                                                                                             \
+                encode_block<B, C>(acc, cur,                                                                    \
+                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)), \
+                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
+                                   inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+                DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
+#undef DQ_BLOCK
+            }
+        }
+
+        // The warp has read all of its rows: the stage now carries the tile's span * B words.  Word i
+        // sits at out_words[off + i] and goes to aligned_dst[off + i], so that the staging area keeps
+        // the 16-byte phase of the output stream; whole quads move 16 bytes per lane, the ragged
+        // ends word by word.
+        __syncwarp();
+        uint32_t* out_words = reinterpret_cast<uint32_t*>(base);
+        const int off = (int)(((int64_t)row0 * B) & 3);
+        if (valid > 0) {
+#pragma unroll
+            for (int i = 0; i < B; ++i) out_words[off + row * B + i] = acc[i];
+        }
+        tma::fence_proxy_async();                // these stores precede the bulk copy that refills the stage
+        __syncwarp();
+        {
+            const int jend = off + span * B;
+            uint32_t* aligned_dst = a.packed + (int64_t)m * a.packed_stride + ((int64_t)row0 * B - off);
+            const int q0 = off ? 1 : 0, q1 = jend >> 2;          // full quads [q0, q1)
+            for (int q = q0 + lane; q < q1; q += 32)
+                reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
+            if (off && lane >= off && lane < 4 && lane < jend) aligned_dst[lane] = out_words[lane];   // head
+            int ts = q1 * 4;                                                                          // tail
+            if (off && ts < 4) ts = 4;
+            if (lane < jend - ts) aligned_dst[ts + lane] = out_words[ts + lane];
+        }
+        __syncwarp();
+        if (ptile < tile_end && lane == 0) issue(st);
+        ++ptile;
+        advance(pm, pkt);
+    }
+    if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
+    if (timed_out) {
+        if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
+        // give copies still in flight a bounded chance to land before the CTA's shared memory is released
+        for (int j = it + 1; j < it + kWStages; ++j)
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(wbar(warp, j % kWStages), (j / kWStages) & 1);
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 6)
+norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
+{
+    const int b = __ldg(a.dev_b);
+    if (b < 1 || b > DQ_MAX_BITS) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
+        return;
+    }
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
+        return;
+    }
+    if (tma::smem_addr(smem) & 1023u) {
+        if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
+        return;
+    }
+    if (a.v.n_seg > 1) {
+        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kWTblOffset);
+        for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
+    }
+    if (threadIdx.x == 0) {
+        tma::prefetch_tensor_map(&map);
+        for (int i = 0; i < kWarps * kWStages; ++i) tma::mbar_init(wbar(0, i), 1);
+        tma::fence_barrier_init();
+    }
+    __syncthreads();
+
+    switch (b) {
+#define DQ_CASE(BB) case BB: fused_warp_tiles<BB>(a, &map); break;
+        DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
+        DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
+#undef DQ_CASE
+        default: break;
+    }
+}
+
+// ---- buckets that span several warps: the CTA is the pipeline -----------------------
 __global__ void __launch_bounds__(kThreads, 5)
 norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
@@ -324,25 +558,41 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
     const bool worker_dim = (M > 1 && worker_stride_elems != 0);
     a.map_has_worker_dim = worker_dim ? 1 : 0;
 
+    const bool per_warp = gpb <= 32;
     CUtensorMap map;
     const uint64_t dims[3] = {32, (uint64_t)a.v.total_groups, worker_dim ? (uint64_t)M : 1};
     const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
-    const uint32_t box[3] = {32, (uint32_t)kThreads, 1};
+    const uint32_t box[3] = {32, per_warp ? 32u : (uint32_t)kThreads, 1};
     if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
                               CU_TENSOR_MAP_SWIZZLE_128B))
         return DQ_ERR_CUDA;
 
-    size_t smem_need = (size_t)kTblOffset;
-    if (L->n_seg > 1) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
-    if (cudaFuncSetAttribute(norms_quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
-        (void)cudaGetLastError();
-        return DQ_ERR_CUDA;
+    const size_t tbl_bytes = L->n_seg > 1 ? (size_t)3 * (L->n_seg + 1) * 4 : 0;
+    if (per_warp) {
+        const size_t smem_need = (size_t)kWTblOffset + tbl_bytes;
+        if (cudaFuncSetAttribute(norms_quantize_pack_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_need) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return DQ_ERR_CUDA;
+        }
+        const int R = 32 >> a.gpb_shift;
+        const int64_t warp_tiles = (int64_t)M * ((L->nb + R - 1) / R);
+        int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
+        if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
+        norms_quantize_pack_warp_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
+    } else {
+        const size_t smem_need = (size_t)kTblOffset + tbl_bytes;
+        if (cudaFuncSetAttribute(norms_quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_need) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return DQ_ERR_CUDA;
+        }
+        const int R = kThreads >> a.gpb_shift;
+        const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
+        int64_t blocks = (int64_t)dq_sm_count() * 5;   // five 42 KB CTAs per SM
+        if (blocks > tiles) blocks = tiles;
+        norms_quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
     }
-    const int R = kThreads >> a.gpb_shift;
-    const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
-    int64_t blocks = (int64_t)dq_sm_count() * 5;       // five 42 KB CTAs per SM
-    if (blocks > tiles) blocks = tiles;
-    norms_quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
