@@ -258,10 +258,7 @@ def run_cuda(args) -> dict:
         def one_step(i, e):
             g = pool[i % npool]
             if order == "algorithm1":
-                e[0].record(); rnd.norms_quantize_(g, SEED, i)
-                e[1].record(); rnd.average_()
-                e[2].record(); rnd.bits_(rule_for(i + 1))
-                e[3].record()
+                rnd.step_fused(g, rule_for(i + 1), SEED, i, overlap=not args.no_overlap, events=e)
             else:
                 e[0].record(); rnd.norms_(g)
                 e[1].record(); rnd.bits_(rule_for(i))
@@ -269,7 +266,7 @@ def run_cuda(args) -> dict:
                 e[3].record(); rnd.average_()
                 e[4].record()
 
-        nev = len(names) + 1
+        nev = 5
         b_of(0, 0)                                  # dev_b holds b_0 before the first step
         dummy = [torch.cuda.Event(enable_timing=True) for _ in range(nev)]
         for i in range(max(W, 3)):
@@ -296,7 +293,10 @@ def run_cuda(args) -> dict:
             tmax = torch.tensor([t_ms], dtype=torch.float64, device=dev)
             dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
             t_ms = float(tmax.item())
-        totals = {n: sum(ev[i][j].elapsed_time(ev[i][j + 1]) for i in range(K)) for j, n in enumerate(names)}
+        # algorithm1: events 0-1 bracket the fused call, 1-2 the average, 3-4 the bit rule (on its own
+        # stream when it overlaps the average); four_call: 0-1-2-3-4 in sequence
+        spans = [(0, 1), (1, 2), (3, 4)] if order == "algorithm1" else [(0, 1), (1, 2), (2, 3), (3, 4)]
+        totals = {n: sum(ev[i][p].elapsed_time(ev[i][q]) for i in range(K)) for n, (p, q) in zip(names, spans)}
         mean_b = sum(bits) / len(bits)
         alg_bytes = {
             "bucket_norms": 4.0 * elems,
@@ -342,7 +342,8 @@ def run_cuda(args) -> dict:
         "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "bits_first_last": [bits[0], bits[-1]], "mean_bits": round(mean_b, 3),
-                   "order": "Algorithm 1: norms+quantize+pack in one pass with b_t, average, b_{t+1} from this step's norms",
+                   "order": "Algorithm 1: norms+quantize+pack in one pass with b_t, average, b_{t+1} from this step's norms"
+                            + ("" if args.no_overlap else " (bit rule on a second stream beside the average)"),
                    "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "roofline": roofline,
@@ -407,6 +408,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-four-call", action="store_true", help="skip the secondary timing of the four separate calls")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="run the bit rule after the average on the same stream instead of beside it")
     ap.add_argument("--source-digests", action="store_true",
                     help="print the digest of each kernel's sources (stored beside a counter capture) and exit")
     args = ap.parse_args()

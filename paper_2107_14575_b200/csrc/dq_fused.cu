@@ -264,7 +264,122 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
     }
 }
 
+// ---- buckets that fit one warp: a tile that touches the end of a tensor ---------------
+// General route of the per-warp pipelines, kept out of line so that the common case does
+// not pay for its registers: buckets may be short, rows of the tile may belong to nobody,
+// and every lane looks its bucket up in the tensor table.  Leaves the lane's words in the
+// staging area (the consumed stage) and returns the tile's span in groups, plus 256 if a
+// norm is not finite.
+template <int B>
+__device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* base, const int row0, const int m, const int kt)
+{
+    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kWTblOffset);
+    constexpr int s = (1 << (B - 1)) - 1;
+    const float sf = (float)s;
+    const int lane = threadIdx.x & 31;
+    const int n1 = a.v.n_seg + 1;
+    const int gpb = 1 << a.gpb_shift;
+    const int bsz = gpb * 32;
+    const int R = 32 >> a.gpb_shift;
+    const int nb = a.v.nb;
+    const int r = lane >> a.gpb_shift;           // bucket of the tile this lane works on
+    const int l = lane & (gpb - 1);              // its group inside that bucket
+    const int k = kt * R + r;
+    int first = 0, len = 0;
+    if (k < nb) {
+        int local, n, g0;
+        if (a.v.n_seg == 1) {
+            local = k; n = a.v.seg0_elems; g0 = 0;
+        } else {
+            int lo = 0, hi = a.v.n_seg;          // last tensor whose first bucket is <= k
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (tbl_s[n1 + mid] <= k) lo = mid; else hi = mid;
+            }
+            local = k - tbl_s[n1 + lo];
+            n = tbl_s[2 * n1 + lo];
+            g0 = tbl_s[lo];
+        }
+        first = g0 + (local << a.gpb_shift);
+        const int left = n - local * bsz;
+        len = left < bsz ? left : bsz;
+    }
+    const int row = first - row0 + l;            // this lane's row of the tile
+    int valid = len - l * 32;                    // elements of its group that count
+    valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
+    const int span = __reduce_max_sync(0xffffffffu, valid > 0 ? row + 1 : 0);   // groups the tile covers
+
+    // norm of the bucket (same operations, same order as dq_bucket_norms)
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    if (valid > 0) {
+        if (valid == 32) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
+                a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+            }
+        } else {                                 // last group of a tensor: what follows is padding
+            for (int e = 0; e < valid; ++e) {
+                const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
+                a0 = fmaf(x, x, a0);
+            }
+        }
+    }
+    float sum = (a0 + a1) + (a2 + a3);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xffffffffu, sum, o);
+        if (o < gpb) sum += other;
+    }
+    const float nrm = sqrtf(sum);
+    int bad = 0;
+    if (l == 0 && k < nb) {
+        a.norms[(int64_t)m * nb + k] = nrm;
+        bad = isfinite(nrm) ? 0 : 256;
+    }
+
+    // codes of this lane's group against that norm
+    uint32_t acc[B];
+    if (valid > 0) {
+        const float inv = (nrm >= 0x1p-100f) ? __fdiv_rz(sf, nrm) : 0.0f;
+        unsigned char* rowp = base + row * 128;
+        const uint32_t sw = (uint32_t)(row & 7);
+        if (valid < 32) {                        // padding after a tensor's end encodes as 0
+            for (int e = valid; e < 32; ++e)
+                *reinterpret_cast<float*>(rowp + ((((e >> 2) ^ sw) << 4) | ((e & 3) << 2))) = 0.0f;
+        }
+        if constexpr (B == 1) {
+            acc[0] = 0u;
+        } else {
+            uint32_t cur = 0;
+            const uint32_t q0 = (uint32_t)(row0 + row) * 4u;
+#define DQ_BLOCK(C)                                                                                             \
+            encode_block<B, C>(acc, cur,                                                                        \
+                               *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)),     \
+                               *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
+                               inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+            DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
+#undef DQ_BLOCK
+        }
+    }
+    __syncwarp();                                // the warp has read all of its rows
+    uint32_t* out_words = reinterpret_cast<uint32_t*>(base);
+    const int off = (int)(((int64_t)row0 * B) & 3);
+    if (valid > 0) {
+#pragma unroll
+        for (int i = 0; i < B; ++i) out_words[off + row * B + i] = acc[i];
+    }
+    return span | __reduce_or_sync(0xffffffffu, bad);
+}
+
 // ---- buckets that fit one warp: per-warp pipelines ---------------------------------
+//
+// Most warp tiles are "regular": all of their 32 / gpb buckets are full buckets of one
+// tensor, so lane i owns row i, every element counts and the tile spans 32 groups.  Whether
+// a tile is regular, and where it starts, depends on the layout alone; the warp works it out
+// two tiles ahead from a cached description of the tensor it is in (when it fetches the
+// tile) and keeps the answer in a two-deep register queue for the consumer side.  Only
+// tiles that touch the end of a tensor take the general route with per-lane table walks.
 template <int B>
 __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUtensorMap* map)
 {
@@ -275,147 +390,167 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n1 = a.v.n_seg + 1;
     const int gpb = 1 << a.gpb_shift;
+    const int bsz_shift = a.gpb_shift + 5;
     const int R = 32 >> a.gpb_shift;                          // buckets per warp tile
     const int nb = a.v.nb;
     const int tiles_per_worker = (nb + R - 1) / R;
     const int64_t total_tiles = (int64_t)a.M * tiles_per_worker;
-    const int bsz = gpb * 32;
     const int64_t nwarps = (int64_t)gridDim.x * kWarps;
     const int64_t gw = (int64_t)blockIdx.x * kWarps + warp;
     const int64_t tile_begin = gw * total_tiles / nwarps;
     const int64_t tile_end = (gw + 1) * total_tiles / nwarps;
 
-    // first group and valid elements of bucket k; `seg` is a walking hint (buckets only move forward)
-    auto locate = [&](int k, int& seg, int& first_group, int& len) {
-        int local, n, g0;
-        if (a.v.n_seg == 1) {
-            local = k; n = a.v.seg0_elems; g0 = 0;
-        } else {
-            while (k >= tbl(n1 + seg + 1)) ++seg;
-            local = k - tbl(n1 + seg);
-            n = tbl(2 * n1 + seg);
-            g0 = tbl(seg);
-        }
-        first_group = g0 + (local << a.gpb_shift);
-        const int left = n - local * bsz;
-        len = left < bsz ? left : bsz;
-    };
     auto advance = [&](int& mm, int& rr) {
         if (++rr == tiles_per_worker) { rr = 0; ++mm; }
     };
 
+    // ---- producer side: the tensor the fetches are in (first bucket, first group, first bucket
+    //      that is not full) and the description of a tile
+    int c_b0 = 0, c_g0 = 0, c_full_end = a.v.n_seg == 1 ? (a.v.seg0_elems >> bsz_shift) : 0;
+    // first group of tile kt2 of any worker, bit 31 set if the tile is regular (identical in all lanes)
+    auto describe = [&](int kt2) -> uint32_t {
+        const int k0 = kt2 * R;
+        if (k0 < c_b0 || k0 + R > c_full_end) {
+            // not inside the full buckets of the cached tensor: look the tile's tensor up again
+            if (a.v.n_seg > 1) {
+                int lo = 0, hi = a.v.n_seg;      // last tensor whose first bucket is <= k0
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (tbl(n1 + mid) <= k0) lo = mid; else hi = mid;
+                }
+                c_b0 = tbl(n1 + lo);
+                c_g0 = tbl(lo);
+                c_full_end = c_b0 + (tbl(2 * n1 + lo) >> bsz_shift);
+            }
+        }
+        const uint32_t regular = (k0 + R <= c_full_end) ? 0x80000000u : 0u;
+        return (uint32_t)(c_g0 + ((k0 - c_b0) << a.gpb_shift)) | regular;
+    };
+
+    const int n_tiles = (int)(tile_end - tile_begin);
     int m = (int)(tile_begin / tiles_per_worker), kt = (int)(tile_begin - (int64_t)m * tiles_per_worker);
-    int pm = m, pkt = kt, pseg = 0, pseg_m = m;
-    int64_t ptile = tile_begin;
-    const uint64_t policy = tma::policy_evict_first();
+    int pm = m, pkt = kt;
     // lane 0 fetches: a tile starts at the first group of its first bucket and is always 32 rows
     // (rows past the tile's span belong to later tiles or lie outside the tensor map; nobody reads them)
-    auto issue = [&](int st) {
-        if (pm != pseg_m) { pseg = 0; pseg_m = pm; }
-        int row0, len0;
-        locate(pkt * R, pseg, row0, len0);
+    auto issue = [&](int st, int row0) {
         tma::mbar_expect_tx(wbar(warp, st), kWTileBytes);
         if (a.stream_reads)
-            tma::load_tile_3d_hint(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? pm : 0, policy);
+            tma::load_tile_3d_hint(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? pm : 0,
+                                   tma::policy_evict_first());
         else
             tma::load_tile_3d(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? pm : 0);
     };
+    uint32_t d_cur = 0, d_nxt = 0;
 #pragma unroll
     for (int st = 0; st < kWStages; ++st) {
-        if (ptile < tile_end && lane == 0) issue(st);
-        ++ptile;
+        uint32_t d = 0;
+        if (st < n_tiles) {
+            d = describe(pkt);
+            if (lane == 0) issue(st, (int)(d & 0x7fffffffu));
+        }
+        if (st == 0) d_cur = d; else d_nxt = d;
         advance(pm, pkt);
     }
 
     const int r = lane >> a.gpb_shift;           // bucket of the tile this lane works on
     const int l = lane & (gpb - 1);              // its group inside that bucket
-    int seg = 0, seg_m = -1;
+    // byte offset of lane's row in stage 0 of this warp with the row's swizzle phase folded in:
+    // chunk c of the row sits at offset own_row ^ (c << 4)
+    const uint32_t own_row0 = (uint32_t)(warp * kWStages * kWTileBytes + lane * 128 + ((lane & 7) << 4));
     int it = 0;
     bool timed_out = false, bad = false;
-    for (int64_t tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, kt)) {
+    for (; it < n_tiles; ++it, advance(m, kt)) {
         const int st = it % kWStages;
-        if (m != seg_m) { seg = 0; seg_m = m; }
-        const int k = kt * R + r;
-        int first = 0, len = 0;
-        if (k < nb) locate(k, seg, first, len);
-        const int row0 = __shfl_sync(0xffffffffu, first, 0);          // lane 0 owns the tile's first group
-        const int row = first - row0 + l;        // this lane's row of the tile
-        int valid = len - l * 32;                // elements of its group that count
-        valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
-        const int span = __reduce_max_sync(0xffffffffu, valid > 0 ? row + 1 : 0);   // groups the tile covers
+        const int row0 = (int)(d_cur & 0x7fffffffu);
+        const bool regular = (d_cur >> 31) != 0;
+        unsigned char* base = wstage(warp, st);
+        uint32_t* out_words = reinterpret_cast<uint32_t*>(base);
+        int span = 32;
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
         // warp-level synchronisations below are always reached by all lanes or by none
         if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, st), (it / kWStages) & 1))) { timed_out = true; break; }
 
-        // ---- norm of the bucket (same operations, same order as dq_bucket_norms)
-        unsigned char* base = wstage(warp, st);
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        if (valid > 0) {
-            if (valid == 32) {
+        if (regular) {
+            // ---- norm of the bucket (same operations, same order as dq_bucket_norms)
+            const uint32_t own = own_row0 + (uint32_t)(st * kWTileBytes);
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
-                    a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
-                }
-            } else {                             // last group of a tensor: what follows is padding
-                for (int e = 0; e < valid; ++e) {
-                    const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
-                    a0 = fmaf(x, x, a0);
-                }
+            for (int c = 0; c < 8; ++c) {
+                const float4 x = *reinterpret_cast<const float4*>(smem + (own ^ (uint32_t)(c << 4)));
+                a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
             }
-        }
-        float sum = (a0 + a1) + (a2 + a3);
+            float sum = (a0 + a1) + (a2 + a3);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float other = __shfl_xor_sync(0xffffffffu, sum, o);
-            if (o < gpb) sum += other;
-        }
-        const float nrm = sqrtf(sum);
-        if (l == 0 && k < nb) {
-            a.norms[(int64_t)m * nb + k] = nrm;
-            bad |= !isfinite(nrm);
-        }
-
-        // ---- codes of this lane's group against that norm
-        uint32_t acc[B];
-        if (valid > 0) {
+            for (int o = 16; o > 0; o >>= 1) {
+                const float other = __shfl_xor_sync(0xffffffffu, sum, o);
+                if (o < gpb) sum += other;
+            }
+            const float nrm = sqrtf(sum);
+            if (l == 0) {
+                a.norms[(int64_t)m * nb + (kt * R + r)] = nrm;
+                bad |= !isfinite(nrm);
+            }
+            // ---- codes of this lane's group against that norm
             const float inv = (nrm >= 0x1p-100f) ? __fdiv_rz(sf, nrm) : 0.0f;
-            unsigned char* rowp = base + row * 128;
-            const uint32_t sw = (uint32_t)(row & 7);
-            if (valid < 32) {                    // padding after a tensor's end encodes as 0
-                for (int e = valid; e < 32; ++e)
-                    *reinterpret_cast<float*>(rowp + ((((e >> 2) ^ sw) << 4) | ((e & 3) << 2))) = 0.0f;
-            }
+            uint32_t acc[B];
             if constexpr (B == 1) {
                 acc[0] = 0u;
             } else {
                 uint32_t cur = 0;
-                const uint32_t q0 = (uint32_t)(row0 + row) * 4u;
+                const uint32_t q0 = (uint32_t)(row0 + lane) * 4u;
 #define DQ_BLOCK(C)                                                                                             \
                 encode_block<B, C>(acc, cur,                                                                    \
-                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)), \
-                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
+                                   *reinterpret_cast<const float4*>(smem + (own ^ (uint32_t)((2 * (C)) << 4))), \
+                                   *reinterpret_cast<const float4*>(smem + (own ^ (uint32_t)((2 * (C) + 1) << 4))), \
                                    inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
                 DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
 #undef DQ_BLOCK
             }
+            __syncwarp();                        // the warp has read all of its rows
+            if constexpr (B % 4 == 0) {
+                // 32 * B words from a 16-byte aligned position: B / 4 quads per lane, no ragged ends
+                stage_words<B>(out_words + lane * B, acc);
+                tma::fence_proxy_async();        // these stores precede the bulk copy that refills the stage
+                __syncwarp();
+                uint4* dst = reinterpret_cast<uint4*>(a.packed + (int64_t)m * a.packed_stride + (int64_t)row0 * B);
+#pragma unroll
+                for (int i = 0; i < B / 4; ++i) dst[lane + 32 * i] = reinterpret_cast<const uint4*>(out_words)[lane + 32 * i];
+                span = 0;                        // nothing left for the general copy below
+            } else {
+                // 32 * B words from word `off` of a 16-byte unit: quads 0 (or 1) .. 8B - 1 in full, the
+                // 4 - off words before quad 1 and the off words after the last quad one by one
+                const int off = (int)(((int64_t)row0 * B) & 3);
+#pragma unroll
+                for (int i = 0; i < B; ++i) out_words[off + lane * B + i] = acc[i];
+                tma::fence_proxy_async();
+                __syncwarp();
+                uint32_t* aligned_dst = a.packed + (int64_t)m * a.packed_stride + ((int64_t)row0 * B - off);
+#pragma unroll
+                for (int i = 0; i < (8 * B + 31) / 32; ++i) {
+                    const int q = lane + 32 * i;
+                    if (q < 8 * B && (q > 0 || off == 0))
+                        reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
+                }
+                if (off != 0 && lane < 4) {
+                    const int idx = lane >= off ? lane : 32 * B + lane;
+                    aligned_dst[idx] = out_words[idx];
+                }
+                span = 0;
+            }
+        } else {
+            const int res = irregular_tile<B>(a, base, row0, m, kt);
+            span = res & 0xff;
+            bad |= (res >> 8) != 0;
         }
 
-        // The warp has read all of its rows: the stage now carries the tile's span * B words.  Word i
-        // sits at out_words[off + i] and goes to aligned_dst[off + i], so that the staging area keeps
-        // the 16-byte phase of the output stream; whole quads move 16 bytes per lane, the ragged
-        // ends word by word.
-        __syncwarp();
-        uint32_t* out_words = reinterpret_cast<uint32_t*>(base);
-        const int off = (int)(((int64_t)row0 * B) & 3);
-        if (valid > 0) {
-#pragma unroll
-            for (int i = 0; i < B; ++i) out_words[off + row * B + i] = acc[i];
-        }
-        tma::fence_proxy_async();                // these stores precede the bulk copy that refills the stage
-        __syncwarp();
-        {
+        // The stage now carries the tile's span * B words.  Word i sits at out_words[off + i] and
+        // goes to aligned_dst[off + i], so that the staging area keeps the 16-byte phase of the
+        // output stream; whole quads move 16 bytes per lane, the ragged ends word by word.
+        if (span > 0) {
+            tma::fence_proxy_async();            // the staging stores precede the bulk copy that refills the stage
+            __syncwarp();
+            const int off = (int)(((int64_t)row0 * B) & 3);
             const int jend = off + span * B;
             uint32_t* aligned_dst = a.packed + (int64_t)m * a.packed_stride + ((int64_t)row0 * B - off);
             const int q0 = off ? 1 : 0, q1 = jend >> 2;          // full quads [q0, q1)
@@ -427,8 +562,15 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
             if (lane < jend - ts) aligned_dst[ts + lane] = out_words[ts + lane];
         }
         __syncwarp();
-        if (ptile < tile_end && lane == 0) issue(st);
-        ++ptile;
+
+        // refill the stage with the tile two ahead and move the queue
+        uint32_t d_new = 0;
+        if (it + kWStages < n_tiles) {
+            d_new = describe(pkt);
+            if (lane == 0) issue(st, (int)(d_new & 0x7fffffffu));
+        }
+        d_cur = d_nxt;
+        d_nxt = d_new;
         advance(pm, pkt);
     }
     if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
@@ -436,7 +578,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
         if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
         // give copies still in flight a bounded chance to land before the CTA's shared memory is released
         for (int j = it + 1; j < it + kWStages; ++j)
-            if (tile_begin + j < tile_end) (void)tma::mbar_wait(wbar(warp, j % kWStages), (j / kWStages) & 1);
+            if (j < n_tiles) (void)tma::mbar_wait(wbar(warp, j % kWStages), (j / kWStages) & 1);
     }
 }
 

@@ -1,9 +1,10 @@
-"""One DQ-SGD communication round on one GPU: buffers plus the four library calls.
+"""One DQ-SGD communication round on one GPU: buffers plus the library calls.
 
 ``Round`` owns the device buffers (torch tensors) of a fixed layout and worker
 count and issues norms -> bit rule -> quantize+pack -> unpack+average on the
-current stream.  It adds no arithmetic of its own: every step is a kernel of
-the C-ABI library.
+current stream, or, in the order of Algorithm 1, norms+quantize+pack -> average
+with the next bit width chosen on a second stream meanwhile.  It adds no
+arithmetic of its own: every step is a kernel of the C-ABI library.
 """
 from __future__ import annotations
 
@@ -26,13 +27,24 @@ class Round:
         self.norms = torch.empty((M, L.nb), dtype=torch.float32, device=self.device)
         self.packed = torch.empty((M, self.packed_stride), dtype=torch.int32, device=self.device)
         self.out = torch.empty(L.D32, dtype=torch.float32, device=self.device)
-        self.dev_b = torch.zeros(2, dtype=torch.int32, device=self.device)
+        # two (b, s) slots of 16 bytes: the rounds of ``step_fused`` alternate between them, so that
+        # the next b can be written while the average still reads the current one
+        self._b = torch.zeros((2, 4), dtype=torch.int32, device=self.device)
+        self._cur = 0
+        self._side = None
+        self._ev_norms = None
+        self._ev_bits = None
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self.scratch_bytes = dq.choose_bits_scratch_bytes(L, M)
         self.scratch = torch.empty(max(self.scratch_bytes, 256), dtype=torch.uint8, device=self.device)
         self._host_in = None
         self._host_out = None
         self._dev_in = None
+
+    @property
+    def dev_b(self) -> torch.Tensor:
+        """The (b, s) slot the calls read and ``bits_`` writes."""
+        return self._b[self._cur]
 
     # ---- the four calls, on device-resident gradients [M, stride] fp32 ----
     def norms_(self, grads) -> None:
@@ -63,14 +75,51 @@ class Round:
         self.average_()
         return self.out
 
-    def step_fused(self, grads, next_rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
+    def step_fused(self, grads, next_rule: dq.Rule, seed: int, step: int, overlap: bool = True,
+                   events=None) -> torch.Tensor:
         """One round in the order of Algorithm 1: quantize with the b chosen after the
-        previous round (one pass over the gradients), average, then choose the next b from
+        previous round (one pass over the gradients), average, and choose the next b from
         this round's norms.  ``dev_b`` must hold a b (a first call to ``bits_`` with the
-        initial b_0 does that)."""
+        initial b_0 does that); on return it holds the next one.
+
+        With ``overlap`` the bit rule runs on a second stream next to the average: it needs
+        only the norms, and writes the other (b, s) slot.  The current stream waits for it
+        before it goes on.  ``events`` = (e0, e1, e2, s0, s1) are recorded around the three
+        calls (e* on the current stream, s* around the bit rule on its own stream).
+        """
+        main = torch.cuda.current_stream(self.device)
+        if events:
+            events[0].record(main)
         self.norms_quantize_(grads, seed, step)
-        self.average_()
-        self.bits_(next_rule)
+        if events:
+            events[1].record(main)
+        if not overlap:
+            self.average_()
+            if events:
+                events[2].record(main)
+                events[3].record(main)
+            self.bits_(next_rule)
+            if events:
+                events[4].record(main)
+            return self.out
+        if self._side is None:
+            self._side = torch.cuda.Stream(self.device)
+            self._ev_norms = torch.cuda.Event()
+            self._ev_bits = torch.cuda.Event()
+        self._ev_norms.record(main)
+        self._side.wait_event(self._ev_norms)
+        if events:
+            events[3].record(self._side)
+        dq.choose_bits(self.layout, self.norms, self.M, next_rule, self._b[1 - self._cur], self.scratch,
+                       self.scratch_bytes, self.status, stream=self._side)
+        if events:
+            events[4].record(self._side)
+        self._ev_bits.record(self._side)
+        self.average_()                      # reads the current slot
+        if events:
+            events[2].record(main)
+        main.wait_event(self._ev_bits)
+        self._cur = 1 - self._cur
         return self.out
 
     def step_host(self, host_grads: torch.Tensor, next_rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
