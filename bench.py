@@ -192,12 +192,10 @@ def run_cuda(args) -> dict:
     import torch
     import torch.distributed as dist
 
-    from paper_2107_14575_b200 import dq, workloads
+    from paper_2107_14575_b200 import dq, replicas, workloads
     from paper_2107_14575_b200.pipeline import Round
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = replicas.env_rank()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
@@ -289,10 +287,7 @@ def run_cuda(args) -> dict:
         clk = sampler.stop() if sampler else None
         t_ms = start.elapsed_time(end)
         assert rnd.read_status() == 0
-        if world > 1:
-            tmax = torch.tensor([t_ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            t_ms = float(tmax.item())
+        t_ms = replicas.max_over_ranks(t_ms, dev)
         # algorithm1: events 0-1 bracket the fused call, 1-2 the average, 3-4 the bit rule (on its own
         # stream when it overlaps the average); four_call: 0-1-2-3-4 in sequence
         spans = [(0, 1), (1, 2), (3, 4)] if order == "algorithm1" else [(0, 1), (1, 2), (2, 3), (3, 4)]
@@ -328,10 +323,10 @@ def run_cuda(args) -> dict:
     four = None
     if not args.no_four_call:
         ms4, bits4, mean_b4, kernels4, _, _ = run_order("four_call")
-        four = {"ms_per_step": ms4 / K, "value": world * 4.0 * M * w.d * K / (ms4 * 1e-3) / 1e9,
+        four = {"ms_per_step": ms4 / K, "value": replicas.whole_job_rate(4.0 * M * w.d * K, world, ms4) / 1e9,
                 "mean_bits": round(mean_b4, 3), "kernels": kernels4}
 
-    value = world * 4.0 * M * w.d * K / (ms * 1e-3) / 1e9
+    value = replicas.whole_job_rate(4.0 * M * w.d * K, world, ms) / 1e9
 
     # ---- end to end: pinned host gradients in, averaged gradient out, copies timed ----
     e2e = None
@@ -359,6 +354,7 @@ def run_cuda(args) -> dict:
 
 
 def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> dict:
+    from paper_2107_14575_b200 import replicas
     Ke = min(K, 10)
     host = [pool[p].cpu().pin_memory() for p in range(2)]
     for i in range(2):
@@ -374,11 +370,8 @@ def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> d
     torch.cuda.synchronize()
     checksum = float(res[:1024].double().abs().sum())        # the result is read on the host
     ms2 = s2.elapsed_time(e2)
-    if world > 1:
-        tmax = torch.tensor([ms2], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms2 = float(tmax.item())
-    return {"value": world * 4.0 * M * d * Ke / (ms2 * 1e-3) / 1e9, "unit": UNIT,
+    ms2 = replicas.max_over_ranks(ms2, dev)
+    return {"value": replicas.whole_job_rate(4.0 * M * d * Ke, world, ms2) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": 4 * M * D32, "d2h_bytes_per_step": 4 * D32, "steps": Ke,
             "ms_per_step": ms2 / Ke, "checksum": checksum}
 

@@ -1,0 +1,173 @@
+"""GPU parity at full workload sizes, in the launch configuration the benchmark times.
+
+The small cases of ``test_gpu_parity.py`` cover every code path element by element; the
+cases here show that nothing changes when the grids are full, the tile ranges long and
+the indices large:
+  * the benchmark workload (ResNet-18 shape, M = 8, bucket 512) through ``Round.step_fused``
+    (one pass norms+quantize+pack, average, bit rule on a second stream), every output
+    compared with the oracle, which finishes this size in seconds;
+  * the VGG-16 and text-classifier shapes (M = 16, buckets 2048 and 1024) the same way;
+  * the bandwidth-sweep sizes that the oracle cannot hold in host memory (d = 2^30 at M = 1,
+    d = 2^26 at M = 32): the oracle checks a prefix of every worker word for word (codes
+    depend only on an element's own bucket, worker, index and the step, so a prefix of the
+    layout is a smaller problem with the same answer), and properties that hold for every
+    element are checked over the whole array on the device: |Q(v) - v| <= norm/s,
+    padding of the staging buffers untouched, mean error within 5 sigma of zero.
+Tolerances are those stated in ``test_gpu_parity.py``.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2107_14575_b200 import dq, workloads as W
+from paper_2107_14575_b200.pipeline import Round
+
+pytestmark = pytest.mark.gpu
+
+NORM_RTOL = 1e-6
+AVG_RTOL = 1e-6
+SEED = 0x0DDB_A11_5EED
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib(dqlib):
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+
+
+def _calibrated_rule(w, norms, t, x0=6.0):
+    G2 = float((norms.astype(np.float64) ** 2).sum() / w.M)
+    eps_hat = w.T * w.alpha ** (w.T - 1) * G2 / x0 ** 2
+    return eps_hat, dq.Rule.dynamic(w.T, t, eps_hat, w.alpha)
+
+
+def _full_round(w, b0, steps=2):
+    """``steps`` rounds of Round.step_fused on workload ``w``; every output of every round against the oracle."""
+    ref = oracle.Layout(w.segments, w.bucket)
+    rnd = Round(w.segments, w.bucket, w.M)
+    rnd.packed.fill_(-1)
+    rnd.bits_(dq.Rule.fixed(b0))
+    b = b0
+    eps_hat = None
+    for t in range(steps):
+        g = W.make_grads(w, ref.offsets, ref.D32, step=t, pad_value=float("nan"))
+        gd = torch.from_numpy(g).cuda()
+        want_norms = oracle.bucket_norms(ref, g)
+        if eps_hat is None:
+            eps_hat, _ = _calibrated_rule(w, want_norms, 0)
+        rule_next = dq.Rule.dynamic(w.T, t + 1, eps_hat, w.alpha)
+        out = rnd.step_fused(gd, rule_next, SEED, t).cpu().numpy()
+        torch.cuda.synchronize()
+        assert rnd.read_status() == 0
+        norms = rnd.norms.cpu().numpy()
+        packed = rnd.packed.cpu().numpy().view(np.uint32)
+        nw = ref.packed_words(b)
+
+        np.testing.assert_allclose(norms, want_norms, rtol=NORM_RTOL, atol=0)
+        # words: bit-exact against the oracle driven with the norms the kernel wrote
+        want_packed = oracle.quantize_pack(ref, g, norms, b, SEED, t)
+        assert np.array_equal(packed[:, :nw], want_packed)
+        if t == 0:
+            assert np.all(packed[:, nw:] == 0xFFFFFFFF)      # nothing written past the words in use
+        # average
+        want_out = oracle.unpack_dequant_average(ref, want_packed, norms, b)
+        err = np.linalg.norm(out.astype(np.float64) - want_out) / max(np.linalg.norm(want_out), 1e-300)
+        assert err <= AVG_RTOL, err
+        # next b: the rule on the same norms
+        b_next, s_next, _ = oracle.choose_bits(norms, w.T, t + 1, eps_hat, w.alpha)
+        assert rnd.bits() == b_next
+        b = b_next
+    return b
+
+
+def test_bench_workload_full_size_two_rounds():
+    w = W.config_resnet18()
+    assert w.M == 8 and w.bucket == 512 and sum(w.segments) == 11173962
+    _full_round(w, b0=4, steps=2)
+
+
+@pytest.mark.parametrize("b0", [7, 16])
+def test_bench_workload_full_size_other_widths(b0):
+    _full_round(W.config_resnet18(), b0=b0, steps=1)
+
+
+def test_vgg16_full_size():
+    w = W.config_vgg16()
+    assert w.M == 16 and w.bucket == 2048
+    _full_round(w, b0=4, steps=1)
+
+
+def test_text_classifier_full_size():
+    w = W.config_text()
+    assert w.M == 16 and w.bucket == 1024
+    _full_round(w, b0=5, steps=1)
+
+
+def _device_normal(M, d, seed):
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(seed)
+    g = torch.empty((M, d), dtype=torch.float32, device="cuda")
+    for m in range(M):
+        g[m].normal_(0.0, 1.0, generator=gen)
+    return g
+
+
+@pytest.mark.parametrize("d,M,bucket,b,prefix", [
+    (1 << 30, 1, 512, 4, 1 << 22),
+    (1 << 30, 1, 4096, 16, 1 << 22),
+    (1 << 28, 1, 128, 1, 1 << 22),
+    (1 << 26, 32, 512, 3, 1 << 20),
+    (1 << 26, 32, 128, 8, 1 << 20),
+])
+def test_sweep_sizes_prefix_parity_and_whole_array_properties(d, M, bucket, b, prefix):
+    s = (1 << (b - 1)) - 1
+    rnd = Round([d], bucket, M, max_bits=b)
+    L = rnd.layout
+    g = _device_normal(M, d, seed=d % 1000 + M)
+    rnd.packed.fill_(-1)
+    rnd.bits_(dq.Rule.fixed(b))
+    rnd.norms_quantize_(g, SEED, 3)
+    torch.cuda.synchronize()
+    assert rnd.read_status() == 0
+
+    # ---- prefix of every worker, word for word
+    ref = oracle.Layout([prefix], bucket)
+    gp = g[:, :prefix].cpu().numpy()
+    want_norms = oracle.bucket_norms(ref, gp)
+    norms_p = rnd.norms[:, : ref.nb].cpu().numpy()
+    np.testing.assert_allclose(norms_p, want_norms, rtol=NORM_RTOL, atol=0)
+    want_packed = oracle.quantize_pack(ref, gp, norms_p, b, SEED, 3)
+    got = rnd.packed[:, : ref.packed_words(b)].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, want_packed)
+    # nothing written past the words in use
+    nw = L.packed_words(b)
+    if rnd.packed_stride > nw:
+        assert bool((rnd.packed[:, nw:] == -1).all())
+
+    # ---- the separate norms kernel gives the same norms at this size
+    fused_norms = rnd.norms.clone()
+    rnd.norms_(g)
+    assert torch.equal(rnd.norms, fused_norms)
+
+    # ---- whole array, M = 1 only (the average of one worker is Q(v) itself)
+    if M == 1:
+        rnd.average_()
+        torch.cuda.synchronize()
+        assert rnd.read_status() == 0
+        q = rnd.out[:d]
+        if b == 1:
+            assert bool((q == 0).all())
+            return
+        step = (rnd.norms[0] / s).repeat_interleave(bucket)[:d]          # one level of each element's bucket
+        err = (q - g[0]).abs()
+        # one level, plus the fp32 rounding of position and product (|x| <= s, so 4 ulp of s levels covers it)
+        assert bool((err <= step * (1.0 + 4.0 * s * 2.0 ** -23)).all())
+        # unbiased: the mean error in units of a level is within 5 sigma of 0 (sigma <= 1/2 per element)
+        mean_err = float(((q - g[0]) / step).double().mean())
+        assert abs(mean_err) <= 5 * 0.5 / np.sqrt(d)
+        # the average's prefix against the oracle as well
+        want_out = oracle.unpack_dequant_average(ref, want_packed, norms_p, b)
+        got_out = rnd.out[:prefix].cpu().numpy()
+        rel = np.linalg.norm(got_out - want_out) / np.linalg.norm(want_out)
+        assert rel <= AVG_RTOL
