@@ -246,8 +246,9 @@ def run_cuda(args) -> dict:
     #     then choose b_{t+1} from this step's norms.  This is the timed headline.
     #  "four_call": norms, bit rule on this step's own norms, quantize (second pass), average.
     def run_order(order, sampler=None):
-        if order == "algorithm1":
-            names = ["norms_quantize_pack", "unpack_dequant_average", "choose_bits"]
+        if order in ("algorithm1", "algorithm1_update"):
+            names = ["norms_quantize_pack", "unpack_dequant_average" if order == "algorithm1" else "unpack_average_update",
+                     "choose_bits"]
             bits = [b_of(0, 0)] + [b_of(i - 1, i) for i in range(1, K)]          # untimed: b of every step
         else:
             names = ["bucket_norms", "choose_bits", "quantize_pack", "unpack_dequant_average"]
@@ -257,6 +258,9 @@ def run_cuda(args) -> dict:
             g = pool[i % npool]
             if order == "algorithm1":
                 rnd.step_fused(g, rule_for(i + 1), SEED, i, overlap=not args.no_overlap, events=e)
+            elif order == "algorithm1_update":
+                rnd.step_fused(g, rule_for(i + 1), SEED, i, overlap=not args.no_overlap, events=e, params=params,
+                               lr=1e-3)
             else:
                 e[0].record(); rnd.norms_(g)
                 e[1].record(); rnd.bits_(rule_for(i))
@@ -290,7 +294,7 @@ def run_cuda(args) -> dict:
         t_ms = replicas.max_over_ranks(t_ms, dev)
         # algorithm1: events 0-1 bracket the fused call, 1-2 the average, 3-4 the bit rule (on its own
         # stream when it overlaps the average); four_call: 0-1-2-3-4 in sequence
-        spans = [(0, 1), (1, 2), (3, 4)] if order == "algorithm1" else [(0, 1), (1, 2), (2, 3), (3, 4)]
+        spans = [(0, 1), (1, 2), (3, 4)] if order != "four_call" else [(0, 1), (1, 2), (2, 3), (3, 4)]
         totals = {n: sum(ev[i][p].elapsed_time(ev[i][q]) for i in range(K)) for n, (p, q) in zip(names, spans)}
         mean_b = sum(bits) / len(bits)
         alg_bytes = {
@@ -299,6 +303,7 @@ def run_cuda(args) -> dict:
             "quantize_pack": (4.0 + mean_b / 8.0) * elems,
             "norms_quantize_pack": (4.0 + mean_b / 8.0) * elems,
             "unpack_dequant_average": (M * mean_b / 8.0 + 4.0) * D32,
+            "unpack_average_update": (M * mean_b / 8.0 + 8.0) * D32,
         }
         kernels = {}
         for n in names:
@@ -320,6 +325,13 @@ def run_cuda(args) -> dict:
         "algorithmic_bytes_per_launch": kernels[dominant]["algorithmic_bytes_per_launch"], "mean_b": round(mean_b, 3),
         "kernels": kernels,
     }
+    upd = None
+    if not args.no_four_call:
+        # the same order with the parameter update of Eq. 2 folded into the server step
+        params = torch.zeros(D32, dtype=torch.float32, device=dev)
+        msu, _, mean_bu, kernelsu, _, _ = run_order("algorithm1_update")
+        upd = {"ms_per_step": msu / K, "value": replicas.whole_job_rate(4.0 * M * w.d * K, world, msu) / 1e9,
+               "mean_bits": round(mean_bu, 3), "kernels": kernelsu}
     four = None
     if not args.no_four_call:
         ms4, bits4, mean_b4, kernels4, _, _ = run_order("four_call")
@@ -342,7 +354,7 @@ def run_cuda(args) -> dict:
                    "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "roofline": roofline,
-        "four_call_order": four,
+        "four_call_order": four, "with_parameter_update": upd,
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

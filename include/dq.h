@@ -226,6 +226,23 @@ int dq_unpack_dequant_average(const dq_layout_t* layout, const uint32_t* dev_pac
                               int64_t packed_stride_words, const float* dev_norms, int32_t M,
                               const int32_t* dev_b, float* dev_out, int32_t* dev_status, void* stream);
 
+/* ------------- Algorithm 1, server side: "Average" and the parameter update
+ * x <- x - eta * g_hat, with g_hat the average dq_unpack_dequant_average computes
+ * (the step "x_{t+1} = x_t - eta * g_hat_t" that follows the averaging in
+ * Algorithm 1; the prose around Eq. 17 prints "+ eta", the listing and Eq. 2
+ * "- eta": descent is meant).  The averaged gradient is formed in registers and
+ * never written: per element M*b/8 + 4 bytes are read and 4 written.
+ *   dev_params[j] <- fmaf(-lr, g_hat[j], dev_params[j])   (one fp32 rounding)
+ * Padding elements of dev_params keep their value (their g_hat is 0), and so does
+ * everything when s = 0 (b = 1).
+ * in : dev_packed, dev_norms [M][nb], dev_b, lr (finite, else DQ_ERR_RANGE)
+ * io : dev_params fp32 [D32], 16-byte aligned, caller-owned, in the padded layout
+ * Device conditions: as dq_unpack_dequant_average. */
+int dq_unpack_average_update(const dq_layout_t* layout, const uint32_t* dev_packed,
+                             int64_t packed_stride_words, const float* dev_norms, int32_t M,
+                             const int32_t* dev_b, float lr, float* dev_params,
+                             int32_t* dev_status, void* stream);
+
 /* Text for a DQ_ERR_* return value (static storage). */
 const char* dq_status_string(int code);
 

@@ -78,6 +78,9 @@ def lib():
             L.oracle_unpack_dequant_average.restype = None
             L.oracle_unpack_dequant_average.argtypes = ([_u32p, C.c_int64, _f32p, C.c_int32, C.c_int32]
                                                         + seg + [_f32p])
+            L.oracle_unpack_average_update.restype = None
+            L.oracle_unpack_average_update.argtypes = ([_u32p, C.c_int64, _f32p, C.c_int32, C.c_int32]
+                                                       + seg + [C.c_double, _f32p])
             L.oracle_set_threads.restype = None
             L.oracle_set_threads.argtypes = [C.c_int32]
             L.oracle_get_threads.restype = C.c_int32
@@ -223,4 +226,17 @@ def unpack_dequant_average(lay: Layout, packed: np.ndarray, norms: np.ndarray, b
     assert norms.shape == (M, lay.nb) and packed.shape[1] >= lay.packed_words(b)
     out = np.zeros(lay.D32, np.float32)
     lib().oracle_unpack_dequant_average(packed, packed.shape[1], norms, M, b, *lay._args(), out)
+    return out
+
+
+def unpack_average_update(lay: Layout, packed: np.ndarray, norms: np.ndarray, b: int, eta: float,
+                          x: np.ndarray) -> np.ndarray:
+    """x - eta * average (Eq. 2); returns a new fp32 array [D32], padding copied from ``x``."""
+    packed = np.ascontiguousarray(packed, np.uint32)
+    norms = np.ascontiguousarray(norms, np.float32)
+    M = packed.shape[0]
+    assert norms.shape == (M, lay.nb) and packed.shape[1] >= lay.packed_words(b)
+    out = np.array(x, dtype=np.float32, copy=True)
+    assert out.shape == (lay.D32,)
+    lib().oracle_unpack_average_update(packed, packed.shape[1], norms, M, b, *lay._args(), float(eta), out)
     return out

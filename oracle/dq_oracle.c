@@ -314,3 +314,35 @@ void oracle_unpack_dequant_average(const uint32_t* packed, int64_t packed_stride
     free(codes);
     free_table(&tb);
 }
+
+/* Eq. 2 / Algorithm 1 "Update the global parameters": x <- x - eta * g_hat, with g_hat the
+ * average above, all in fp64 and rounded to fp32 once.  Padding elements keep their value. */
+void oracle_unpack_average_update(const uint32_t* packed, int64_t packed_stride,
+                                  const float* norms, int32_t M, int32_t b,
+                                  const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                                  double eta, float* x)
+{
+    table_t tb = make_table(seg_elems, n_seg, bucket);
+    const int64_t D32 = oracle_padded_elems(seg_elems, n_seg);
+    const int32_t s = (1 << (b - 1)) - 1;
+    uint32_t* codes = (uint32_t*)malloc(sizeof(uint32_t) * (size_t)((int64_t)M * D32 + 1));
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int32_t m = 0; m < M; ++m)
+        oracle_unpack(packed + (int64_t)m * packed_stride, D32, b, codes + (int64_t)m * D32);
+
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int64_t k = 0; k < tb.nb; ++k) {
+        for (int64_t e = 0; e < tb.len[k]; ++e) {
+            const int64_t j = tb.start[k] + e;
+            double acc = 0.0;
+            for (int32_t m = 0; m < M; ++m) {
+                const double q = (double)codes[(int64_t)m * D32 + j] - (double)s;     /* sgn * level */
+                if (s > 0) acc += q * (double)norms[(int64_t)m * tb.nb + k] / (double)s;
+            }
+            const double g_hat = acc / (double)M;
+            x[j] = (float)((double)x[j] - eta * g_hat);
+        }
+    }
+    free(codes);
+    free_table(&tb);
+}

@@ -19,6 +19,8 @@
  *                     the single number s + sgn * level in 0 .. 2s
  *   pack / unpack     b-bit codes concatenated LSB-first into 32-bit words
  *   unpack_dequant_average   Algorithm 1, server step "Average", with Eq. 5
+ *   unpack_average_update    the same followed by the parameter update of Eq. 2
+ *                     (Algorithm 1, "Update the global parameters")
  *   philox4x32_10     Salmon, Moraes, Dror, Shaw, "Parallel random numbers:
  *                     as easy as 1, 2, 3" (SC'11), Philox-4x32 with 10 rounds
  *
@@ -92,6 +94,12 @@ void oracle_unpack_dequant_average(const uint32_t* packed, int64_t packed_stride
                                    const float* norms /*[M][nb]*/, int32_t M, int32_t b,
                                    const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
                                    float* out /*[D32]*/);
+
+/* ---- Eq. 2: x <- x - eta * average, fp64 arithmetic, one rounding to fp32; pads untouched ---- */
+void oracle_unpack_average_update(const uint32_t* packed, int64_t packed_stride,
+                                  const float* norms /*[M][nb]*/, int32_t M, int32_t b,
+                                  const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                                  double eta, float* x /*[D32], in and out*/);
 
 /* number of OpenMP threads the loops over workers/buckets may use (default 1) */
 void    oracle_set_threads(int32_t n);

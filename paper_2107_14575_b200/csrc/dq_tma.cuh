@@ -94,6 +94,16 @@ __device__ __forceinline__ void load_tile_3d(void* dst, const CUtensorMap* map, 
         : "memory");
 }
 
+// 2-D tiled tensor copy global -> shared (rows outside the tensor arrive as zeros and still
+// count towards the barrier's bytes), completion counted on `bar`.
+__device__ __forceinline__ void load_tile_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(smem_addr(dst)), "l"(map), "r"(smem_addr(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+
 // L2 policy for data that is read once and should be the first to leave the cache.
 __device__ __forceinline__ uint64_t policy_evict_first()
 {

@@ -13,6 +13,12 @@
 // worker.  The 128 x 32 results of a tile go through a swizzled shared-memory
 // tile and leave with one bulk tensor store.
 // HBM traffic per output element: M*b/8 bytes read, 4 written.
+//
+// dq_unpack_average_update is the same kernel with the parameter update of
+// Algorithm 1 as its epilogue, x <- x - eta * average: the tile of x is fetched into
+// the output tile by a bulk tensor load while the codes are decoded, updated in place
+// and stored back; the averaged gradient itself never reaches memory (M*b/8 + 4 bytes
+// read and 4 written per element).
 #include "dq_common.cuh"
 #include "dq_device.cuh"
 #include "dq_tma.cuh"
@@ -33,10 +39,11 @@ extern __shared__ __align__(1024) unsigned char smem[];
 constexpr int kOutBytes = kThreads * 128;
 constexpr int kStageOffset = kOutBytes;
 constexpr int kScaleOffset = kStageOffset + kStages * kStageWords * 4;            // [kMaxChunk][kThreads] floats
-constexpr int kBarOffset = kScaleOffset + kMaxChunk * kThreads * 4;
-constexpr int kTblOffset = kBarOffset + kStages * 8;
+constexpr int kBarOffset = kScaleOffset + kMaxChunk * kThreads * 4;     // kStages stage barriers, then the one of the x tile
+constexpr int kTblOffset = kBarOffset + (kStages + 1) * 8;
 
 __device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
+__device__ __forceinline__ uint64_t* x_bar() { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + kStages; }
 __device__ __forceinline__ uint32_t* stage_words(int st) { return reinterpret_cast<uint32_t*>(smem + kStageOffset) + st * kStageWords; }
 
 struct AverageArgs {
@@ -51,6 +58,7 @@ struct AverageArgs {
     uint32_t div_magic;
     int32_t div_shift;
     uint32_t magic;               // 0x4B000000, kept out of the compiler's sight (see and_or)
+    float neg_lr;                 // -eta of the parameter update (update kernel only)
 };
 
 __device__ __forceinline__ uint32_t div_gpb(const AverageArgs& a, uint32_t n)
@@ -144,7 +152,8 @@ __device__ __forceinline__ void issue_unit(const AverageArgs& a, int st, int row
                        a.packed + (int64_t)(m0 + j) * a.packed_stride + (int64_t)row0 * B, bytes, full_bar(st));
 }
 
-template <int B>
+// UPDATE = false: out = average.  UPDATE = true: out holds the parameters x and becomes x - eta * average.
+template <int B, bool UPDATE>
 __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtensorMap* out_map, const bool tbl_in_smem)
 {
     constexpr int s = (1 << (B - 1)) - 1;
@@ -207,21 +216,23 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
     };
 
     if constexpr (B == 1) {
-        // s = 0: every value is 0
-        for (int tile = tile_begin; tile < tile_end; ++tile) {
-            if (tid == 0) tma::store_wait_read();
-            __syncthreads();
+        // s = 0: every value is 0, and an update by 0 leaves x as it is
+        if constexpr (!UPDATE) {
+            for (int tile = tile_begin; tile < tile_end; ++tile) {
+                if (tid == 0) tma::store_wait_read();
+                __syncthreads();
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) = make_float4(0.f, 0.f, 0.f, 0.f);
-            tma::fence_proxy_async();
-            __syncthreads();
-            if (tid == 0) {
-                tma::store_tile_2d(out_map, smem, 0, tile * kThreads);
-                tma::store_commit();
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) = make_float4(0.f, 0.f, 0.f, 0.f);
+                tma::fence_proxy_async();
+                __syncthreads();
+                if (tid == 0) {
+                    tma::store_tile_2d(out_map, smem, 0, tile * kThreads);
+                    tma::store_commit();
+                }
             }
+            if (tid == 0) tma::store_wait_read();
         }
-        if (tid == 0) tma::store_wait_read();
         return;
     } else {
         // Software pipeline over the units: while unit u is decoded, the scales of unit u + 1
@@ -244,6 +255,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         float acc[32];
         bool timed_out = false;
         int u = 0;
+        int tiles_done = 0;
         for (int tile = tile_begin; tile < tile_end && !timed_out; ++tile) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
@@ -270,6 +282,15 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                         nxt[j] = (has_next && j < nmc && nvalid > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) * unit : 0.0f;
                 }
 
+                if constexpr (UPDATE) {
+                    // the tile of x travels into the output tile while the codes are decoded; the
+                    // previous tile's store must have drained it first
+                    if (c == 0 && tid == 0) {
+                        tma::store_wait_read();
+                        tma::mbar_expect_tx(x_bar(), kOutBytes);
+                        tma::load_tile_2d(smem, out_map, x_bar(), 0, tile * kThreads);
+                    }
+                }
                 const int st = u % kStages;
                 if (!tma::mbar_wait(full_bar(st), (u / kStages) & 1)) { timed_out = true; break; }
                 const uint32_t* base = stage_words(st) + tid * B;
@@ -284,7 +305,9 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                 for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j];
 
                 // the previous tile's bulk store must have drained the output tile before it is rewritten below
-                if (last_chunk && tid == 0) tma::store_wait_read();
+                if constexpr (!UPDATE) {
+                    if (last_chunk && tid == 0) tma::store_wait_read();
+                }
                 __syncthreads();                  // the stage is free again
                 if (tid == 0) {
                     const int nu = u + kStages;
@@ -304,10 +327,22 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                     if (e >= valid) acc[e] = 0.0f;
             }
             // own row of the swizzled output tile (conflict-free), then one bulk tensor store per tile
+            if constexpr (UPDATE) {
+                if (!tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u)) { timed_out = true; break; }
+                const float neg_lr = a.neg_lr;
 #pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) =
-                    make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+                for (int c = 0; c < 8; ++c) {
+                    float4* p = reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c));
+                    const float4 x = *p;
+                    *p = make_float4(fmaf(neg_lr, acc[4 * c], x.x), fmaf(neg_lr, acc[4 * c + 1], x.y),
+                                     fmaf(neg_lr, acc[4 * c + 2], x.z), fmaf(neg_lr, acc[4 * c + 3], x.w));
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c)
+                    *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) =
+                        make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
+            }
             tma::fence_proxy_async();
             __syncthreads();
             if (tid == 0) {
@@ -316,17 +351,21 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
             }
             bucket = nbucket;
             valid = nvalid;
+            ++tiles_done;
         }
 
         if (tid == 0) tma::store_wait_read();         // shared memory must outlive the last store's reads
         if (timed_out) {
             if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
+            // give copies still in flight a bounded chance to land before the shared memory is released
             for (int k = 1; k < kStages; ++k)
                 if (u + k < my_units) (void)tma::mbar_wait(full_bar((u + k) % kStages), ((u + k) / kStages) & 1);
+            if constexpr (UPDATE) (void)tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u);
         }
     }
 }
 
+template <bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 4)
 unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_constant__ CUtensorMap out_map)
 {
@@ -352,12 +391,13 @@ unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_consta
         tma::prefetch_tensor_map(&out_map);
 #pragma unroll
         for (int st = 0; st < kStages; ++st) tma::mbar_init(full_bar(st), 1);
+        tma::mbar_init(x_bar(), 1);
         tma::fence_barrier_init();
     }
     __syncthreads();
 
     switch (b) {
-#define DQ_CASE(BB) case BB: average_tiles<BB>(a, &out_map, tbl_in_smem); break;
+#define DQ_CASE(BB) case BB: average_tiles<BB, UPDATE>(a, &out_map, tbl_in_smem); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -372,11 +412,11 @@ size_t smem_bytes(int n_seg)
     return n;
 }
 
-}  // namespace
-
-extern "C" int dq_unpack_dequant_average(const dq_layout_t* L, const uint32_t* dev_packed,
-                                         int64_t packed_stride_words, const float* dev_norms, int32_t M,
-                                         const int32_t* dev_b, float* dev_out, int32_t* dev_status, void* stream)
+// Checks, tensor map and launch shared by the two entry points; `dev_out` is the averaged
+// gradient (update = false) or the parameters, read and written (update = true).
+template <bool UPDATE>
+int launch_average(const dq_layout_t* L, const uint32_t* dev_packed, int64_t packed_stride_words, const float* dev_norms,
+                   int32_t M, const int32_t* dev_b, float lr, float* dev_out, int32_t* dev_status, void* stream)
 {
     const int rc = dq_check_common(L, M);
     if (rc != DQ_OK) return rc;
@@ -386,6 +426,7 @@ extern "C" int dq_unpack_dequant_average(const dq_layout_t* L, const uint32_t* d
         (reinterpret_cast<uintptr_t>(dev_status) & 3u))
         return DQ_ERR_ALIGN;
     if (packed_stride_words < L->padded / 32) return DQ_ERR_RANGE;
+    if (UPDATE && !(lr == lr && lr - lr == 0.0f)) return DQ_ERR_RANGE;      // eta must be finite
 
     AverageArgs a;
     a.v = make_view(L);
@@ -397,6 +438,7 @@ extern "C" int dq_unpack_dequant_average(const dq_layout_t* L, const uint32_t* d
     a.status = dev_status;
     a.M = M;
     a.magic = 0x4B000000u;
+    a.neg_lr = -lr;
     const uint32_t gpb = (uint32_t)a.v.groups_per_bucket;
     if ((gpb & (gpb - 1)) == 0) {
         a.div_shift = 0;
@@ -417,14 +459,33 @@ extern "C" int dq_unpack_dequant_average(const dq_layout_t* L, const uint32_t* d
         return DQ_ERR_CUDA;
 
     const size_t smem_need = smem_bytes(L->n_seg);
-    if (cudaFuncSetAttribute(unpack_average_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
+    if (cudaFuncSetAttribute(unpack_average_kernel<UPDATE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
         (void)cudaGetLastError();
         return DQ_ERR_CUDA;
     }
     const int64_t tiles = ((int64_t)a.v.total_groups + kThreads - 1) / kThreads;
     int64_t blocks = (int64_t)dq_sm_count() * 4;       // four 53 KB CTAs per SM
     if (blocks > tiles) blocks = tiles;
-    unpack_average_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, out_map);
+    unpack_average_kernel<UPDATE><<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, out_map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+}  // namespace
+
+extern "C" int dq_unpack_dequant_average(const dq_layout_t* L, const uint32_t* dev_packed,
+                                         int64_t packed_stride_words, const float* dev_norms, int32_t M,
+                                         const int32_t* dev_b, float* dev_out, int32_t* dev_status, void* stream)
+{
+    return launch_average<false>(L, dev_packed, packed_stride_words, dev_norms, M, dev_b, 0.0f, dev_out, dev_status,
+                                 stream);
+}
+
+extern "C" int dq_unpack_average_update(const dq_layout_t* L, const uint32_t* dev_packed,
+                                        int64_t packed_stride_words, const float* dev_norms, int32_t M,
+                                        const int32_t* dev_b, float lr, float* dev_params, int32_t* dev_status,
+                                        void* stream)
+{
+    return launch_average<true>(L, dev_packed, packed_stride_words, dev_norms, M, dev_b, lr, dev_params, dev_status,
+                                stream);
 }

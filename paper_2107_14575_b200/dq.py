@@ -24,7 +24,8 @@ SYMBOLS = [
     "dq_layout_table_bytes", "dq_layout_bind_device_table",
     "dq_bucket_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
     "dq_choose_bits_noalloc_max_norms", "dq_choose_bits_noalloc",
-    "dq_quantize_pack", "dq_norms_quantize_pack", "dq_unpack_dequant_average", "dq_status_string",
+    "dq_quantize_pack", "dq_norms_quantize_pack", "dq_unpack_dequant_average",
+    "dq_unpack_average_update", "dq_status_string",
 ]
 
 
@@ -97,6 +98,8 @@ def lib():
         L.dq_norms_quantize_pack.argtypes = [vp, vp, i64, i32, vp, u64, u32, vp, vp, i64, vp, vp]
         L.dq_unpack_dequant_average.restype = C.c_int
         L.dq_unpack_dequant_average.argtypes = [vp, vp, i64, vp, i32, vp, vp, vp, vp]
+        L.dq_unpack_average_update.restype = C.c_int
+        L.dq_unpack_average_update.argtypes = [vp, vp, i64, vp, i32, vp, C.c_float, vp, vp, vp]
         L.dq_status_string.restype = C.c_char_p
         L.dq_status_string.argtypes = [C.c_int]
         _lib = L
@@ -225,3 +228,11 @@ def unpack_dequant_average(layout: Layout, packed, packed_stride_words: int, nor
     _check(lib().dq_unpack_dequant_average(layout.handle, _ptr(packed), int(packed_stride_words), _ptr(norms),
                                            int(M), _ptr(dev_b), _ptr(out), _ptr(status), _stream(stream)),
            "dq_unpack_dequant_average")
+
+
+def unpack_average_update(layout: Layout, packed, packed_stride_words: int, norms, M: int, dev_b, lr: float, params,
+                          status, stream=None) -> None:
+    """``params <- params - lr * average`` (Eq. 2), the average formed on the fly."""
+    _check(lib().dq_unpack_average_update(layout.handle, _ptr(packed), int(packed_stride_words), _ptr(norms),
+                                          int(M), _ptr(dev_b), float(lr), _ptr(params), _ptr(status),
+                                          _stream(stream)), "dq_unpack_average_update")

@@ -67,6 +67,11 @@ class Round:
         dq.unpack_dequant_average(self.layout, self.packed, self.packed_stride, self.norms, self.M, self.dev_b,
                                   self.out, self.status)
 
+    def update_(self, params, lr: float) -> None:
+        """``params <- params - lr * average`` (Eq. 2) from the packed codes; the average itself is not stored."""
+        dq.unpack_average_update(self.layout, self.packed, self.packed_stride, self.norms, self.M, self.dev_b, lr,
+                                 params, self.status)
+
     def step(self, grads, rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
         """Whole round on device gradients; returns the averaged gradient [D32] (device)."""
         self.norms_(grads)
@@ -76,7 +81,7 @@ class Round:
         return self.out
 
     def step_fused(self, grads, next_rule: dq.Rule, seed: int, step: int, overlap: bool = True,
-                   events=None) -> torch.Tensor:
+                   events=None, params=None, lr: float = 0.0) -> torch.Tensor:
         """One round in the order of Algorithm 1: quantize with the b chosen after the
         previous round (one pass over the gradients), average, and choose the next b from
         this round's norms.  ``dev_b`` must hold a b (a first call to ``bits_`` with the
@@ -86,7 +91,17 @@ class Round:
         only the norms, and writes the other (b, s) slot.  The current stream waits for it
         before it goes on.  ``events`` = (e0, e1, e2, s0, s1) are recorded around the three
         calls (e* on the current stream, s* around the bit rule on its own stream).
+
+        With ``params`` (fp32 [D32] in the padded layout) the server step also applies the
+        update of Eq. 2, ``params <- params - lr * average``, in the same kernel; ``out`` is
+        then not written and ``params`` is returned.
         """
+        def server_step():
+            if params is None:
+                self.average_()
+            else:
+                self.update_(params, lr)
+        result = self.out if params is None else params
         main = torch.cuda.current_stream(self.device)
         if events:
             events[0].record(main)
@@ -94,14 +109,14 @@ class Round:
         if events:
             events[1].record(main)
         if not overlap:
-            self.average_()
+            server_step()
             if events:
                 events[2].record(main)
                 events[3].record(main)
             self.bits_(next_rule)
             if events:
                 events[4].record(main)
-            return self.out
+            return result
         if self._side is None:
             self._side = torch.cuda.Stream(self.device)
             self._ev_norms = torch.cuda.Event()
@@ -115,12 +130,12 @@ class Round:
         if events:
             events[4].record(self._side)
         self._ev_bits.record(self._side)
-        self.average_()                      # reads the current slot
+        server_step()                        # reads the current slot
         if events:
             events[2].record(main)
         main.wait_event(self._ev_bits)
         self._cur = 1 - self._cur
-        return self.out
+        return result
 
     def step_host(self, host_grads: torch.Tensor, next_rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
         """``step_fused`` on pinned host gradients [M, stride]; returns a pinned host tensor [D32].

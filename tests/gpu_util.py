@@ -91,6 +91,14 @@ class GpuRound:
                                   self.g_b.view, self.g_out.view, self.status)
         return self.g_out.view.cpu().numpy()
 
+    def update(self, lr: float, x: np.ndarray) -> np.ndarray:
+        """Average and parameter update in one call; the parameters live in the guarded output buffer."""
+        assert x.shape == (self.lay.D32,) and x.dtype == np.float32
+        self.g_out.view.copy_(torch.from_numpy(x))
+        dq.unpack_average_update(self.lay, self.g_packed.view, self.pstride, self.g_norms.view, self.M,
+                                 self.g_b.view, lr, self.g_out.view, self.status)
+        return self.g_out.view.cpu().numpy()
+
     def read_status(self) -> int:
         return int(self.status.item())
 

@@ -171,3 +171,25 @@ def test_sweep_sizes_prefix_parity_and_whole_array_properties(d, M, bucket, b, p
         got_out = rnd.out[:prefix].cpu().numpy()
         rel = np.linalg.norm(got_out - want_out) / np.linalg.norm(want_out)
         assert rel <= AVG_RTOL
+
+
+def test_bench_workload_full_size_with_parameter_update():
+    """Round.step_fused with the update of Eq. 2 in the server step, full bench workload."""
+    w = W.config_resnet18()
+    ref = oracle.Layout(w.segments, w.bucket)
+    rnd = Round(w.segments, w.bucket, w.M)
+    b, lr = 5, 0.1
+    rnd.bits_(dq.Rule.fixed(b))
+    g = W.make_grads(w, ref.offsets, ref.D32, step=0)
+    x = np.random.default_rng(1).normal(size=ref.D32).astype(np.float32) * 1e-2
+    xd = torch.from_numpy(x).cuda()
+    got = rnd.step_fused(torch.from_numpy(g).cuda(), dq.Rule.fixed(b), SEED, 0, params=xd, lr=lr)
+    torch.cuda.synchronize()
+    assert rnd.read_status() == 0 and got is xd
+    norms = rnd.norms.cpu().numpy()
+    packed = rnd.packed.cpu().numpy().view(np.uint32)[:, : ref.packed_words(b)]
+    assert np.array_equal(packed, oracle.quantize_pack(ref, g, norms, b, SEED, 0))
+    want = oracle.unpack_average_update(ref, packed, norms, b, lr, x)
+    avg = oracle.unpack_dequant_average(ref, packed, norms, b)
+    tol = 1e-6 * lr * np.abs(avg).max() + 2.0 ** -23 * np.abs(want) + 1e-30
+    assert np.all(np.abs(got.cpu().numpy().astype(np.float64) - want) <= tol)

@@ -373,6 +373,90 @@ def test_on_level_workers_average_exactly(G):
     assert np.array_equal(r.average(), row[0])
 
 
+# ------------------------------------------- average + parameter update (Eq. 2)
+
+def _update_tolerance(lr, avg, want):
+    # the fp32 average is within 1e-6 of the fp64 one (relative to the bucket's scale, bounded here by
+    # the largest entry), and the result is rounded to fp32 once on each side
+    return 1e-6 * abs(lr) * np.abs(avg).max() + 2.0 ** -23 * np.abs(want) + 1e-30
+
+
+@pytest.mark.parametrize("b", [1, 2, 3, 4, 5, 8, 11, 16])
+@pytest.mark.parametrize("M", [1, 4, 32])
+def test_average_update_matches_oracle(G, M, b):
+    w = W.config_flat(d=9000 + 13, M=M, bucket=128, sigma=0.5, seed=M)
+    ref, g = _make(w)
+    norms = oracle.bucket_norms(ref, g)
+    packed = oracle.quantize_pack(ref, g, norms, b, SEED, 1)
+    r = G.GpuRound(w.segments, w.bucket, M, packed_stride=(ref.packed_words(b) + 3) // 4 * 4 + 8)
+    full = np.full((M, r.pstride), 0xA5A5A5A5, np.uint32)
+    full[:, : ref.packed_words(b)] = packed
+    r.set_packed(full)
+    r.set_norms(norms)
+    r.set_b(b)
+    rng = np.random.default_rng(b * 100 + M)
+    x = rng.normal(size=ref.D32).astype(np.float32)
+    x[9013:] = 123.0                                               # padding of the parameters
+    lr = 0.37
+    got = r.update(lr, x)
+    want = oracle.unpack_average_update(ref, packed, norms, b, lr, x)
+    avg = oracle.unpack_dequant_average(ref, packed, norms, b)
+    assert np.all(np.abs(got.astype(np.float64) - want) <= _update_tolerance(lr, avg, want))
+    assert np.array_equal(got[9013:], x[9013:])                    # padding keeps its value
+    if b == 1:
+        assert np.array_equal(got, x)
+    else:
+        assert not np.array_equal(got[:9013], x[:9013])
+    assert r.read_status() == 0 and r.guards_intact()
+
+
+@pytest.mark.parametrize("name,M,b", [("ragged-b96", 4, 3), ("resnet/64", 8, 5), ("vgg/256", 16, 7),
+                                       ("text/128", 16, 4), ("flat-b4096", 2, 12)])
+def test_average_update_multi_tensor(G, name, M, b):
+    w = CASES[name]
+    w = W.Workload(**{**w.__dict__})
+    w.M = M
+    ref, g = _make(w)
+    norms = oracle.bucket_norms(ref, g)
+    packed = oracle.quantize_pack(ref, g, norms, b, 77, 0)
+    r = G.GpuRound(w.segments, w.bucket, M)
+    full = np.zeros((M, r.pstride), np.uint32)
+    full[:, : ref.packed_words(b)] = packed
+    r.set_packed(full)
+    r.set_norms(norms)
+    r.set_b(b)
+    x = np.random.default_rng(5).normal(size=ref.D32).astype(np.float32) * 0.01
+    lr = -0.05                                                     # ascent is allowed: eta is just a number
+    got = r.update(lr, x)
+    want = oracle.unpack_average_update(ref, packed, norms, b, lr, x)
+    avg = oracle.unpack_dequant_average(ref, packed, norms, b)
+    assert np.all(np.abs(got.astype(np.float64) - want) <= _update_tolerance(lr, avg, want))
+    # the same average as the plain call: x - lr * out, rounded once
+    out = r.average()
+    assert np.array_equal(got, (x.astype(np.float64) - np.float64(np.float32(lr)) * out).astype(np.float32))
+    assert r.read_status() == 0 and r.guards_intact()
+
+
+def test_update_on_level_workers_is_exact_and_rejects_bad_eta(G):
+    b = 4
+    row = np.zeros((1, 64), np.float32)
+    row[0, :3] = [2 * 0.25, -3 * 0.25, 6 * 0.25]
+    row[0, 32:35] = [-6.0, 2.0, 3.0]
+    g = np.ascontiguousarray(np.broadcast_to(row, (8, 64)))
+    r = G.GpuRound([64], 32, 8)
+    r.set_grads(g)
+    r.norms()
+    r.set_b(b)
+    r.quantize(5, 5)
+    x = np.arange(64, dtype=np.float32) * 0.125 - 3.0
+    assert np.array_equal(r.update(0.5, x), x - np.float32(0.5) * row[0])
+    from paper_2107_14575_b200 import dq
+    for bad in (float("nan"), float("inf")):
+        with pytest.raises(dq.DQError) as e:
+            r.update(bad, x)
+        assert e.value.code == dq.ERR_RANGE
+
+
 # ------------------------------------------------------- whole step, device b
 
 @pytest.mark.parametrize("name", ["resnet/64", "vgg/256", "text/128"])
