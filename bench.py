@@ -245,6 +245,8 @@ def run_cuda(args) -> dict:
     #     previous step's norms, in ONE pass together with the norms (dq_norms_quantize_pack), average,
     #     then choose b_{t+1} from this step's norms.  This is the timed headline.
     #  "four_call": norms, bit rule on this step's own norms, quantize (second pass), average.
+    host_ms = {}
+
     def run_order(order, sampler=None):
         if order in ("algorithm1", "algorithm1_update"):
             names = ["norms_quantize_pack", "unpack_dequant_average" if order == "algorithm1" else "unpack_average_update",
@@ -284,9 +286,11 @@ def run_cuda(args) -> dict:
         if sampler:
             sampler.start()
         start.record()
+        h0 = time.perf_counter()
         for i in range(K):
             one_step(i, ev[i])
         end.record()
+        host_ms[order] = (time.perf_counter() - h0) * 1e3 / K      # host time to submit one step
         torch.cuda.synchronize()
         clk = sampler.stop() if sampler else None
         t_ms = start.elapsed_time(end)
@@ -355,6 +359,7 @@ def run_cuda(args) -> dict:
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "roofline": roofline,
         "four_call_order": four, "with_parameter_update": upd,
+        "host_submit_ms_per_step": round(host_ms["algorithm1"], 5),
     }
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

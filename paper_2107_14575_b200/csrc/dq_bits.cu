@@ -15,9 +15,12 @@
 
 namespace {
 
-constexpr int kThreads = 256;       // threads of the second kernel
+// Both kernels are small on purpose (128 threads, well under 100 registers): in the order of
+// Algorithm 1 they run on a second stream beside the average, whose persistent CTAs leave
+// about a fifth of an SM's registers free, and CTAs of this size fit into that room.
+constexpr int kThreads = 128;       // threads of the second kernel
 constexpr int kChunk = 8192;        // norms per CTA of the first kernel
-constexpr int kSumThreads = 512;    // threads of the first kernel: 16 norms each, all loads in flight at once
+constexpr int kSumThreads = 128;    // threads of the first kernel: 64 norms each, all loads in flight at once
 
 // Sum over the CTA in a fixed order: shuffle tree inside each warp, then the warp sums
 // added in warp order by thread 0.  Returns the total in thread 0.
@@ -36,23 +39,27 @@ __device__ __forceinline__ double block_sum(double v, double* sh)
     return total;
 }
 
-__global__ void __launch_bounds__(kSumThreads)
+__global__ void __launch_bounds__(kSumThreads, 8)
 norm_square_partials(const float* __restrict__ norms, const int64_t n, double* __restrict__ partial)
 {
     __shared__ double sh[kSumThreads / 32];
-    constexpr int kPer = kChunk / kSumThreads;
+    constexpr int kPer = kChunk / kSumThreads;     // 64 norms per thread, fetched 32 at a time
+    constexpr int kBatch = 32;
     const int64_t base = (int64_t)blockIdx.x * kChunk + threadIdx.x;
-    float x[kPer];
-#pragma unroll
-    for (int i = 0; i < kPer; ++i) {
-        const int64_t j = base + (int64_t)i * kSumThreads;
-        x[i] = (j < n) ? __ldg(norms + j) : 0.0f;
-    }
     double a0 = 0.0, a1 = 0.0;
 #pragma unroll
-    for (int i = 0; i < kPer; i += 2) {
-        a0 = fma((double)x[i], (double)x[i], a0);
-        a1 = fma((double)x[i + 1], (double)x[i + 1], a1);
+    for (int h = 0; h < kPer / kBatch; ++h) {
+        float x[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) {
+            const int64_t j = base + (int64_t)(h * kBatch + i) * kSumThreads;
+            x[i] = (j < n) ? __ldg(norms + j) : 0.0f;
+        }
+#pragma unroll
+        for (int i = 0; i < kBatch; i += 2) {
+            a0 = fma((double)x[i], (double)x[i], a0);
+            a1 = fma((double)x[i + 1], (double)x[i + 1], a1);
+        }
     }
     const double s = block_sum<kSumThreads>(a0 + a1, sh);
     if (threadIdx.x == 0) partial[blockIdx.x] = s;
