@@ -88,6 +88,25 @@ __device__ __forceinline__ uint32_t encode(const float g, const float inv, const
     return __float_as_uint(t);
 }
 
+// inv = RZ(s / norm), the scale of Eq. 5 rounded toward zero (0 for norm < 2^-100, where the
+// quotient could overflow, and for a NaN norm).  Written out instead of calling the library's
+// division so that it stays inline: reciprocal estimate r (relative error <= 2^-23), q = s * r,
+// one Newton step q <- q + (s - q * norm) * r, which brings q to within 2^-44 of the quotient
+// before its rounding, i.e. to one of the two floats that enclose s / norm; the sign of the
+// exactly rounded residual s - q * norm then tells which, and the upper one steps down an ulp.
+// Norms above 2^125, whose reciprocal estimate would be flushed to zero, take the library route.
+__device__ __forceinline__ float inv_scale(const float sf, const float norm)
+{
+    if (!(norm >= 0x1p-100f)) return 0.0f;
+    if (norm > 0x1p125f) return __fdiv_rz(sf, norm);
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(norm));
+    float q = __fmul_rn(sf, r);
+    q = __fmaf_rn(__fmaf_rn(-q, norm, sf), r, q);
+    const float e = __fmaf_rn(-q, norm, sf);
+    return __uint_as_float(__float_as_uint(q) - (e < 0.0f ? 1u : 0u));
+}
+
 // Appends code number E of a group to the group's little-endian bit string.
 // `cur` is a shift register: a funnel shift pushes the B code bits in at the
 // top, so after 32 bits the first code sits at bit 0 and the word is complete.

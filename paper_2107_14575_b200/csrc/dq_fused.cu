@@ -208,7 +208,7 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
         // ---- codes of this thread's group against that norm
         const int off = (int)(((int64_t)row0 * B) & 3);      // staging keeps the stream's 16-byte phase
         if (valid > 0) {
-            const float inv = (nrm >= 0x1p-100f) ? __fdiv_rz(sf, nrm) : 0.0f;
+            const float inv = inv_scale(sf, nrm);
             unsigned char* rowp = base + row * 128;
             const uint32_t sw = (uint32_t)(row & 7);
             if (valid < 32) {                    // padding after a tensor's end encodes as 0
@@ -341,7 +341,7 @@ __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* ba
     // codes of this lane's group against that norm
     uint32_t acc[B];
     if (valid > 0) {
-        const float inv = (nrm >= 0x1p-100f) ? __fdiv_rz(sf, nrm) : 0.0f;
+        const float inv = inv_scale(sf, nrm);
         unsigned char* rowp = base + row * 128;
         const uint32_t sw = (uint32_t)(row & 7);
         if (valid < 32) {                        // padding after a tensor's end encodes as 0
@@ -492,7 +492,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 bad |= !isfinite(nrm);
             }
             // ---- codes of this lane's group against that norm
-            const float inv = (nrm >= 0x1p-100f) ? __fdiv_rz(sf, nrm) : 0.0f;
+            const float inv = inv_scale(sf, nrm);
             uint32_t acc[B];
             if constexpr (B == 1) {
                 acc[0] = 0u;

@@ -138,7 +138,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
             valid = left < 32 ? left : 32;
         }
         const float norm = active ? __ldg(a.norms + (int64_t)m * a.v.nb + bucket) : 0.0f;
-        const float inv = (norm >= 0x1p-100f) ? __fdiv_rz(sf, norm) : 0.0f;
+        const float inv = inv_scale(sf, norm);
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
         // warp-level synchronisations below are always reached by all lanes or by none

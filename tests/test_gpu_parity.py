@@ -313,6 +313,41 @@ def test_choose_bits_many_norms_and_zero(G):
     assert r.read_status() & G.dq.STAT_NONFINITE
 
 
+@pytest.mark.parametrize("b", [2, 5, 9, 16])
+def test_scale_division_is_exact_over_the_norm_range(G, b):
+    """inv = RZ(s / norm) decides every code; one bucket of 32 elements per norm, norms over the whole
+    exponent range, quotients that are exact, and the bounds of the kernel's inline division."""
+    s = (1 << (b - 1)) - 1
+    nbk = 1 << 15
+    rng = np.random.default_rng(b)
+    mant = (1.0 + rng.random(nbk)).astype(np.float32)
+    expo = rng.integers(-95, 120, size=nbk)
+    norms = np.ldexp(mant, expo).astype(np.float32)
+    special = []
+    for k in (-60, -7, 0, 3, 40):
+        special += [np.ldexp(1.0, k), np.ldexp(float(s), k)]                 # quotient a power of two
+        special += [np.ldexp(float(s) / m, k) for m in (1, 3, 7, 31, 151) if s % m == 0]   # exact quotients
+        special += [np.ldexp(3.0, k), np.ldexp(1.0 - 2.0 ** -24, k), np.ldexp(1.0 + 2.0 ** -23, k)]
+    special += [2.0 ** -100, np.nextafter(np.float32(2.0 ** -100), np.float32(0)), 2.0 ** -120, 0.0,
+                2.0 ** 125, np.nextafter(np.float32(2.0 ** 125), np.float32(np.inf)), 2.0 ** 126, 3.0e38]
+    norms[: len(special)] = np.array(special, np.float32)
+    u = rng.random((nbk, 32)).astype(np.float32)
+    u[:, 0] = 1.0                                                              # an entry as large as the norm
+    u[:, 1] = np.float32(1.0 - 2.0 ** -24)
+    sign = np.where(rng.random((nbk, 32)) < 0.5, -1.0, 1.0).astype(np.float32)
+    g = (norms[:, None] * u * sign).astype(np.float32).reshape(1, -1)
+    assert np.all(np.abs(g.reshape(nbk, 32)) <= norms[:, None])
+    ref = oracle.Layout([nbk * 32], 32)
+    r = G.GpuRound([nbk * 32], 32, 1)
+    r.set_grads(g)
+    r.set_norms(norms.reshape(1, -1))
+    r.set_b(b)
+    got = r.quantize(SEED, 7, fill=0)
+    want = oracle.quantize_pack(ref, g, norms.reshape(1, -1), b, SEED, 7)
+    assert np.array_equal(got[:, : ref.packed_words(b)], want)
+    assert r.read_status() == 0 and r.guards_intact()
+
+
 # ------------------------------------------------- unpack + dequantize + average
 
 @pytest.mark.parametrize("b", list(range(1, 17)))
