@@ -585,15 +585,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
 __global__ void __launch_bounds__(kThreads, 6)
 norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
-    const int b = __ldg(a.dev_b);
-    if (b < 1 || b > DQ_MAX_BITS) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
-        return;
-    }
-    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
-        return;
-    }
+    const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
         return;
@@ -608,6 +600,14 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
         tma::fence_barrier_init();
     }
     __syncthreads();
+    if (b < 1 || b > DQ_MAX_BITS) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
+        return;
+    }
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
+        return;
+    }
 
     switch (b) {
 #define DQ_CASE(BB) case BB: fused_warp_tiles<BB>(a, &map); break;
@@ -622,15 +622,7 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
 __global__ void __launch_bounds__(kThreads, 5)
 norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
-    const int b = __ldg(a.dev_b);
-    if (b < 1 || b > DQ_MAX_BITS) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
-        return;
-    }
-    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
-        return;
-    }
+    const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
         return;
@@ -646,6 +638,14 @@ norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_con
         tma::fence_barrier_init();
     }
     __syncthreads();
+    if (b < 1 || b > DQ_MAX_BITS) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
+        return;
+    }
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
+        return;
+    }
 
     switch (b) {
 #define DQ_CASE(BB) case BB: fused_tiles<BB>(a, &map); break;

@@ -202,15 +202,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
 __global__ void __launch_bounds__(kThreads, 6)
 quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_constant__ CUtensorMap map)
 {
-    const int b = __ldg(a.dev_b);
-    if (b < 1 || b > DQ_MAX_BITS) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
-        return;
-    }
-    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
-        return;
-    }
+    const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {           // the swizzled tiles need a 1024-byte aligned base
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
         return;
@@ -226,6 +218,14 @@ quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_consta
         tma::fence_barrier_init();
     }
     __syncthreads();
+    if (b < 1 || b > DQ_MAX_BITS) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
+        return;
+    }
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
+        return;
+    }
 
     switch (b) {
 #define DQ_CASE(BB) case BB: quantize_tiles<BB>(a, &map, tbl_in_smem); break;

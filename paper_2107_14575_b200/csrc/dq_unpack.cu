@@ -369,15 +369,7 @@ template <bool UPDATE>
 __global__ void __launch_bounds__(kThreads, 4)
 unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_constant__ CUtensorMap out_map)
 {
-    const int b = __ldg(a.dev_b);
-    if (b < 1 || b > DQ_MAX_BITS) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
-        return;
-    }
-    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
-        return;
-    }
+    const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {           // the swizzled tile needs a 1024-byte aligned base
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
         return;
@@ -395,6 +387,14 @@ unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_consta
         tma::fence_barrier_init();
     }
     __syncthreads();
+    if (b < 1 || b > DQ_MAX_BITS) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
+        return;
+    }
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
+        return;
+    }
 
     switch (b) {
 #define DQ_CASE(BB) case BB: average_tiles<BB, UPDATE>(a, &out_map, tbl_in_smem); break;
