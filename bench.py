@@ -264,11 +264,12 @@ def run_cuda(args) -> dict:
                 rnd.step_fused(g, rule_for(i + 1), SEED, i, overlap=not args.no_overlap, events=e, params=params,
                                lr=1e-3)
             else:
-                e[0].record(); rnd.norms_(g)
-                e[1].record(); rnd.bits_(rule_for(i))
-                e[2].record(); rnd.quantize_(g, SEED, i)
-                e[3].record(); rnd.average_()
-                e[4].record()
+                rec = (lambda j: e[j].record()) if e else (lambda j: None)
+                rec(0); rnd.norms_(g)
+                rec(1); rnd.bits_(rule_for(i))
+                rec(2); rnd.quantize_(g, SEED, i)
+                rec(3); rnd.average_()
+                rec(4)
 
         nev = 5
         b_of(0, 0)                                  # dev_b holds b_0 before the first step
@@ -278,7 +279,10 @@ def run_cuda(args) -> dict:
         b_of(0, 0)
         torch.cuda.synchronize()
         assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(K)]
+        # Per-call events cost about 3 us of device time each (the stream drains around them), so only
+        # every `ev_stride`-th timed step carries them; the others run as a user's steps do.
+        ev_stride = max(1, K // 12)
+        ev = {i: [torch.cuda.Event(enable_timing=True) for _ in range(nev)] for i in range(0, K, ev_stride)}
         start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if world > 1:
             dist.barrier()
@@ -288,7 +292,7 @@ def run_cuda(args) -> dict:
         start.record()
         h0 = time.perf_counter()
         for i in range(K):
-            one_step(i, ev[i])
+            one_step(i, ev.get(i))
         end.record()
         host_ms[order] = (time.perf_counter() - h0) * 1e3 / K      # host time to submit one step
         torch.cuda.synchronize()
@@ -299,19 +303,21 @@ def run_cuda(args) -> dict:
         # algorithm1: events 0-1 bracket the fused call, 1-2 the average, 3-4 the bit rule (on its own
         # stream when it overlaps the average); four_call: 0-1-2-3-4 in sequence
         spans = [(0, 1), (1, 2), (3, 4)] if order != "four_call" else [(0, 1), (1, 2), (2, 3), (3, 4)]
-        totals = {n: sum(ev[i][p].elapsed_time(ev[i][q]) for i in range(K)) for n, (p, q) in zip(names, spans)}
+        totals = {n: sum(e[p].elapsed_time(e[q]) for e in ev.values()) for n, (p, q) in zip(names, spans)}
+        nsamp = len(ev)
         mean_b = sum(bits) / len(bits)
+        mean_bs = sum(bits[i] for i in ev) / nsamp                 # of the steps that carried events
         alg_bytes = {
             "bucket_norms": 4.0 * elems,
             "choose_bits": 4.0 * M * L.nb,
-            "quantize_pack": (4.0 + mean_b / 8.0) * elems,
-            "norms_quantize_pack": (4.0 + mean_b / 8.0) * elems,
-            "unpack_dequant_average": (M * mean_b / 8.0 + 4.0) * D32,
-            "unpack_average_update": (M * mean_b / 8.0 + 8.0) * D32,
+            "quantize_pack": (4.0 + mean_bs / 8.0) * elems,
+            "norms_quantize_pack": (4.0 + mean_bs / 8.0) * elems,
+            "unpack_dequant_average": (M * mean_bs / 8.0 + 4.0) * D32,
+            "unpack_average_update": (M * mean_bs / 8.0 + 8.0) * D32,
         }
         kernels = {}
         for n in names:
-            avg_ms = totals[n] / K
+            avg_ms = totals[n] / nsamp
             gbs = alg_bytes[n] / (avg_ms * 1e-3) / 1e9
             kernels[n] = {"avg_ms": round(avg_ms, 5), "achieved_gbs": round(gbs, 1), "frac": round(gbs / peak, 4),
                           "share": round(totals[n] / sum(totals.values()), 4),
@@ -329,6 +335,26 @@ def run_cuda(args) -> dict:
         "algorithmic_bytes_per_launch": kernels[dominant]["algorithmic_bytes_per_launch"], "mean_b": round(mean_b, 3),
         "kernels": kernels,
     }
+    # The events that bracket a single launch also see its launch latency (the stream drains at
+    # every record).  For context, the same kernel launched back to back between two events:
+    if dominant == "norms_quantize_pack":
+        nb2b = 10
+        b_last = bits[-1]
+        rnd.bits_(dq.Rule.fixed(b_last))
+        for i in range(3):
+            rnd.norms_quantize_(pool[i % npool], SEED, i)
+        torch.cuda.synchronize()
+        s3, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s3.record()
+        for i in range(nb2b):
+            rnd.norms_quantize_(pool[i % npool], SEED, i)
+        e3.record()
+        torch.cuda.synchronize()
+        b2b_ms = s3.elapsed_time(e3) / nb2b
+        b2b_bytes = (4.0 + b_last / 8.0) * elems
+        roofline["back_to_back"] = {"launches": nb2b, "b": b_last, "avg_ms": round(b2b_ms, 5),
+                                    "achieved": round(b2b_bytes / (b2b_ms * 1e-3) / 1e9, 1),
+                                    "frac": round(b2b_bytes / (b2b_ms * 1e-3) / 1e9 / peak, 4)}
     upd = None
     if not args.no_four_call:
         # the same order with the parameter update of Eq. 2 folded into the server step
@@ -356,6 +382,8 @@ def run_cuda(args) -> dict:
                    "order": "Algorithm 1: norms+quantize+pack in one pass with b_t, average, b_{t+1} from this step's norms"
                             + ("" if args.no_overlap else " (bit rule on a second stream beside the average)"),
                    "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
+                   "kernel_events": "CUDA events around each call on every %d-th timed step (%d samples)"
+                                    % (max(1, K // 12), len(range(0, K, max(1, K // 12)))),
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "roofline": roofline,
         "four_call_order": four, "with_parameter_update": upd,
