@@ -2,13 +2,20 @@
  * dq.h -- C ABI of the DQ-SGD gradient quantizer hot path for NVIDIA B200 (sm_100a).
  *
  * Method: "DQ-SGD: Dynamic Quantization in SGD for Communication-Efficient
- * Distributed Learning" (arXiv 2107.14575).  One training step of Algorithm 1
- * maps to four calls, all asynchronous on the caller's CUDA stream:
+ * Distributed Learning" (arXiv 2107.14575).  The steps of one iteration of
+ * Algorithm 1, all asynchronous on the caller's CUDA stream:
  *
  *   dq_bucket_norms            ||g||_2 of Eq. 5, per bucket          (workers)
  *   dq_choose_bits             bit rule Eq. 17 -> b, s on the device (server)
  *   dq_quantize_pack           Q_b[g] of Eq. 5/6, b-bit codes packed (workers)
  *   dq_unpack_dequant_average  "Average" step of Algorithm 1         (server)
+ *
+ * and two calls that merge neighbouring steps:
+ *
+ *   dq_norms_quantize_pack     norms and quantizer in one pass over the gradients
+ *                              (b_t is known before step t: Algorithm 1 derives
+ *                              b_{t+1} from iteration t)
+ *   dq_unpack_average_update   the average followed by x <- x - eta * average (Eq. 2)
  *
  * M workers are M gradient buffers on one GPU: worker m's data is at
  * base + m * stride for every per-worker array.  There is no CPU fallback.

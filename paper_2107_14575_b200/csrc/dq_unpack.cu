@@ -7,6 +7,9 @@
 // registers).  The M workers' words of a tile are fetched in chunks of a few
 // workers by linear bulk copies (TMA) into a ring of shared-memory stages, so
 // the copies of the next chunks overlap the decoding of the current one.  A
+// fifth warp does nothing but issue those copies: a bulk copy holds its issuing
+// thread until the copy engine accepts it, about a microsecond per tile when the
+// SM's four CTAs queue there at once, and nobody waits for that warp.  A
 // code is decoded where it stands in its word (mask under the exponent of 2^23,
 // subtract 2^23 + s: see decode_code) and accumulated with one FMA; the power
 // of two its position carries is removed once per element after the last
@@ -25,7 +28,8 @@
 
 namespace {
 
-constexpr int kThreads = 128;                 // groups per tile
+constexpr int kThreads = 128;                 // groups per tile = consumer threads (warps 0..3)
+constexpr int kBlock = kThreads + 32;         // plus the warp that issues the copies
 constexpr int kStages = 2;
 constexpr int kStageWords = 4096;             // 16 KB per stage
 constexpr int kMaxChunk = 8;                  // workers per stage at most
@@ -39,11 +43,16 @@ extern __shared__ __align__(1024) unsigned char smem[];
 constexpr int kOutBytes = kThreads * 128;
 constexpr int kStageOffset = kOutBytes;
 constexpr int kScaleOffset = kStageOffset + kStages * kStageWords * 4;            // [kMaxChunk][kThreads] floats
-constexpr int kBarOffset = kScaleOffset + kMaxChunk * kThreads * 4;     // kStages stage barriers, then the one of the x tile
-constexpr int kTblOffset = kBarOffset + (kStages + 1) * 8;
+// barriers: kStages "stage filled" (copies landed), kStages "stage drained" (one arrival per
+// consumer warp), then the one of the x tile
+constexpr int kBarOffset = kScaleOffset + kMaxChunk * kThreads * 4;
+constexpr int kTblOffset = kBarOffset + (2 * kStages + 1) * 8;
 
 __device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
-__device__ __forceinline__ uint64_t* x_bar() { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + kStages; }
+__device__ __forceinline__ uint64_t* empty_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + kStages + st; }
+__device__ __forceinline__ uint64_t* x_bar() { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + 2 * kStages; }
+// barrier among the consumer warps only (the copy warp runs ahead on its own)
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
 __device__ __forceinline__ uint32_t* stage_words(int st) { return reinterpret_cast<uint32_t*>(smem + kStageOffset) + st * kStageWords; }
 
 struct AverageArgs {
@@ -175,12 +184,22 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
     const int tile_begin = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
     const int tile_end = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
     const int my_units = (B == 1) ? 0 : (tile_end - tile_begin) * nchunk;
-    if (tid == 0) {
-        for (int u = 0; u < kStages && u < my_units; ++u) {
-            const int tile = tile_begin + u / nchunk;
-            const int m0 = (u % nchunk) * MC;
-            issue_unit<B>(a, u, tile * kThreads, m0, (M - m0) < MC ? (M - m0) : MC);
+    if (tid >= kThreads) {
+        // the copy warp: unit u goes into stage u % kStages as soon as the consumers have drained
+        // what was there (unit u - kStages)
+        if (tid == kThreads) {
+            for (int u = 0; u < my_units; ++u) {
+                const int st = u % kStages;
+                if (u >= kStages && !tma::mbar_wait(empty_bar(st), (uint32_t)(u / kStages - 1) & 1u)) {
+                    atomicOr(a.status, DQ_STAT_WAIT);
+                    break;
+                }
+                const int tile = tile_begin + u / nchunk;
+                const int m0 = (u % nchunk) * MC;
+                issue_unit<B>(a, st, tile * kThreads, m0, (M - m0) < MC ? (M - m0) : MC);
+            }
         }
+        return;
     }
 
     // Bucket and valid elements of this thread's group in a tile.  The first lookup of a CTA
@@ -220,12 +239,12 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         if constexpr (!UPDATE) {
             for (int tile = tile_begin; tile < tile_end; ++tile) {
                 if (tid == 0) tma::store_wait_read();
-                __syncthreads();
+                consumer_sync();
 #pragma unroll
                 for (int c = 0; c < 8; ++c)
                     *reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c)) = make_float4(0.f, 0.f, 0.f, 0.f);
                 tma::fence_proxy_async();
-                __syncthreads();
+                consumer_sync();
                 if (tid == 0) {
                     tma::store_tile_2d(out_map, smem, 0, tile * kThreads);
                     tma::store_commit();
@@ -235,10 +254,11 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         }
         return;
     } else {
-        // Software pipeline over the units: while unit u is decoded, the scales of unit u + 1
-        // (norm * 1/(s M) per worker of the chunk, for this thread's bucket) are already on
-        // their way in registers; they replace the current ones in the scale buffer once the
-        // decode is done.
+        // Software pipeline over the units: while unit u is decoded, the norms of unit u + 1 (one
+        // per worker of the chunk, for this thread's bucket) are already on their way in registers.
+        // Nothing touches them before the decode is done -- the first use of a loaded value is
+        // where the warp would wait for it -- and only then do they become scales
+        // (norm * 1/(s M)) in the scale buffer.
         int bucket, valid, nbucket = 0, nvalid = 0;
         lookup(tile_begin, bucket, valid);
         float nxt[MC];
@@ -247,9 +267,9 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
             const float* nrm = a.norms + bucket;
 #pragma unroll
             for (int j = 0; j < MC; ++j)
-                nxt[j] = (j < mc0 && valid > 0 && my_units > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) * unit : 0.0f;
+                nxt[j] = (j < mc0 && valid > 0 && my_units > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) : 0.0f;
 #pragma unroll
-            for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j];
+            for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j] * unit;
         }
 
         float acc[32];
@@ -279,7 +299,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                     const float* nrm = a.norms + (int64_t)nm0 * a.v.nb + nbucket;
 #pragma unroll
                     for (int j = 0; j < MC; ++j)
-                        nxt[j] = (has_next && j < nmc && nvalid > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) * unit : 0.0f;
+                        nxt[j] = (has_next && j < nmc && nvalid > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) : 0.0f;
                 }
 
                 if constexpr (UPDATE) {
@@ -302,24 +322,18 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                     AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
                 }
 #pragma unroll
-                for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j];
+                for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j] * unit;
 
-                // the previous tile's bulk store must have drained the output tile before it is rewritten below
-                if constexpr (!UPDATE) {
-                    if (last_chunk && tid == 0) tma::store_wait_read();
-                }
-                __syncthreads();                  // the stage is free again
-                if (tid == 0) {
-                    const int nu = u + kStages;
-                    if (nu < my_units) {
-                        tma::fence_proxy_async();
-                        const int ntile = tile_begin + nu / nchunk;
-                        const int um0 = (nu % nchunk) * MC;
-                        issue_unit<B>(a, st, ntile * kThreads, um0, (M - um0) < MC ? (M - um0) : MC);
-                    }
-                }
+                // this warp is done with the stage: once all four have said so the copy warp refills it
+                __syncwarp();
+                if ((tid & 31) == 0) tma::mbar_arrive(empty_bar(st));
             }
             if (timed_out) break;
+            // the previous tile's bulk store must have drained the output tile before it is rewritten below
+            if constexpr (!UPDATE) {
+                if (tid == 0) tma::store_wait_read();
+            }
+            consumer_sync();
             Normalise<B, 0>::run(acc);
             if (valid < 32) {
 #pragma unroll
@@ -344,7 +358,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                         make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
             }
             tma::fence_proxy_async();
-            __syncthreads();
+            consumer_sync();
             if (tid == 0) {
                 tma::store_tile_2d(out_map, smem, 0, tile * kThreads);
                 tma::store_commit();
@@ -366,7 +380,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
 }
 
 template <bool UPDATE>
-__global__ void __launch_bounds__(kThreads, 4)
+__global__ void __launch_bounds__(kBlock, 4)
 unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_constant__ CUtensorMap out_map)
 {
     const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
@@ -377,12 +391,15 @@ unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_consta
     const bool tbl_in_smem = a.v.n_seg > 1 && a.v.n_seg <= kMaxSmemSegs;
     if (tbl_in_smem) {
         int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
-        for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
+        for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kBlock) tbl_s[i] = __ldg(a.v.seg_group0 + i);
     }
     if (threadIdx.x == 0) {
         tma::prefetch_tensor_map(&out_map);
 #pragma unroll
-        for (int st = 0; st < kStages; ++st) tma::mbar_init(full_bar(st), 1);
+        for (int st = 0; st < kStages; ++st) {
+            tma::mbar_init(full_bar(st), 1);
+            tma::mbar_init(empty_bar(st), kThreads / 32);
+        }
         tma::mbar_init(x_bar(), 1);
         tma::fence_barrier_init();
     }
@@ -466,7 +483,7 @@ int launch_average(const dq_layout_t* L, const uint32_t* dev_packed, int64_t pac
     const int64_t tiles = ((int64_t)a.v.total_groups + kThreads - 1) / kThreads;
     int64_t blocks = (int64_t)dq_sm_count() * 4;       // four 53 KB CTAs per SM
     if (blocks > tiles) blocks = tiles;
-    unpack_average_kernel<UPDATE><<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, out_map);
+    unpack_average_kernel<UPDATE><<<(unsigned)blocks, kBlock, smem_need, static_cast<cudaStream_t>(stream)>>>(a, out_map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
