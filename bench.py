@@ -315,13 +315,20 @@ def run_cuda(args) -> dict:
             "unpack_dequant_average": (M * mean_bs / 8.0 + 4.0) * D32,
             "unpack_average_update": (M * mean_bs / 8.0 + 8.0) * D32,
         }
+        # shares are of the time on the main stream; a bit rule that runs beside the average on the
+        # second stream is not on that path (its interval there includes waiting for room on the SMs)
+        beside = order != "four_call" and not args.no_overlap
+        on_path = [n for n in names if not (beside and n == "choose_bits")]
+        path_total = sum(totals[n] for n in on_path)
         kernels = {}
         for n in names:
             avg_ms = totals[n] / nsamp
             gbs = alg_bytes[n] / (avg_ms * 1e-3) / 1e9
             kernels[n] = {"avg_ms": round(avg_ms, 5), "achieved_gbs": round(gbs, 1), "frac": round(gbs / peak, 4),
-                          "share": round(totals[n] / sum(totals.values()), 4),
+                          "share": round(totals[n] / path_total, 4) if n in on_path else None,
                           "algorithmic_bytes_per_launch": alg_bytes[n]}
+            if n not in on_path:
+                kernels[n]["runs_beside"] = names[1]
         return t_ms, bits, mean_b, kernels, clk, len(names) + (1 if "choose_bits" in names else 0)
 
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", ""))
