@@ -4,8 +4,9 @@
 
 Sizes d = 2^20 ... 2^30 at M = 1 and d = 2^26 at M = 32, bit widths 1..16 at bucket 512
 and {2, 4, 8, 16} at buckets 128 and 4096.  Every kernel is timed alone with CUDA events
-(3 warm-up launches, median of 8-20), over rotating inputs that together exceed the L2.
-Each row gives the time, GB/s of algorithmic bytes (norms 4, quantizers 4 + b/8 per
+(3 warm-up launches, median of 8-20), over rotating inputs that together exceed the L2,
+and once more as a train of launches between two events (the sustained rate: launch latency
+overlaps the previous launch).  Each row gives both times, GB/s of algorithmic bytes (norms 4, quantizers 4 + b/8 per
 element and worker, average M b/8 + 4 per element) and GB/s of fp32 gradient (4 M d).
 Points below a few hundred microseconds are bound by the host's launch cost, not by the GPU.
 """
@@ -32,7 +33,14 @@ def _time(fn, reps):
         evs[i][1].record()
     torch.cuda.synchronize()
     ts = sorted(a.elapsed_time(b) for a, b in evs)
-    return ts[len(ts) // 2] * 1e3, ts[0] * 1e3
+    # sustained: the same launches back to back between two events
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(reps):
+        fn(i)
+    b.record()
+    torch.cuda.synchronize()
+    return ts[len(ts) // 2] * 1e3, ts[0] * 1e3, a.elapsed_time(b) * 1e3 / reps
 
 
 def run(quick: bool = False):
@@ -50,9 +58,10 @@ def run(quick: bool = False):
             gs = [torch.randn((M, D32), device="cuda") for _ in range(nbuf)]
             reps = 20 if d * M <= (1 << 28) else 8
 
-            def add(kernel, b, med, best, nbytes):
+            def add(kernel, b, med, best, train, nbytes):
                 rows.append({"kernel": kernel, "d": d, "M": M, "bucket": bucket, "b": b, "med_us": med, "best_us": best,
-                             "gbs": nbytes / med / 1e3, "grad_gbs": 4.0 * M * d / med / 1e3})
+                             "train_us": train, "gbs": nbytes / med / 1e3, "train_gbs": nbytes / train / 1e3,
+                             "grad_gbs": 4.0 * M * d / med / 1e3})
 
             add("bucket_norms", 0, *_time(lambda i: rnd.norms_(gs[i % nbuf]), reps), 4.0 * M * D32)
             for b in bits:
@@ -81,8 +90,9 @@ def main():
         with open(args.out, "w") as fh:
             json.dump(rows, fh)
     for r in rows:
-        sys.stdout.write("%-24s d=2^%-2d M=%-2d bucket=%-4d b=%-2d %9.1f us %7.0f GB/s  gradient %7.0f GB/s\n" % (
-            r["kernel"], r["d"].bit_length() - 1, r["M"], r["bucket"], r["b"], r["med_us"], r["gbs"], r["grad_gbs"]))
+        sys.stdout.write("%-24s d=2^%-2d M=%-2d bucket=%-4d b=%-2d %9.1f us %7.0f GB/s | in a train %9.1f us %7.0f GB/s | "
+                         "gradient %7.0f GB/s\n" % (r["kernel"], r["d"].bit_length() - 1, r["M"], r["bucket"], r["b"],
+                                                    r["med_us"], r["gbs"], r["train_us"], r["train_gbs"], r["grad_gbs"]))
 
 
 if __name__ == "__main__":
