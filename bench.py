@@ -2,8 +2,12 @@
 """Benchmark of the DQ-SGD quantizer hot path on B200.
 
 One step = one communication round of Algorithm 1 on one batch of synthetic
-gradients: bucket norms -> bit rule -> quantize+pack -> unpack+dequantize+average,
-all through the C-ABI library.  The workload is the ResNet-18-shaped gradient
+gradients, all through the C-ABI library: bucket norms and quantize+pack in one
+pass with the bit width chosen after the previous round, unpack+dequantize+average,
+and the bit rule for the next round beside the average.  The same steps as four
+separate calls (norms -> bit rule -> quantize+pack -> average) and with the
+parameter update folded into the average are timed as secondary figures.
+The workload is the ResNet-18-shaped gradient
 (62 tensors, 11,173,962 fp32 per worker, M = 8 workers, bucket 512, Laplace
 values, dynamic b over T = 100 steps, norms shrinking by 0.98 per step).
 
