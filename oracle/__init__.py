@@ -55,6 +55,8 @@ def lib():
             L.oracle_bucket_table.argtypes = seg + [_i64p, _i64p]
             L.oracle_bucket_norms.restype = None
             L.oracle_bucket_norms.argtypes = [C.c_void_p, C.c_int64, C.c_int32] + seg + [_f32p]
+            L.oracle_bucket_norms_p.restype = None
+            L.oracle_bucket_norms_p.argtypes = [C.c_void_p, C.c_int64, C.c_int32] + seg + [C.c_int32, _f32p]
             L.oracle_choose_bits.restype = C.c_int32
             L.oracle_choose_bits.argtypes = [_f32p, C.c_int64, C.c_int32, C.c_int32, C.c_int32,
                                              C.c_double, C.c_double, C.c_int32, C.c_int32, C.c_int32,
@@ -135,10 +137,23 @@ def _check_grads(lay: Layout, grads: np.ndarray):
     return grads.ctypes.data, grads.strides[0] // 4, grads.shape[0]
 
 
-def bucket_norms(lay: Layout, grads: np.ndarray) -> np.ndarray:
+NORM_L2, NORM_LINF = 2, 0
+
+
+def whole_tensor_bucket(seg_elems) -> int:
+    """Bucket size that gives every tensor a single bucket (the paper's own normalisation, Eq. 5)."""
+    return max(32, (int(max(seg_elems)) + 31) // 32 * 32)
+
+
+def bucket_norms(lay: Layout, grads: np.ndarray, p: int = NORM_L2) -> np.ndarray:
+    """Per-bucket norms; ``p`` = NORM_L2 (default) or NORM_LINF."""
+    assert p in (NORM_L2, NORM_LINF)
     ptr, stride, M = _check_grads(lay, grads)
     norms = np.zeros((M, lay.nb), np.float32)
-    lib().oracle_bucket_norms(ptr, stride, M, *lay._args(), norms)
+    if p == NORM_L2:
+        lib().oracle_bucket_norms(ptr, stride, M, *lay._args(), norms)
+    else:
+        lib().oracle_bucket_norms_p(ptr, stride, M, *lay._args(), p, norms)
     return norms
 
 

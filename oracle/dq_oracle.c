@@ -94,6 +94,33 @@ void oracle_bucket_norms(const float* grads, int64_t worker_stride, int32_t M,
     free_table(&tb);
 }
 
+/* The l_infinity member of the family ||g||_p of Eq. 5: the largest magnitude of the
+ * bucket (exact in fp32).  p_kind 2 is the l_2 norm above, p_kind 0 stands for p = infinity. */
+void oracle_bucket_norms_p(const float* grads, int64_t worker_stride, int32_t M,
+                           const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                           int32_t p_kind, float* norms)
+{
+    if (p_kind == 2) {
+        oracle_bucket_norms(grads, worker_stride, M, seg_elems, n_seg, bucket, norms);
+        return;
+    }
+    table_t tb = make_table(seg_elems, n_seg, bucket);
+    const int64_t total = (int64_t)M * tb.nb;
+#pragma omp parallel for schedule(static) num_threads(g_threads) if (g_threads > 1)
+    for (int64_t w = 0; w < total; ++w) {
+        const int64_t m = w / tb.nb, k = w % tb.nb;
+        const float* g = grads + m * worker_stride + tb.start[k];
+        float big = 0.0f;
+        for (int64_t j = 0; j < tb.len[k]; ++j) {
+            const float a = fabsf(g[j]);
+            if (a > big || a != a) big = a;          /* a NaN entry makes the norm NaN */
+            if (big != big) break;
+        }
+        norms[w] = big;
+    }
+    free_table(&tb);
+}
+
 /* ---------------------------------------------------------------- bit rule */
 
 int32_t oracle_choose_bits(const float* norms, int64_t nb, int32_t M,
@@ -196,7 +223,7 @@ void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
         /* s / norm and g * inv are both rounded toward zero: then |x| <= s for every
          * element with |g| <= norm (the norm of a bucket dominates its entries), so the
          * code stays in 0 .. 2s without a clamp, and inputs on a level stay exact. */
-        float xs[4096];                      /* a bucket has at most 4096 elements */
+        float* xs = (float*)malloc(sizeof(float) * (size_t)(tb.len[k] > 0 ? tb.len[k] : 1));
         fesetround(FE_TOWARDZERO);
         {
             const volatile float inv = (norm >= ORACLE_TINY_NORM) ? sf / norm : 0.0f;
@@ -218,6 +245,7 @@ void oracle_quantize(const float* grads, int64_t worker_stride, int32_t M,
             if (x_out) x_out[m * D32 + j] = x;
             if (v_out) v_out[m * D32 + j] = v;
         }
+        free(xs);
     }
     free_table(&tb);
 }

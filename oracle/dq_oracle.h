@@ -12,7 +12,8 @@
  *                     by the norm of the whole vector, Eq. 5; one bucket per
  *                     tensor reproduces that, smaller buckets apply the same
  *                     formula per bucket)
- *   bucket_norms      ||g||_2 of Eq. 5, per bucket
+ *   bucket_norms      ||g||_2 of Eq. 5, per bucket; bucket_norms_p also the l_infinity
+ *                     member of the paper's l_p family (Eq. 5 leaves p open)
  *   choose_bits       Eq. 17 with G-bar of Lemma 1, integer b by ceiling
  *   quantize          Eq. 5 and Eq. 6 (stochastic map zeta), s = 2^(b-1)-1; the b-bit
  *                     code of Sec. IV-A (a sign and b-1 bits of zeta) is stored as
@@ -31,7 +32,8 @@
  * Layout convention: tensor i with n_i elements starts at padded offset
  * P_i = sum_{j<i} roundup32(n_j); the worker buffer holds D32 = sum roundup32(n_i)
  * floats; buckets of `bucket` elements never cross a tensor, the last bucket
- * of a tensor may be short.  `bucket` is a multiple of 32.
+ * of a tensor may be short.  `bucket` is a multiple of 32; a bucket at least as
+ * large as every tensor is the paper's own case (one norm per vector).
  */
 #ifndef DQ_ORACLE_H
 #define DQ_ORACLE_H
@@ -54,6 +56,12 @@ void    oracle_bucket_table(const int64_t* seg_elems, int32_t n_seg, int32_t buc
 void oracle_bucket_norms(const float* grads, int64_t worker_stride, int32_t M,
                          const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
                          float* norms /*[M][nb]*/);
+
+/* ---- Eq. 5 with another member of the l_p family: p_kind = 2 is the call above,
+ *      p_kind = 0 stands for p = infinity (largest magnitude of the bucket, exact) ---- */
+void oracle_bucket_norms_p(const float* grads, int64_t worker_stride, int32_t M,
+                           const int64_t* seg_elems, int32_t n_seg, int32_t bucket,
+                           int32_t p_kind, float* norms /*[M][nb]*/);
 
 /* ---- Eq. 17: bit rule.  Returns b; writes s and the real-valued x with
  *      b* = log2(x + 1) + 1.  fixed_b != 0 bypasses the rule. ---- */
