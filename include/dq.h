@@ -75,6 +75,12 @@ extern "C" {
 #define DQ_MAX_BUCKET   4096
 #define DQ_MAX_WORKERS  4096
 
+/* ---- members of the quantizer family of Eq. 5 ("||g||_p is the l_p norm") ---- */
+#define DQ_NORM_L2      2   /* p = 2, the default                                      */
+#define DQ_NORM_LINF    0   /* p = infinity: the largest magnitude of the bucket        */
+#define DQ_BUCKET_WHOLE_TENSOR 0  /* bucket argument: one norm per tensor, as Eq. 5 is written */
+#define DQ_MAX_TENSOR_ELEMS (1 << 30)  /* largest tensor of a whole-tensor layout       */
+
 typedef struct dq_layout dq_layout_t;   /* host object, immutable after create */
 
 /* Parameters of the bit rule, Eq. 17:
@@ -99,6 +105,18 @@ typedef struct dq_rule {
  * 32..DQ_MAX_BUCKET.  The padded total must stay below 2^31 elements.
  * Errors: DQ_ERR_ARG (NULL, n_seg < 1), DQ_ERR_RANGE. */
 int     dq_layout_create(const int64_t* seg_elems, int32_t n_seg, int32_t bucket, dq_layout_t** out);
+/* The same with the member of the family of Eq. 5 chosen: `norm` is DQ_NORM_L2 or
+ * DQ_NORM_LINF (what dq_bucket_norms, dq_tensor_norms and dq_norms_quantize_pack compute
+ * for this layout; the quantizer and the average take whatever norms they are given).
+ * bucket = DQ_BUCKET_WHOLE_TENSOR gives every non-empty tensor a single bucket, which is
+ * Eq. 5 as the paper writes it (the vector is normalised by its own norm); tensors may
+ * then have up to DQ_MAX_TENSOR_ELEMS elements, and the norms come from dq_tensor_norms.
+ * dq_layout_create(.., bucket, ..) is dq_layout_create_ex(.., bucket, DQ_NORM_L2, ..).
+ * Errors: as dq_layout_create; DQ_ERR_ARG for an unknown norm. */
+int     dq_layout_create_ex(const int64_t* seg_elems, int32_t n_seg, int32_t bucket, int32_t norm,
+                            dq_layout_t** out);
+int32_t dq_layout_norm(const dq_layout_t* layout);          /* DQ_NORM_L2 / DQ_NORM_LINF          */
+int32_t dq_layout_whole_tensor(const dq_layout_t* layout);  /* 1 for a whole-tensor layout, else 0 */
 void    dq_layout_destroy(dq_layout_t* layout);
 int32_t dq_layout_num_segments(const dq_layout_t* layout);
 int64_t dq_layout_padded_elems(const dq_layout_t* layout);            /* D32                     */
@@ -120,7 +138,9 @@ int     dq_layout_bind_device_table(dq_layout_t* layout, void* dev_buf, size_t b
 
 /* ------------------------------------------------------------- norms, Eq. 5
  * dev_norms[m*nb + k] = sqrt( sum of squares of the valid elements of bucket k
- * of worker m ), the l_2 member of the paper's ||g||_p applied per bucket.
+ * of worker m ), the l_2 member of the paper's ||g||_p applied per bucket; for a
+ * layout created with DQ_NORM_LINF, the largest magnitude among those elements
+ * (exact; a NaN element makes the norm NaN).
  * in : dev_grads  fp32, worker m at dev_grads + m*worker_stride_elems,
  *                 each holding D32 elements in the padded layout
  * out: dev_norms  fp32 [M][nb]
@@ -129,6 +149,23 @@ int     dq_layout_bind_device_table(dq_layout_t* layout, void* dev_buf, size_t b
  * 1e-6 relative of an fp64 evaluation. */
 int dq_bucket_norms(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
                     int32_t M, float* dev_norms, int32_t* dev_status, void* stream);
+
+/* ------------------------------------------- one norm per tensor, Eq. 5 as written
+ * For layouts created with bucket = DQ_BUCKET_WHOLE_TENSOR: dev_norms[m*nb + k] is the
+ * norm (l_2 or l_inf, as the layout says) of the k-th non-empty tensor of worker m, nb the
+ * number of non-empty tensors.  Two kernels: partial results of 4096-element pieces into
+ * dev_scratch, then one reduction per (worker, tensor) in a fixed order (fp64 for the sums
+ * of squares), so results are deterministic and the l_2 norms within 1e-6 relative of an
+ * fp64 evaluation; l_inf norms are exact.  dq_bucket_norms and dq_norms_quantize_pack
+ * return DQ_ERR_RANGE for such layouts (a tensor's codes need the norm of the whole
+ * tensor, so the gradients are read twice); dq_quantize_pack, dq_choose_bits and the
+ * average calls work on them as on any other layout.
+ * dev_scratch: dq_tensor_norms_scratch_bytes() bytes, 16-byte aligned, used only during
+ * the call's kernels.  Sets DQ_STAT_NONFINITE if a norm is not finite. */
+size_t dq_tensor_norms_scratch_bytes(const dq_layout_t* layout, int32_t M);
+int dq_tensor_norms(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
+                    int32_t M, float* dev_norms, void* dev_scratch, size_t scratch_bytes,
+                    int32_t* dev_status, void* stream);
 
 /* --------------------------------------------------------- bit rule, Eq. 17
  * G-bar^2 = (1/M) sum_m sum_k dev_norms[m][k]^2 (Lemma 1; for p = 2 the sum of

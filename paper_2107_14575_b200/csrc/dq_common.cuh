@@ -23,8 +23,13 @@ struct dq_layout {
     //   [0]            first 32-element group of tensor i (last entry: D32/32)
     //   [n_seg+1]      first bucket of tensor i           (last entry: nb)
     //   [2(n_seg+1)]   valid elements of tensor i         (last entry: 0)
+    // A whole-tensor layout appends a second image of the same shape whose middle array counts
+    // 4096-element pieces instead of buckets (the pieces dq_tensor_norms reduces first).
     std::vector<int32_t> table;
     const int32_t* dev_table = nullptr; // caller-owned copy, set by bind
+    int32_t norm = DQ_NORM_L2;          // member of the l_p family the norm calls compute
+    bool whole_tensor = false;          // one bucket per non-empty tensor
+    int64_t n_pieces = 0;               // whole-tensor layouts: 4096-element pieces per worker
 };
 
 // What a kernel needs to map 32-element groups and buckets to tensors.
@@ -50,6 +55,23 @@ inline LayoutView make_view(const dq_layout* L)
     v.seg_group0 = L->dev_table;
     v.seg_bucket0 = L->dev_table ? L->dev_table + (L->n_seg + 1) : nullptr;
     v.seg_elems = L->dev_table ? L->dev_table + 2 * (L->n_seg + 1) : nullptr;
+    return v;
+}
+
+// The same tensors cut into 4096-element pieces (whole-tensor layouts only): the view the
+// first kernel of dq_tensor_norms works on.
+inline LayoutView make_piece_view(const dq_layout* L)
+{
+    LayoutView v;
+    const int32_t n1 = L->n_seg + 1;
+    v.n_seg = L->n_seg;
+    v.groups_per_bucket = 128;
+    v.total_groups = (int32_t)(L->padded / 32);
+    v.nb = (int32_t)L->n_pieces;
+    v.seg0_elems = (int32_t)L->seg_elems[0];
+    v.seg_group0 = L->dev_table ? L->dev_table + 3 * n1 : nullptr;
+    v.seg_bucket0 = L->dev_table ? L->dev_table + 4 * n1 : nullptr;
+    v.seg_elems = L->dev_table ? L->dev_table + 5 * n1 : nullptr;
     return v;
 }
 

@@ -8,6 +8,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "dq.h"
+
 // Round keys of Philox4x32-10: key + r * (0x9E3779B9, 0xBB67AE85).  They are the
 // same for the whole grid, so the host computes them and they travel as kernel
 // arguments (constant bank), which keeps them out of the register file.
@@ -48,6 +50,34 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
         c2 = n2;
     }
     out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// The three places where the members of the l_p family differ.  P = DQ_NORM_L2: sum of
+// squares, square root at the end.  P = DQ_NORM_LINF: running maximum of the magnitudes
+// (max.NaN, so that a NaN entry is not skipped and reaches the status word), nothing at the end.
+__device__ __forceinline__ float max_nan(const float a, const float b)
+{
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+    return d;
+}
+template <int P>
+__device__ __forceinline__ float take(const float acc, const float x)
+{
+    if constexpr (P == DQ_NORM_L2) return fmaf(x, x, acc);
+    else return max_nan(acc, fabsf(x));
+}
+template <int P>
+__device__ __forceinline__ float join(const float a, const float b)
+{
+    if constexpr (P == DQ_NORM_L2) return a + b;
+    else return max_nan(a, b);
+}
+template <int P>
+__device__ __forceinline__ float finish(const float a)
+{
+    if constexpr (P == DQ_NORM_L2) return sqrtf(a);
+    else return a;
 }
 
 // (a & mask) | c as one three-input logic operation.  `c` must come from a register the

@@ -1,5 +1,5 @@
-// dq_norms_quantize_pack: bucket norms (Eq. 5) and quantize+pack (Eq. 5/6) in one
-// pass over the gradients.
+// dq_norms_quantize_pack: bucket norms (Eq. 5; l_2 or l_inf, as the layout says) and
+// quantize+pack (Eq. 5/6) in one pass over the gradients.
 //
 // Algorithm 1 takes b_{t+1} from the gradients of iteration t, so the bit width of
 // a step is known before its gradients are: once a bucket sits in shared
@@ -77,7 +77,7 @@ struct FusedArgs {
     uint32_t one_bits;            // 0x3F800040, kept out of the compiler's sight (see and_or)
 };
 
-template <int B>
+template <int B, int P>
 __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMap* map)
 {
     // the tensor table of a multi-tensor layout always sits in shared memory here (the host
@@ -175,31 +175,31 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
-                    a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                    a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
                 }
             } else {                             // last group of a tensor: what follows is padding
                 for (int e = 0; e < valid; ++e) {
                     const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
-                    a0 = fmaf(x, x, a0);
+                    a0 = take<P>(a0, x);
                 }
             }
         }
-        float sum = (a0 + a1) + (a2 + a3);
+        float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
         // butterfly over the threads of the bucket: the steps up to its size, smallest distance last
         // (the same order as in dq_bucket_norms)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const float other = __shfl_xor_sync(0xffffffffu, sum, o);
-            if (o < gpb) sum += other;
+            if (o < gpb) sum = join<P>(sum, other);
         }
         if (gpb > 32) {
             if (lane == 0) part[warp] = sum;
             __syncthreads();
             sum = 0.f;
             const int w0 = (tid >> a.gpb_shift << a.gpb_shift) >> 5;        // first warp of this bucket
-            for (int i = 0; i < (gpb >> 5); ++i) sum += part[w0 + i];
+            for (int i = 0; i < (gpb >> 5); ++i) sum = join<P>(sum, part[w0 + i]);
         }
-        const float nrm = sqrtf(sum);
+        const float nrm = finish<P>(sum);
         if (l == 0 && k < nb) {
             a.norms[(int64_t)m * nb + k] = nrm;
             bad |= !isfinite(nrm);
@@ -270,7 +270,7 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
 // and every lane looks its bucket up in the tensor table.  Leaves the lane's words in the
 // staging area (the consumed stage) and returns the tile's span in groups, plus 256 if a
 // norm is not finite.
-template <int B>
+template <int B, int P>
 __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* base, const int row0, const int m, const int kt)
 {
     const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kWTblOffset);
@@ -316,22 +316,22 @@ __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* ba
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
-                a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
             }
         } else {                                 // last group of a tensor: what follows is padding
             for (int e = 0; e < valid; ++e) {
                 const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
-                a0 = fmaf(x, x, a0);
+                a0 = take<P>(a0, x);
             }
         }
     }
-    float sum = (a0 + a1) + (a2 + a3);
+    float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         const float other = __shfl_xor_sync(0xffffffffu, sum, o);
-        if (o < gpb) sum += other;
+        if (o < gpb) sum = join<P>(sum, other);
     }
-    const float nrm = sqrtf(sum);
+    const float nrm = finish<P>(sum);
     int bad = 0;
     if (l == 0 && k < nb) {
         a.norms[(int64_t)m * nb + k] = nrm;
@@ -380,7 +380,7 @@ __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* ba
 // two tiles ahead from a cached description of the tensor it is in (when it fetches the
 // tile) and keeps the answer in a two-deep register queue for the consumer side.  Only
 // tiles that touch the end of a tensor take the general route with per-lane table walks.
-template <int B>
+template <int B, int P>
 __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUtensorMap* map)
 {
     const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kWTblOffset);
@@ -478,15 +478,15 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float4 x = *reinterpret_cast<const float4*>(smem + (own ^ (uint32_t)(c << 4)));
-                a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
             }
-            float sum = (a0 + a1) + (a2 + a3);
+            float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
                 const float other = __shfl_xor_sync(0xffffffffu, sum, o);
-                if (o < gpb) sum += other;
+                if (o < gpb) sum = join<P>(sum, other);
             }
-            const float nrm = sqrtf(sum);
+            const float nrm = finish<P>(sum);
             if (l == 0) {
                 a.norms[(int64_t)m * nb + (kt * R + r)] = nrm;
                 bad |= !isfinite(nrm);
@@ -539,7 +539,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 span = 0;
             }
         } else {
-            const int res = irregular_tile<B>(a, base, row0, m, kt);
+            const int res = irregular_tile<B, P>(a, base, row0, m, kt);
             span = res & 0xff;
             bad |= (res >> 8) != 0;
         }
@@ -582,6 +582,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
     }
 }
 
+template <int P>
 __global__ void __launch_bounds__(kThreads, 6)
 norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
@@ -610,7 +611,7 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
     }
 
     switch (b) {
-#define DQ_CASE(BB) case BB: fused_warp_tiles<BB>(a, &map); break;
+#define DQ_CASE(BB) case BB: fused_warp_tiles<BB, P>(a, &map); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -619,6 +620,7 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
 }
 
 // ---- buckets that span several warps: the CTA is the pipeline -----------------------
+template <int P>
 __global__ void __launch_bounds__(kThreads, 5)
 norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
@@ -648,7 +650,7 @@ norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_con
     }
 
     switch (b) {
-#define DQ_CASE(BB) case BB: fused_tiles<BB>(a, &map); break;
+#define DQ_CASE(BB) case BB: fused_tiles<BB, P>(a, &map); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -672,6 +674,7 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
         return DQ_ERR_ALIGN;
     if (M > 1 && worker_stride_elems < L->padded && worker_stride_elems != 0) return DQ_ERR_RANGE;
     if (packed_stride_words < L->padded / 32) return DQ_ERR_RANGE;
+    if (L->whole_tensor) return DQ_ERR_RANGE;           // one norm per tensor: the codes need a second pass
 
     const uint32_t gpb = (uint32_t)(L->bucket / 32);
     if ((gpb & (gpb - 1)) != 0 || L->n_seg > kMaxSmemSegs) {
@@ -712,7 +715,9 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
     const size_t tbl_bytes = L->n_seg > 1 ? (size_t)3 * (L->n_seg + 1) * 4 : 0;
     if (per_warp) {
         const size_t smem_need = (size_t)kWTblOffset + tbl_bytes;
-        if (cudaFuncSetAttribute(norms_quantize_pack_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        const auto kernel = (L->norm == DQ_NORM_LINF) ? norms_quantize_pack_warp_kernel<DQ_NORM_LINF>
+                                                      : norms_quantize_pack_warp_kernel<DQ_NORM_L2>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem_need) != cudaSuccess) {
             (void)cudaGetLastError();
             return DQ_ERR_CUDA;
@@ -721,10 +726,12 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
         const int64_t warp_tiles = (int64_t)M * ((L->nb + R - 1) / R);
         int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
         if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
-        norms_quantize_pack_warp_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
+        kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
     } else {
         const size_t smem_need = (size_t)kTblOffset + tbl_bytes;
-        if (cudaFuncSetAttribute(norms_quantize_pack_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        const auto kernel = (L->norm == DQ_NORM_LINF) ? norms_quantize_pack_kernel<DQ_NORM_LINF>
+                                                      : norms_quantize_pack_kernel<DQ_NORM_L2>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem_need) != cudaSuccess) {
             (void)cudaGetLastError();
             return DQ_ERR_CUDA;
@@ -733,7 +740,7 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
         const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
         int64_t blocks = (int64_t)dq_sm_count() * 5;   // five 42 KB CTAs per SM
         if (blocks > tiles) blocks = tiles;
-        norms_quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
+        kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
     }
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;

@@ -7,43 +7,78 @@
 
 static inline int64_t up32(int64_t n) { return (n + 31) / 32 * 32; }
 
-extern "C" int dq_layout_create(const int64_t* seg_elems, int32_t n_seg, int32_t bucket, dq_layout_t** out)
+extern "C" int dq_layout_create_ex(const int64_t* seg_elems, int32_t n_seg, int32_t bucket, int32_t norm,
+                                   dq_layout_t** out)
 {
     if (!seg_elems || !out || n_seg < 1) return DQ_ERR_ARG;
-    if (bucket < 32 || bucket > DQ_MAX_BUCKET || bucket % 32 != 0) return DQ_ERR_RANGE;
-    int64_t padded = 0, nb = 0;
+    if (norm != DQ_NORM_L2 && norm != DQ_NORM_LINF) return DQ_ERR_ARG;
+    const bool whole = (bucket == DQ_BUCKET_WHOLE_TENSOR);
+    if (!whole && (bucket < 32 || bucket > DQ_MAX_BUCKET || bucket % 32 != 0)) return DQ_ERR_RANGE;
+    int64_t padded = 0, largest = 0;
     for (int32_t i = 0; i < n_seg; ++i) {
         if (seg_elems[i] < 0 || seg_elems[i] >= (int64_t(1) << 31)) return DQ_ERR_RANGE;
+        if (whole && seg_elems[i] > DQ_MAX_TENSOR_ELEMS) return DQ_ERR_RANGE;
         padded += up32(seg_elems[i]);
-        nb += (seg_elems[i] + bucket - 1) / bucket;
+        if (seg_elems[i] > largest) largest = seg_elems[i];
         if (padded >= (int64_t(1) << 31)) return DQ_ERR_RANGE;
     }
     if (padded == 0) return DQ_ERR_RANGE;
+    if (whole) {
+        // a bucket of 32 * 2^k elements that holds the largest tensor: every tensor is one bucket,
+        // and the kernels that map groups to buckets divide by a power of two
+        int64_t bk = 32;
+        while (bk < largest) bk *= 2;
+        bucket = (int32_t)bk;
+    }
     dq_layout* L = new (std::nothrow) dq_layout;
     if (!L) return DQ_ERR_ARG;
     L->n_seg = n_seg;
     L->bucket = bucket;
     L->padded = padded;
-    L->nb = nb;
+    L->norm = norm;
+    L->whole_tensor = whole;
     L->seg_elems.assign(seg_elems, seg_elems + n_seg);
     L->seg_offset.resize(n_seg);
     const int32_t n1 = n_seg + 1;
-    L->table.assign(size_t(3) * n1, 0);
-    int64_t p = 0, k = 0;
+    L->table.assign(size_t(whole ? 6 : 3) * n1, 0);
+    constexpr int64_t kPiece = 4096;
+    int64_t p = 0, k = 0, c = 0;
     for (int32_t i = 0; i < n_seg; ++i) {
         L->seg_offset[i] = p;
         L->table[i] = (int32_t)(p / 32);
         L->table[n1 + i] = (int32_t)k;
         L->table[2 * n1 + i] = (int32_t)seg_elems[i];
+        if (whole) {
+            L->table[3 * n1 + i] = (int32_t)(p / 32);
+            L->table[4 * n1 + i] = (int32_t)c;
+            L->table[5 * n1 + i] = (int32_t)seg_elems[i];
+            c += (seg_elems[i] + kPiece - 1) / kPiece;
+        }
         p += up32(seg_elems[i]);
         k += (seg_elems[i] + bucket - 1) / bucket;
     }
     L->table[n_seg] = (int32_t)(p / 32);
     L->table[n1 + n_seg] = (int32_t)k;
     L->table[2 * n1 + n_seg] = 0;
+    if (whole) {
+        L->table[3 * n1 + n_seg] = (int32_t)(p / 32);
+        L->table[4 * n1 + n_seg] = (int32_t)c;
+        L->table[5 * n1 + n_seg] = 0;
+    }
+    L->nb = k;
+    L->n_pieces = c;
     *out = L;
     return DQ_OK;
 }
+
+extern "C" int dq_layout_create(const int64_t* seg_elems, int32_t n_seg, int32_t bucket, dq_layout_t** out)
+{
+    if (bucket == DQ_BUCKET_WHOLE_TENSOR) return DQ_ERR_RANGE;      // only through dq_layout_create_ex
+    return dq_layout_create_ex(seg_elems, n_seg, bucket, DQ_NORM_L2, out);
+}
+
+extern "C" int32_t dq_layout_norm(const dq_layout_t* L) { return L ? L->norm : DQ_NORM_L2; }
+extern "C" int32_t dq_layout_whole_tensor(const dq_layout_t* L) { return (L && L->whole_tensor) ? 1 : 0; }
 
 extern "C" void dq_layout_destroy(dq_layout_t* layout) { delete layout; }
 

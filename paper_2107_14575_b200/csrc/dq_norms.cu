@@ -1,5 +1,6 @@
-// dq_bucket_norms: per-bucket l2 norm of every worker's gradient (the scale
-// factor ||g||_p of Eq. 5 with p = 2, applied per bucket).
+// dq_bucket_norms: per-bucket norm of every worker's gradient (the scale factor
+// ||g||_p of Eq. 5 applied per bucket; p = 2, or p = infinity for layouts created
+// with DQ_NORM_LINF), and dq_tensor_norms: one norm per tensor.
 //
 // One team of LANES threads (8, 16 or a full warp, by bucket size) owns a
 // bucket: 128-bit coalesced loads, four independent fp32 accumulators per
@@ -8,6 +9,7 @@
 // searched once per run and then followed; neighbouring warps read neighbouring
 // memory.  HBM-bound: 4 bytes read per element, 4/bucket bytes written.
 #include "dq_common.cuh"
+#include "dq_device.cuh"
 #include "dq_tma.cuh"
 
 namespace {
@@ -15,7 +17,7 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kRun = 8;            // bucket rows a warp handles per run
 
-template <int LANES>
+template <int LANES, int P>
 __global__ void __launch_bounds__(kThreads)
 bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const int64_t worker_stride,
                     float* __restrict__ norms, int32_t* __restrict__ status)
@@ -69,24 +71,24 @@ bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const i
                 const float4 x1 = __ldg(g4 + i + LANES);
                 const float4 x2 = __ldg(g4 + i + 2 * LANES);
                 const float4 x3 = __ldg(g4 + i + 3 * LANES);
-                a0 = fmaf(x0.x, x0.x, a0); a1 = fmaf(x0.y, x0.y, a1); a2 = fmaf(x0.z, x0.z, a2); a3 = fmaf(x0.w, x0.w, a3);
-                a0 = fmaf(x1.x, x1.x, a0); a1 = fmaf(x1.y, x1.y, a1); a2 = fmaf(x1.z, x1.z, a2); a3 = fmaf(x1.w, x1.w, a3);
-                a0 = fmaf(x2.x, x2.x, a0); a1 = fmaf(x2.y, x2.y, a1); a2 = fmaf(x2.z, x2.z, a2); a3 = fmaf(x2.w, x2.w, a3);
-                a0 = fmaf(x3.x, x3.x, a0); a1 = fmaf(x3.y, x3.y, a1); a2 = fmaf(x3.z, x3.z, a2); a3 = fmaf(x3.w, x3.w, a3);
+                a0 = take<P>(a0, x0.x); a1 = take<P>(a1, x0.y); a2 = take<P>(a2, x0.z); a3 = take<P>(a3, x0.w);
+                a0 = take<P>(a0, x1.x); a1 = take<P>(a1, x1.y); a2 = take<P>(a2, x1.z); a3 = take<P>(a3, x1.w);
+                a0 = take<P>(a0, x2.x); a1 = take<P>(a1, x2.y); a2 = take<P>(a2, x2.z); a3 = take<P>(a3, x2.w);
+                a0 = take<P>(a0, x3.x); a1 = take<P>(a1, x3.y); a2 = take<P>(a2, x3.z); a3 = take<P>(a3, x3.w);
             }
             for (; i < n4; i += LANES) {
                 const float4 x = __ldg(g4 + i);
-                a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
             }
             if (lane < (len & 3)) {                       // ragged tail of the tensor's last bucket
                 const float x = __ldg(g + n4 * 4 + lane);
-                a0 = fmaf(x, x, a0);
+                a0 = take<P>(a0, x);
             }
-            float sum = (a0 + a1) + (a2 + a3);
+            float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
 #pragma unroll
-            for (int o = LANES / 2; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o, LANES);
+            for (int o = LANES / 2; o > 0; o >>= 1) sum = join<P>(sum, __shfl_xor_sync(0xffffffffu, sum, o, LANES));
             if (lane == 0 && active) {
-                const float nrm = sqrtf(sum);
+                const float nrm = finish<P>(sum);
                 nw[k] = nrm;
                 bad |= !isfinite(nrm);
             }
@@ -101,6 +103,7 @@ bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const i
 // eight buckets with independent accumulators, and finally reduces the eight
 // per-lane sums together with a butterfly that halves the number of live
 // values at each of its first three steps (9 shuffles instead of 40).
+template <int P>
 __global__ void __launch_bounds__(kThreads)
 bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, const int64_t worker_stride,
                          float* __restrict__ norms, int32_t* __restrict__ status)
@@ -170,16 +173,16 @@ bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, co
                 const float4 x1 = (i + 32 < n4) ? __ldg(g4 + i + 32) : z;
                 const float4 x2 = (i + 64 < n4) ? __ldg(g4 + i + 64) : z;
                 const float4 x3 = (i + 96 < n4) ? __ldg(g4 + i + 96) : z;
-                a0 = fmaf(x0.x, x0.x, a0); a1 = fmaf(x0.y, x0.y, a1); a2 = fmaf(x0.z, x0.z, a2); a3 = fmaf(x0.w, x0.w, a3);
-                a0 = fmaf(x1.x, x1.x, a0); a1 = fmaf(x1.y, x1.y, a1); a2 = fmaf(x1.z, x1.z, a2); a3 = fmaf(x1.w, x1.w, a3);
-                a0 = fmaf(x2.x, x2.x, a0); a1 = fmaf(x2.y, x2.y, a1); a2 = fmaf(x2.z, x2.z, a2); a3 = fmaf(x2.w, x2.w, a3);
-                a0 = fmaf(x3.x, x3.x, a0); a1 = fmaf(x3.y, x3.y, a1); a2 = fmaf(x3.z, x3.z, a2); a3 = fmaf(x3.w, x3.w, a3);
+                a0 = take<P>(a0, x0.x); a1 = take<P>(a1, x0.y); a2 = take<P>(a2, x0.z); a3 = take<P>(a3, x0.w);
+                a0 = take<P>(a0, x1.x); a1 = take<P>(a1, x1.y); a2 = take<P>(a2, x1.z); a3 = take<P>(a3, x1.w);
+                a0 = take<P>(a0, x2.x); a1 = take<P>(a1, x2.y); a2 = take<P>(a2, x2.z); a3 = take<P>(a3, x2.w);
+                a0 = take<P>(a0, x3.x); a1 = take<P>(a1, x3.y); a2 = take<P>(a2, x3.z); a3 = take<P>(a3, x3.w);
             }
             if (lane < (len[r] & 3)) {                 // ragged tail of a tensor's last bucket
                 const float x = __ldg(gw + (int64_t)first[r] * 4 + n4 * 4 + lane);
-                a0 = fmaf(x, x, a0);
+                a0 = take<P>(a0, x);
             }
-            part[r] = (a0 + a1) + (a2 + a3);
+            part[r] = join<P>(join<P>(a0, a1), join<P>(a2, a3));
         }
         // butterfly: after the three halving steps lane l holds bucket (l & 7) summed over its octet
         float q[4], h[2], t;
@@ -187,23 +190,23 @@ bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, co
         for (int i = 0; i < 4; ++i) {
             const float keep = (lane & 1) ? part[2 * i + 1] : part[2 * i];
             const float give = (lane & 1) ? part[2 * i] : part[2 * i + 1];
-            q[i] = keep + __shfl_xor_sync(0xffffffffu, give, 1);
+            q[i] = join<P>(keep, __shfl_xor_sync(0xffffffffu, give, 1));
         }
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const float keep = (lane & 2) ? q[2 * i + 1] : q[2 * i];
             const float give = (lane & 2) ? q[2 * i] : q[2 * i + 1];
-            h[i] = keep + __shfl_xor_sync(0xffffffffu, give, 2);
+            h[i] = join<P>(keep, __shfl_xor_sync(0xffffffffu, give, 2));
         }
         {
             const float keep = (lane & 4) ? h[1] : h[0];
             const float give = (lane & 4) ? h[0] : h[1];
-            t = keep + __shfl_xor_sync(0xffffffffu, give, 4);
+            t = join<P>(keep, __shfl_xor_sync(0xffffffffu, give, 4));
         }
-        t += __shfl_xor_sync(0xffffffffu, t, 8);
-        t += __shfl_xor_sync(0xffffffffu, t, 16);
+        t = join<P>(t, __shfl_xor_sync(0xffffffffu, t, 8));
+        t = join<P>(t, __shfl_xor_sync(0xffffffffu, t, 16));
         if (lane < kRun && k0 + lane < v.nb) {
-            const float nrm = sqrtf(t);
+            const float nrm = finish<P>(t);
             nw[k0 + lane] = nrm;
             bad |= !isfinite(nrm);
         }
@@ -243,6 +246,10 @@ struct NormsArgs {
     int32_t stream_reads;        // 1: the gradients exceed the L2, read them with the evict-first policy
 };
 
+// RAW: the kernel writes the unfinished reduction (sum of squares, or maximum) of every
+// bucket instead of its norm -- the first step of dq_tensor_norms, whose "buckets" are the
+// 4096-element pieces of the tensors.
+template <int P, bool RAW>
 __global__ void __launch_bounds__(kTmaThreads)
 bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_constant__ CUtensorMap map)
 {
@@ -342,29 +349,29 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
-                    a0 = fmaf(x.x, x.x, a0); a1 = fmaf(x.y, x.y, a1); a2 = fmaf(x.z, x.z, a2); a3 = fmaf(x.w, x.w, a3);
+                    a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
                 }
             } else {                             // last group of a tensor: what follows is padding
                 for (int e = 0; e < valid; ++e) {
                     const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
-                    a0 = fmaf(x, x, a0);
+                    a0 = take<P>(a0, x);
                 }
             }
         }
-        float sum = (a0 + a1) + (a2 + a3);
+        float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
         // combine the gpb threads of a bucket: inside a warp by shuffles ...
         const int w = gpb < 32 ? gpb : 32;
-        for (int o = w >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        for (int o = w >> 1; o > 0; o >>= 1) sum = join<P>(sum, __shfl_xor_sync(0xffffffffu, sum, o));
         if (gpb > 32) {                          // ... and across the warps of a bucket through shared memory
             if (lane == 0) part[warp] = sum;
             __syncthreads();
             if (l == 0) {
                 sum = 0.f;
-                for (int i = 0; i < (gpb >> 5); ++i) sum += part[(tid >> 5) + i];
+                for (int i = 0; i < (gpb >> 5); ++i) sum = join<P>(sum, part[(tid >> 5) + i]);
             }
         }
         if (l == 0 && k < nb) {
-            const float nrm = sqrtf(sum);
+            const float nrm = RAW ? sum : finish<P>(sum);
             a.norms[(int64_t)m * nb + k] = nrm;
             bad |= !isfinite(nrm);
         }
@@ -381,58 +388,103 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
     }
 }
 
-}  // namespace
+// Second step of dq_tensor_norms: block (tensor, worker) reduces the unfinished results of the
+// tensor's pieces in a fixed order -- thread t takes pieces t, t + 256, ..., then a tree over the
+// block -- and writes the tensor's norm.  Sums of squares are added in fp64 and rounded to fp32
+// before the square root, which keeps norm >= |g_j| for every entry (each piece's sum is at
+// least fl(g_j^2), rounding is monotone, and sqrtf(fl(g^2)) = |g|).
+constexpr int kJoinThreads = 256;
 
-extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
-                               int32_t M, float* dev_norms, int32_t* dev_status, void* stream)
+template <int P>
+__global__ void __launch_bounds__(kJoinThreads)
+tensor_norms_join_kernel(const int32_t n_seg, const int32_t* __restrict__ piece0, const int32_t* __restrict__ bucket0,
+                         const int32_t n_pieces, const int32_t nb, const float* __restrict__ partial,
+                         float* __restrict__ norms, int32_t* __restrict__ status)
 {
-    const int rc = dq_check_common(L, M);
-    if (rc != DQ_OK) return rc;
-    if (!dev_grads || !dev_norms || !dev_status) return DQ_ERR_ARG;
-    if (!aligned16(dev_grads) || (worker_stride_elems % 32) != 0 || (reinterpret_cast<uintptr_t>(dev_norms) & 3u) ||
-        (reinterpret_cast<uintptr_t>(dev_status) & 3u))
-        return DQ_ERR_ALIGN;
-    if (M > 1 && worker_stride_elems < L->padded && worker_stride_elems != 0) return DQ_ERR_RANGE;
-
-    const LayoutView v = make_view(L);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const uint32_t gpb = (uint32_t)v.groups_per_bucket;
-    if ((gpb & (gpb - 1)) == 0) {
-        // bucket = 32 * 2^k: bulk-copy kernel
-        NormsArgs a;
-        a.v = v;
-        a.grads = dev_grads;
-        a.norms = dev_norms;
-        a.status = dev_status;
-        a.M = M;
-        a.gpb_shift = 0;
-        while ((1u << a.gpb_shift) < gpb) ++a.gpb_shift;
-        a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
-        const bool worker_dim = (M > 1 && worker_stride_elems != 0);
-        a.map_has_worker_dim = worker_dim ? 1 : 0;
-        CUtensorMap map;
-        const uint64_t dims[3] = {32, (uint64_t)v.total_groups, worker_dim ? (uint64_t)M : 1};
-        const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
-        const uint32_t box[3] = {32, (uint32_t)kTmaThreads, 1};
-        if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
-                                  CU_TENSOR_MAP_SWIZZLE_128B))
-            return DQ_ERR_CUDA;
-        size_t smem_need = (size_t)kTblOffset;
-        if (L->n_seg > 1 && L->n_seg <= kTmaMaxSmemSegs) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
-        if (cudaFuncSetAttribute(bucket_norms_tma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return DQ_ERR_CUDA;
-        }
-        const int R = kTmaThreads >> a.gpb_shift;
-        const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
-        int64_t blocks = (int64_t)dq_sm_count() * 3;    // three 65 KB CTAs per SM
-        if (blocks > tiles) blocks = tiles;
-        bucket_norms_tma_kernel<<<(unsigned)blocks, kTmaThreads, smem_need, st>>>(a, map);
-        if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
-        return DQ_OK;
+    __shared__ double part_d[kJoinThreads / 32];
+    __shared__ float part_f[kJoinThreads / 32];
+    const int seg = blockIdx.x, m = blockIdx.y;
+    int c0 = 0, c1 = n_pieces, k = 0;
+    if (n_seg > 1) {
+        c0 = __ldg(piece0 + seg);
+        c1 = __ldg(piece0 + seg + 1);
+        k = __ldg(bucket0 + seg);
     }
+    if (c0 >= c1) return;                                    // an empty tensor has no norm
+    const float* src = partial + (int64_t)m * n_pieces;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    float nrm;
+    if constexpr (P == DQ_NORM_L2) {
+        double acc = 0.0;
+        for (int i = c0 + tid; i < c1; i += kJoinThreads) acc += (double)__ldg(src + i);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) part_d[warp] = acc;
+        __syncthreads();
+        if (tid != 0) return;
+        double total = 0.0;
+        for (int w = 0; w < kJoinThreads / 32; ++w) total += part_d[w];
+        nrm = sqrtf((float)total);
+    } else {
+        float acc = 0.0f;
+        for (int i = c0 + tid; i < c1; i += kJoinThreads) acc = max_nan(acc, __ldg(src + i));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc = max_nan(acc, __shfl_xor_sync(0xffffffffu, acc, o));
+        if (lane == 0) part_f[warp] = acc;
+        __syncthreads();
+        if (tid != 0) return;
+        float total = 0.0f;
+        for (int w = 0; w < kJoinThreads / 32; ++w) total = max_nan(total, part_f[w]);
+        nrm = total;
+    }
+    norms[(int64_t)m * nb + k] = nrm;
+    if (!isfinite(nrm)) atomicOr(status, DQ_STAT_NONFINITE);
+}
 
-    // other bucket sizes: plain-load kernels
+// Launch of the bulk-copy kernel over view `v` (groups per bucket a power of two, at most 128).
+template <int P, bool RAW>
+int launch_tma(const dq_layout_t* L, const LayoutView& v, const float* dev_grads, int64_t worker_stride_elems, int32_t M,
+               float* dev_out, int32_t* dev_status, cudaStream_t st)
+{
+    const uint32_t gpb = (uint32_t)v.groups_per_bucket;
+    NormsArgs a;
+    a.v = v;
+    a.grads = dev_grads;
+    a.norms = dev_out;
+    a.status = dev_status;
+    a.M = M;
+    a.gpb_shift = 0;
+    while ((1u << a.gpb_shift) < gpb) ++a.gpb_shift;
+    a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
+    const bool worker_dim = (M > 1 && worker_stride_elems != 0);
+    a.map_has_worker_dim = worker_dim ? 1 : 0;
+    CUtensorMap map;
+    const uint64_t dims[3] = {32, (uint64_t)v.total_groups, worker_dim ? (uint64_t)M : 1};
+    const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
+    const uint32_t box[3] = {32, (uint32_t)kTmaThreads, 1};
+    if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
+                              CU_TENSOR_MAP_SWIZZLE_128B))
+        return DQ_ERR_CUDA;
+    size_t smem_need = (size_t)kTblOffset;
+    if (L->n_seg > 1 && L->n_seg <= kTmaMaxSmemSegs) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
+    if (cudaFuncSetAttribute(bucket_norms_tma_kernel<P, RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return DQ_ERR_CUDA;
+    }
+    const int R = kTmaThreads >> a.gpb_shift;
+    const int64_t tiles = (int64_t)M * ((v.nb + R - 1) / R);
+    int64_t blocks = (int64_t)dq_sm_count() * 3;    // three 65 KB CTAs per SM
+    if (blocks > tiles) blocks = tiles;
+    bucket_norms_tma_kernel<P, RAW><<<(unsigned)blocks, kTmaThreads, smem_need, st>>>(a, map);
+    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+// other bucket sizes: plain-load kernels
+template <int P>
+int launch_plain(const dq_layout_t* L, const LayoutView& v, const float* dev_grads, int64_t worker_stride_elems, int32_t M,
+                 float* dev_norms, int32_t* dev_status, cudaStream_t st)
+{
     const int lanes = L->bucket >= 128 ? 32 : (L->bucket >= 64 ? 16 : 8);
     const int64_t chunk = (int64_t)kRun * (32 / lanes);
     const int64_t nchunks = (L->nb + chunk - 1) / chunk;
@@ -445,12 +497,85 @@ extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int
     const dim3 grid((unsigned)bx, (unsigned)M);
     if (lanes == 32) {
         const size_t smem = (L->n_seg > 1 && (size_t)3 * (L->n_seg + 1) * 4 <= 12 * 1024) ? (size_t)3 * (L->n_seg + 1) * 4 : 0;
-        bucket_norms_warp_kernel<<<grid, kThreads, smem, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+        bucket_norms_warp_kernel<P><<<grid, kThreads, smem, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
     }
     else if (lanes == 16)
-        bucket_norms_kernel<16><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+        bucket_norms_kernel<16, P><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
     else
-        bucket_norms_kernel<8><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+        bucket_norms_kernel<8, P><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
+    return DQ_OK;
+}
+
+int check_norm_args(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems, int32_t M,
+                    const float* dev_norms, const int32_t* dev_status)
+{
+    const int rc = dq_check_common(L, M);
+    if (rc != DQ_OK) return rc;
+    if (!dev_grads || !dev_norms || !dev_status) return DQ_ERR_ARG;
+    if (!aligned16(dev_grads) || (worker_stride_elems % 32) != 0 || (reinterpret_cast<uintptr_t>(dev_norms) & 3u) ||
+        (reinterpret_cast<uintptr_t>(dev_status) & 3u))
+        return DQ_ERR_ALIGN;
+    if (M > 1 && worker_stride_elems < L->padded && worker_stride_elems != 0) return DQ_ERR_RANGE;
+    return DQ_OK;
+}
+
+}  // namespace
+
+extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
+                               int32_t M, float* dev_norms, int32_t* dev_status, void* stream)
+{
+    const int rc = check_norm_args(L, dev_grads, worker_stride_elems, M, dev_norms, dev_status);
+    if (rc != DQ_OK) return rc;
+    if (L->whole_tensor) return DQ_ERR_RANGE;           // one norm per tensor comes from dq_tensor_norms
+
+    const LayoutView v = make_view(L);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const uint32_t gpb = (uint32_t)v.groups_per_bucket;
+    const bool linf = (L->norm == DQ_NORM_LINF);
+    if ((gpb & (gpb - 1)) == 0) {
+        // bucket = 32 * 2^k: bulk-copy kernel
+        return linf ? launch_tma<DQ_NORM_LINF, false>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st)
+                    : launch_tma<DQ_NORM_L2, false>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st);
+    }
+    return linf ? launch_plain<DQ_NORM_LINF>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st)
+                : launch_plain<DQ_NORM_L2>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st);
+}
+
+extern "C" size_t dq_tensor_norms_scratch_bytes(const dq_layout_t* L, int32_t M)
+{
+    if (!L || !L->whole_tensor || M < 1) return 0;
+    return (size_t)M * (size_t)L->n_pieces * sizeof(float);
+}
+
+extern "C" int dq_tensor_norms(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems, int32_t M,
+                               float* dev_norms, void* dev_scratch, size_t scratch_bytes, int32_t* dev_status,
+                               void* stream)
+{
+    const int rc = check_norm_args(L, dev_grads, worker_stride_elems, M, dev_norms, dev_status);
+    if (rc != DQ_OK) return rc;
+    if (!L->whole_tensor) return DQ_ERR_RANGE;          // bucketed layouts: dq_bucket_norms
+    if (!dev_scratch) return DQ_ERR_ARG;
+    if (!aligned16(dev_scratch)) return DQ_ERR_ALIGN;
+    if (scratch_bytes < dq_tensor_norms_scratch_bytes(L, M)) return DQ_ERR_RANGE;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float* partial = static_cast<float*>(dev_scratch);
+    const LayoutView pv = make_piece_view(L);
+    const bool linf = (L->norm == DQ_NORM_LINF);
+    const int r1 = linf ? launch_tma<DQ_NORM_LINF, true>(L, pv, dev_grads, worker_stride_elems, M, partial, dev_status, st)
+                        : launch_tma<DQ_NORM_L2, true>(L, pv, dev_grads, worker_stride_elems, M, partial, dev_status, st);
+    if (r1 != DQ_OK) return r1;
+    const int32_t n1 = L->n_seg + 1;
+    const int32_t* piece0 = L->n_seg > 1 ? L->dev_table + 4 * n1 : nullptr;
+    const int32_t* bucket0 = L->n_seg > 1 ? L->dev_table + n1 : nullptr;
+    const dim3 grid((unsigned)L->n_seg, (unsigned)M);
+    if (linf)
+        tensor_norms_join_kernel<DQ_NORM_LINF><<<grid, kJoinThreads, 0, st>>>(L->n_seg, piece0, bucket0, (int32_t)L->n_pieces,
+                                                                             (int32_t)L->nb, partial, dev_norms, dev_status);
+    else
+        tensor_norms_join_kernel<DQ_NORM_L2><<<grid, kJoinThreads, 0, st>>>(L->n_seg, piece0, bucket0, (int32_t)L->n_pieces,
+                                                                           (int32_t)L->nb, partial, dev_norms, dev_status);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }

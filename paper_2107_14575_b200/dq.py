@@ -16,13 +16,15 @@ LIB_PATH = os.path.join(_PKG, "libdq.so")
 
 OK, ERR_ARG, ERR_ALIGN, ERR_RANGE, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
 STAT_NONFINITE, STAT_BAD_BITS, STAT_CAPACITY, STAT_WAIT, STAT_INTERNAL = 1, 2, 4, 8, 16
+NORM_L2, NORM_LINF = 2, 0          # DQ_NORM_*: member of the l_p family of Eq. 5
+BUCKET_WHOLE_TENSOR = 0            # DQ_BUCKET_WHOLE_TENSOR: one norm per tensor
 
 # every symbol include/dq.h declares
 SYMBOLS = [
-    "dq_layout_create", "dq_layout_destroy", "dq_layout_num_segments", "dq_layout_padded_elems",
+    "dq_layout_create", "dq_layout_create_ex", "dq_layout_norm", "dq_layout_whole_tensor", "dq_layout_destroy", "dq_layout_num_segments", "dq_layout_padded_elems",
     "dq_layout_seg_offset", "dq_layout_num_buckets", "dq_layout_packed_words", "dq_layout_bucket",
     "dq_layout_table_bytes", "dq_layout_bind_device_table",
-    "dq_bucket_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
+    "dq_bucket_norms", "dq_tensor_norms_scratch_bytes", "dq_tensor_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
     "dq_choose_bits_noalloc_max_norms", "dq_choose_bits_noalloc",
     "dq_quantize_pack", "dq_norms_quantize_pack", "dq_unpack_dequant_average",
     "dq_unpack_average_update", "dq_status_string",
@@ -64,6 +66,12 @@ def lib():
         vp, i32, i64, u32, u64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_size_t
         L.dq_layout_create.restype = C.c_int
         L.dq_layout_create.argtypes = [C.POINTER(i64), i32, i32, C.POINTER(vp)]
+        L.dq_layout_create_ex.restype = C.c_int
+        L.dq_layout_create_ex.argtypes = [C.POINTER(i64), i32, i32, i32, C.POINTER(vp)]
+        L.dq_layout_norm.restype = i32
+        L.dq_layout_norm.argtypes = [vp]
+        L.dq_layout_whole_tensor.restype = i32
+        L.dq_layout_whole_tensor.argtypes = [vp]
         L.dq_layout_destroy.restype = None
         L.dq_layout_destroy.argtypes = [vp]
         L.dq_layout_num_segments.restype = i32
@@ -84,6 +92,10 @@ def lib():
         L.dq_layout_bind_device_table.argtypes = [vp, vp, sz, vp]
         L.dq_bucket_norms.restype = C.c_int
         L.dq_bucket_norms.argtypes = [vp, vp, i64, i32, vp, vp, vp]
+        L.dq_tensor_norms_scratch_bytes.restype = sz
+        L.dq_tensor_norms_scratch_bytes.argtypes = [vp, i32]
+        L.dq_tensor_norms.restype = C.c_int
+        L.dq_tensor_norms.argtypes = [vp, vp, i64, i32, vp, vp, sz, vp, vp]
         L.dq_choose_bits_scratch_bytes.restype = sz
         L.dq_choose_bits_scratch_bytes.argtypes = [vp, i32]
         L.dq_choose_bits.restype = C.c_int
@@ -134,14 +146,23 @@ def _stream(stream) -> int:
 
 
 class Layout:
-    """``dq_layout_t``: the padded, bucketed layout of a list of tensors."""
+    """``dq_layout_t``: the padded, bucketed layout of a list of tensors.
 
-    def __init__(self, seg_elems: Sequence[int], bucket: int):
+    ``bucket = BUCKET_WHOLE_TENSOR`` gives one norm per tensor (Eq. 5 as written);
+    ``norm`` picks the member of the l_p family the norm calls compute."""
+
+    def __init__(self, seg_elems: Sequence[int], bucket: int, norm: int = NORM_L2):
         arr = (C.c_int64 * len(seg_elems))(*[int(x) for x in seg_elems])
         h = C.c_void_p()
-        _check(lib().dq_layout_create(arr, len(seg_elems), int(bucket), C.byref(h)), "dq_layout_create")
+        if norm == NORM_L2 and bucket != BUCKET_WHOLE_TENSOR:
+            _check(lib().dq_layout_create(arr, len(seg_elems), int(bucket), C.byref(h)), "dq_layout_create")
+        else:
+            _check(lib().dq_layout_create_ex(arr, len(seg_elems), int(bucket), int(norm), C.byref(h)),
+                   "dq_layout_create_ex")
         self._h = h
         self.bucket = int(bucket)
+        self.norm = int(lib().dq_layout_norm(h))
+        self.whole_tensor = bool(lib().dq_layout_whole_tensor(h))
         self.n_seg = int(lib().dq_layout_num_segments(h))
         self.D32 = int(lib().dq_layout_padded_elems(h))
         self.nb = int(lib().dq_layout_num_buckets(h))
@@ -188,6 +209,17 @@ class Layout:
 def bucket_norms(layout: Layout, grads, worker_stride_elems: int, M: int, norms, status, stream=None) -> None:
     _check(lib().dq_bucket_norms(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(norms),
                                  _ptr(status), _stream(stream)), "dq_bucket_norms")
+
+
+def tensor_norms_scratch_bytes(layout: Layout, M: int) -> int:
+    return int(lib().dq_tensor_norms_scratch_bytes(layout.handle, int(M)))
+
+
+def tensor_norms(layout: Layout, grads, worker_stride_elems: int, M: int, norms, scratch, scratch_bytes: int, status,
+                 stream=None) -> None:
+    """One norm per tensor of a whole-tensor layout (``dq_tensor_norms``)."""
+    _check(lib().dq_tensor_norms(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(norms),
+                                 _ptr(scratch), int(scratch_bytes), _ptr(status), _stream(stream)), "dq_tensor_norms")
 
 
 def choose_bits_scratch_bytes(layout: Layout, M: int) -> int:

@@ -17,9 +17,9 @@ from . import dq
 
 class Round:
     def __init__(self, seg_elems: Sequence[int], bucket: int, M: int, max_bits: int = 16,
-                 device: str = "cuda", worker_stride: Optional[int] = None):
+                 device: str = "cuda", worker_stride: Optional[int] = None, norm: int = dq.NORM_L2):
         self.device = torch.device(device)
-        self.layout = dq.Layout(seg_elems, bucket).bind(self.device)
+        self.layout = dq.Layout(seg_elems, bucket, norm).bind(self.device)
         self.M = int(M)
         L = self.layout
         self.stride = L.D32 if worker_stride is None else int(worker_stride)
@@ -37,6 +37,9 @@ class Round:
         self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
         self.scratch_bytes = dq.choose_bits_scratch_bytes(L, M)
         self.scratch = torch.empty(max(self.scratch_bytes, 256), dtype=torch.uint8, device=self.device)
+        self.norm_scratch_bytes = dq.tensor_norms_scratch_bytes(L, M)
+        self.norm_scratch = (torch.empty(self.norm_scratch_bytes, dtype=torch.uint8, device=self.device)
+                             if self.norm_scratch_bytes else None)
         self._host_in = None
         self._host_out = None
         self._dev_in = None
@@ -48,7 +51,11 @@ class Round:
 
     # ---- the four calls, on device-resident gradients [M, stride] fp32 ----
     def norms_(self, grads) -> None:
-        dq.bucket_norms(self.layout, grads, self.stride, self.M, self.norms, self.status)
+        if self.layout.whole_tensor:
+            dq.tensor_norms(self.layout, grads, self.stride, self.M, self.norms, self.norm_scratch,
+                            self.norm_scratch_bytes, self.status)
+        else:
+            dq.bucket_norms(self.layout, grads, self.stride, self.M, self.norms, self.status)
 
     def bits_(self, rule: dq.Rule) -> None:
         dq.choose_bits(self.layout, self.norms, self.M, rule, self.dev_b, self.scratch, self.scratch_bytes,
@@ -59,7 +66,12 @@ class Round:
                          self.packed, self.packed_stride, self.status)
 
     def norms_quantize_(self, grads, seed: int, step: int) -> None:
-        """Norms and quantize+pack in one pass, with the b already in ``dev_b``."""
+        """Norms and quantize+pack in one pass, with the b already in ``dev_b`` (two passes for a
+        whole-tensor layout, whose codes need the norm of the whole tensor)."""
+        if self.layout.whole_tensor:
+            self.norms_(grads)
+            self.quantize_(grads, seed, step)
+            return
         dq.norms_quantize_pack(self.layout, grads, self.stride, self.M, self.dev_b, seed, step, self.norms,
                                self.packed, self.packed_stride, self.status)
 

@@ -27,8 +27,8 @@ class Guarded:
 class GpuRound:
     """Device state for one layout and worker count, driven through the C ABI."""
 
-    def __init__(self, segs, bucket, M, stride=None, packed_stride=None, max_bits=16):
-        self.lay = dq.Layout(segs, bucket).bind()
+    def __init__(self, segs, bucket, M, stride=None, packed_stride=None, max_bits=16, norm=dq.NORM_L2):
+        self.lay = dq.Layout(segs, bucket, norm).bind()
         self.M = M
         self.stride = self.lay.D32 if stride is None else stride
         self.pstride = ((self.lay.packed_words(max_bits) + 3) // 4 * 4) if packed_stride is None else packed_stride
@@ -39,6 +39,8 @@ class GpuRound:
         self.status = torch.zeros(1, dtype=torch.int32, device="cuda")
         self.sbytes = dq.choose_bits_scratch_bytes(self.lay, M)
         self.scratch = torch.empty(max(self.sbytes, 256), dtype=torch.uint8, device="cuda")
+        self.nbytes = dq.tensor_norms_scratch_bytes(self.lay, M)
+        self.g_nscratch = Guarded(max(self.nbytes // 4, 4), torch.float32)
         self.grads = None
 
     # -- inputs
@@ -59,7 +61,11 @@ class GpuRound:
 
     # -- calls
     def norms(self) -> np.ndarray:
-        dq.bucket_norms(self.lay, self.grads, self.stride, self.M, self.g_norms.view, self.status)
+        if self.lay.whole_tensor:
+            dq.tensor_norms(self.lay, self.grads, self.stride, self.M, self.g_norms.view, self.g_nscratch.view,
+                            self.nbytes, self.status)
+        else:
+            dq.bucket_norms(self.lay, self.grads, self.stride, self.M, self.g_norms.view, self.status)
         return self.g_norms.view.cpu().numpy().reshape(self.M, self.lay.nb)
 
     def bits(self, rule) -> tuple:
@@ -106,7 +112,8 @@ class GpuRound:
         self.status.zero_()
 
     def guards_intact(self) -> bool:
-        return self.g_norms.intact() and self.g_packed.intact() and self.g_out.intact() and self.g_b.intact()
+        return (self.g_norms.intact() and self.g_packed.intact() and self.g_out.intact() and self.g_b.intact()
+                and self.g_nscratch.intact())
 
 
 def rel_l2(a: np.ndarray, b: np.ndarray) -> float:

@@ -115,3 +115,44 @@ def test_argument_errors_need_no_gpu(dqlib):
     assert L.dq_bucket_norms(multi.handle, A, 256, 1, A, A, 0) == dqlib.ERR_STATE
     assert multi.table_bytes() == 36
     assert dqlib.choose_bits_scratch_bytes(lay, 4) == 256
+
+
+def test_norm_family_layouts(dqlib):
+    """Whole-tensor layouts agree with the oracle's (a bucket as large as the largest tensor), the
+    norm kind is remembered, and the host checks of the new calls need no GPU."""
+    segs = [1000, 33, 0, 5000, 1]
+    lay = dqlib.Layout(segs, dqlib.BUCKET_WHOLE_TENSOR, dqlib.NORM_LINF)
+    ref = oracle.Layout(segs, oracle.whole_tensor_bucket(segs))
+    assert lay.whole_tensor and lay.norm == dqlib.NORM_LINF
+    assert lay.D32 == ref.D32 and lay.nb == ref.nb == 4 and lay.offsets == ref.offsets.tolist()
+    for k in range(ref.nb):
+        assert lay.bucket_range(k) == (int(ref.bucket_start[k]), int(ref.bucket_len[k]))
+    assert lay.table_bytes() == 24 * (len(segs) + 1)         # bucket table and 4096-element piece table
+    # pieces: ceil(1000/4096) + ceil(33/4096) + 0 + ceil(5000/4096) + 1 = 5 per worker
+    assert dqlib.tensor_norms_scratch_bytes(lay, 3) == 3 * 5 * 4
+    plain = dqlib.Layout(segs, 64)
+    assert not plain.whole_tensor and plain.norm == dqlib.NORM_L2
+    assert dqlib.tensor_norms_scratch_bytes(plain, 3) == 0
+    assert dqlib.Layout(segs, 64, dqlib.NORM_LINF).norm == dqlib.NORM_LINF
+
+    L = dqlib.lib()
+    arr = (C.c_int64 * 1)(100)
+    h = C.c_void_p()
+    assert L.dq_layout_create_ex(arr, 1, 32, 7, C.byref(h)) == dqlib.ERR_ARG          # unknown norm
+    assert L.dq_layout_create(arr, 1, 0, C.byref(h)) == dqlib.ERR_RANGE               # whole tensor only via _ex
+    big = (C.c_int64 * 1)((1 << 30) + 1)
+    assert L.dq_layout_create_ex(big, 1, 0, dqlib.NORM_L2, C.byref(h)) == dqlib.ERR_RANGE
+
+    A = 0x7f0000001000
+    one = dqlib.Layout([10000], dqlib.BUCKET_WHOLE_TENSOR)
+    assert one.nb == 1 and one.table_bytes() == 0
+    need = dqlib.tensor_norms_scratch_bytes(one, 2)
+    assert need == 2 * 3 * 4
+    # the bucketed calls refuse a whole-tensor layout and the other way round
+    assert L.dq_bucket_norms(one.handle, A, 10016, 2, A, A, 0) == dqlib.ERR_RANGE
+    assert L.dq_norms_quantize_pack(one.handle, A, 10016, 2, A, 0, 0, A, A, 10016, A, 0) == dqlib.ERR_RANGE
+    flat = dqlib.Layout([10000], 512)
+    assert L.dq_tensor_norms(flat.handle, A, 10016, 2, A, A, 1 << 20, A, 0) == dqlib.ERR_RANGE
+    assert L.dq_tensor_norms(one.handle, A, 10016, 2, A, 0, need, A, 0) == dqlib.ERR_ARG
+    assert L.dq_tensor_norms(one.handle, A, 10016, 2, A, A + 4, need, A, 0) == dqlib.ERR_ALIGN
+    assert L.dq_tensor_norms(one.handle, A, 10016, 2, A, A, need - 1, A, 0) == dqlib.ERR_RANGE
