@@ -126,6 +126,26 @@ int64_t dq_layout_packed_words(const dq_layout_t* layout, int32_t b); /* b * D32
 /* start (padded element index) and valid length of bucket k; DQ_ERR_RANGE if k is invalid */
 int     dq_layout_bucket(const dq_layout_t* layout, int64_t k, int64_t* start, int64_t* len);
 
+/* ---- cutting the path across several GPUs (one worker per GPU, Algorithm 1's send /
+ * collect / average with the server's work divided among the GPUs).  The padded buffer is
+ * cut into contiguous ranges of whole buckets; GPU r averages range r of every worker's
+ * packed stream.  Range [k0, k1) of buckets owns the contiguous words
+ * [b * first_elem / 32, b * (first_elem + padded_elems(slice)) / 32) of a packed stream, the
+ * norms [k0, k1) and the same element range of the output.
+ *   dq_layout_shard_bounds  bounds[0..n_shards]: bounds[j] is the first bucket of shard j,
+ *                           bounds[n_shards] = nb; shards carry nearly equal numbers of
+ *                           elements (a shard may be empty when there are few buckets)
+ *   dq_layout_slice         buckets [k0, k1) as a layout of their own (same bucket size and
+ *                           norm; its tensors are the pieces of the parent's tensors inside
+ *                           the range; bucket j of the slice is bucket k0 + j of the parent);
+ *                           *first_elem (optional) = where the slice starts in the parent's
+ *                           padded buffer.  The caller destroys the slice, and binds a device
+ *                           table to it like to any layout with several tensors.
+ * Errors: DQ_ERR_ARG (NULL, n_shards < 1), DQ_ERR_RANGE (empty or invalid bucket range). */
+int     dq_layout_shard_bounds(const dq_layout_t* layout, int32_t n_shards, int64_t* bounds);
+int     dq_layout_slice(const dq_layout_t* layout, int64_t k0, int64_t k1, dq_layout_t** out,
+                        int64_t* first_elem);
+
 /* Layouts with more than one tensor need a small table on the device.  The
  * caller provides dq_layout_table_bytes() bytes of 16-byte aligned device
  * memory and keeps it alive while the layout is in use; bind copies the table
@@ -241,6 +261,17 @@ int dq_quantize_pack(const dq_layout_t* layout, const float* dev_grads, int64_t 
                      uint32_t* dev_packed, int64_t packed_stride_words,
                      int32_t* dev_status, void* stream);
 
+/* The same for workers first_worker .. first_worker + M - 1 of a larger job: worker m of
+ * the call draws the uniforms of worker first_worker + m (the third counter word above).
+ * With one worker per GPU, GPU r passes M = 1 and first_worker = r, and the words it
+ * produces are those of row r of a single call over all workers (Lemma 1's 1/W variance
+ * of the average needs the workers' draws to be independent). */
+int dq_quantize_pack_worker(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
+                            int32_t M, const float* dev_norms, const int32_t* dev_b,
+                            uint64_t seed, uint32_t step, uint32_t first_worker,
+                            uint32_t* dev_packed, int64_t packed_stride_words,
+                            int32_t* dev_status, void* stream);
+
 /* --------------------------- norms and quantizer in one pass, Eq. 5 and 6
  * dq_bucket_norms followed by dq_quantize_pack on the same gradients, with every
  * gradient byte read once: dev_norms receives exactly what dq_bucket_norms
@@ -257,6 +288,13 @@ int dq_norms_quantize_pack(const dq_layout_t* layout, const float* dev_grads, in
                            int32_t M, const int32_t* dev_b, uint64_t seed, uint32_t step,
                            float* dev_norms, uint32_t* dev_packed, int64_t packed_stride_words,
                            int32_t* dev_status, void* stream);
+
+/* dq_norms_quantize_pack for workers first_worker .. first_worker + M - 1 (see
+ * dq_quantize_pack_worker). */
+int dq_norms_quantize_pack_worker(const dq_layout_t* layout, const float* dev_grads, int64_t worker_stride_elems,
+                                  int32_t M, const int32_t* dev_b, uint64_t seed, uint32_t step,
+                                  uint32_t first_worker, float* dev_norms, uint32_t* dev_packed,
+                                  int64_t packed_stride_words, int32_t* dev_status, void* stream);
 
 /* ----------------------------------- Algorithm 1, server side: "Average"
  * dev_out[j] = (1/M) sum_m (code_m - s) * norm_m / s   (Eq. 5 inverted, then

@@ -70,6 +70,7 @@ struct FusedArgs {
     int32_t* status;
     PhiloxKeys keys;
     uint32_t step;
+    uint32_t worker0;             // worker m of the call draws the uniforms of worker worker0 + m
     int32_t M;
     int32_t map_has_worker_dim;
     int32_t gpb_shift;            // log2(groups per bucket)
@@ -226,7 +227,7 @@ __device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMa
                 encode_block<B, C>(acc, cur,                                                                    \
                                    *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)), \
                                    *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
-                                   inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+                                   inv, q0 + (C), (uint32_t)m + a.worker0, a.step, a.keys, a.one_bits);
                 DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
 #undef DQ_BLOCK
             }
@@ -357,7 +358,7 @@ __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* ba
             encode_block<B, C>(acc, cur,                                                                        \
                                *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)),     \
                                *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
-                               inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+                               inv, q0 + (C), (uint32_t)m + a.worker0, a.step, a.keys, a.one_bits);
             DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
 #undef DQ_BLOCK
         }
@@ -503,7 +504,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 encode_block<B, C>(acc, cur,                                                                    \
                                    *reinterpret_cast<const float4*>(smem + (own ^ (uint32_t)((2 * (C)) << 4))), \
                                    *reinterpret_cast<const float4*>(smem + (own ^ (uint32_t)((2 * (C) + 1) << 4))), \
-                                   inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+                                   inv, q0 + (C), (uint32_t)m + a.worker0, a.step, a.keys, a.one_bits);
                 DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
 #undef DQ_BLOCK
             }
@@ -660,10 +661,10 @@ norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_con
 
 }  // namespace
 
-extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
-                                      int32_t M, const int32_t* dev_b, uint64_t seed, uint32_t step,
-                                      float* dev_norms, uint32_t* dev_packed, int64_t packed_stride_words,
-                                      int32_t* dev_status, void* stream)
+extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
+                                             int32_t M, const int32_t* dev_b, uint64_t seed, uint32_t step,
+                                             uint32_t first_worker, float* dev_norms, uint32_t* dev_packed,
+                                             int64_t packed_stride_words, int32_t* dev_status, void* stream)
 {
     const int rc = dq_check_common(L, M);
     if (rc != DQ_OK) return rc;
@@ -682,8 +683,8 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
         // holds: the two separate passes give the same result
         const int r1 = dq_bucket_norms(L, dev_grads, worker_stride_elems, M, dev_norms, dev_status, stream);
         if (r1 != DQ_OK) return r1;
-        return dq_quantize_pack(L, dev_grads, worker_stride_elems, M, dev_norms, dev_b, seed, step, dev_packed,
-                                packed_stride_words, dev_status, stream);
+        return dq_quantize_pack_worker(L, dev_grads, worker_stride_elems, M, dev_norms, dev_b, seed, step, first_worker,
+                                       dev_packed, packed_stride_words, dev_status, stream);
     }
 
     FusedArgs a;
@@ -695,6 +696,7 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
     a.status = dev_status;
     a.keys = make_philox_keys(seed);
     a.step = step;
+    a.worker0 = first_worker;
     a.M = M;
     a.one_bits = 0x3F800040u;
     a.gpb_shift = 0;
@@ -744,4 +746,13 @@ extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_gra
     }
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+extern "C" int dq_norms_quantize_pack(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
+                                      int32_t M, const int32_t* dev_b, uint64_t seed, uint32_t step,
+                                      float* dev_norms, uint32_t* dev_packed, int64_t packed_stride_words,
+                                      int32_t* dev_status, void* stream)
+{
+    return dq_norms_quantize_pack_worker(L, dev_grads, worker_stride_elems, M, dev_b, seed, step, 0u, dev_norms,
+                                         dev_packed, packed_stride_words, dev_status, stream);
 }

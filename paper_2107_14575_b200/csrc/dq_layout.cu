@@ -116,6 +116,56 @@ extern "C" int dq_layout_bucket(const dq_layout_t* L, int64_t k, int64_t* start,
     return DQ_OK;
 }
 
+// Balanced contiguous ranges of whole buckets: bound j is the first bucket whose start lies at or
+// beyond j / n_shards of the padded buffer (so shards carry nearly equal numbers of elements).
+extern "C" int dq_layout_shard_bounds(const dq_layout_t* L, int32_t n_shards, int64_t* bounds)
+{
+    if (!L || !bounds || n_shards < 1) return DQ_ERR_ARG;
+    bounds[0] = 0;
+    int64_t k = 0;
+    for (int32_t j = 1; j < n_shards; ++j) {
+        const int64_t target = L->padded * j / n_shards;
+        while (k < L->nb) {
+            int64_t start = 0, len = 0;
+            dq_layout_bucket(L, k, &start, &len);
+            if (start >= target) break;
+            ++k;
+        }
+        bounds[j] = k;
+    }
+    bounds[n_shards] = L->nb;
+    return DQ_OK;
+}
+
+// Buckets [k0, k1) as a layout of their own.  Its tensors are the pieces of the parent's tensors
+// that the range covers: every piece but a tensor's last is a whole number of buckets (a multiple
+// of 32 elements), so the pieces sit in the slice's padded buffer exactly as they sit in the
+// parent's, first_elem elements further on.
+extern "C" int dq_layout_slice(const dq_layout_t* L, int64_t k0, int64_t k1, dq_layout_t** out, int64_t* first_elem)
+{
+    if (!L || !out) return DQ_ERR_ARG;
+    if (k0 < 0 || k1 > L->nb || k0 >= k1) return DQ_ERR_RANGE;
+    const int32_t n1 = L->n_seg + 1;
+    std::vector<int64_t> pieces;
+    int64_t first = -1;
+    for (int32_t i = 0; i < L->n_seg; ++i) {
+        const int64_t b0 = L->table[n1 + i], b1 = L->table[n1 + i + 1];      // this tensor's buckets
+        const int64_t lo = (k0 > b0 ? k0 : b0), hi = (k1 < b1 ? k1 : b1);
+        if (lo >= hi) continue;
+        const int64_t e0 = (lo - b0) * L->bucket;
+        int64_t e1 = (hi - b0) * L->bucket;
+        if (e1 > L->seg_elems[i]) e1 = L->seg_elems[i];
+        if (first < 0) first = L->seg_offset[i] + e0;
+        pieces.push_back(e1 - e0);
+    }
+    if (pieces.empty()) return DQ_ERR_RANGE;
+    const int rc = dq_layout_create_ex(pieces.data(), (int32_t)pieces.size(),
+                                       L->whole_tensor ? DQ_BUCKET_WHOLE_TENSOR : L->bucket, L->norm, out);
+    if (rc != DQ_OK) return rc;
+    if (first_elem) *first_elem = first;
+    return DQ_OK;
+}
+
 extern "C" size_t dq_layout_table_bytes(const dq_layout_t* L)
 {
     if (!L || L->n_seg == 1) return 0;

@@ -52,6 +52,7 @@ struct QuantizeArgs {
     int32_t* status;
     PhiloxKeys keys;
     uint32_t step;
+    uint32_t worker0;             // worker m of the call draws the uniforms of worker worker0 + m
     int32_t M;
     int32_t map_has_worker_dim;   // 0 when all workers read the same buffer (stride 0)
     uint32_t div_magic;           // groups_per_bucket: division by multiply-shift, or by shift if a power of two
@@ -161,7 +162,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
             encode_block<B, C>(acc, cur,                                                                        \
                                *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C)) ^ sw) << 4)),      \
                                *reinterpret_cast<const float4*>(row + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)),  \
-                               inv, q0 + (C), (uint32_t)m, a.step, a.keys, a.one_bits);
+                               inv, q0 + (C), (uint32_t)m + a.worker0, a.step, a.keys, a.one_bits);
             DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
 #undef DQ_BLOCK
         }
@@ -245,11 +246,11 @@ size_t smem_bytes(int n_seg)
 
 }  // namespace
 
-extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
-                                int32_t M, const float* dev_norms, const int32_t* dev_b,
-                                uint64_t seed, uint32_t step,
-                                uint32_t* dev_packed, int64_t packed_stride_words,
-                                int32_t* dev_status, void* stream)
+extern "C" int dq_quantize_pack_worker(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
+                                       int32_t M, const float* dev_norms, const int32_t* dev_b,
+                                       uint64_t seed, uint32_t step, uint32_t first_worker,
+                                       uint32_t* dev_packed, int64_t packed_stride_words,
+                                       int32_t* dev_status, void* stream)
 {
     const int rc = dq_check_common(L, M);
     if (rc != DQ_OK) return rc;
@@ -270,6 +271,7 @@ extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, in
     a.status = dev_status;
     a.keys = make_philox_keys(seed);
     a.step = step;
+    a.worker0 = first_worker;
     a.M = M;
     a.one_bits = 0x3F800040u;
     a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
@@ -306,4 +308,14 @@ extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, in
     quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+extern "C" int dq_quantize_pack(const dq_layout_t* L, const float* dev_grads, int64_t worker_stride_elems,
+                                int32_t M, const float* dev_norms, const int32_t* dev_b,
+                                uint64_t seed, uint32_t step,
+                                uint32_t* dev_packed, int64_t packed_stride_words,
+                                int32_t* dev_status, void* stream)
+{
+    return dq_quantize_pack_worker(L, dev_grads, worker_stride_elems, M, dev_norms, dev_b, seed, step, 0u, dev_packed,
+                                   packed_stride_words, dev_status, stream);
 }

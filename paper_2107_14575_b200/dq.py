@@ -23,10 +23,10 @@ BUCKET_WHOLE_TENSOR = 0            # DQ_BUCKET_WHOLE_TENSOR: one norm per tensor
 SYMBOLS = [
     "dq_layout_create", "dq_layout_create_ex", "dq_layout_norm", "dq_layout_whole_tensor", "dq_layout_destroy", "dq_layout_num_segments", "dq_layout_padded_elems",
     "dq_layout_seg_offset", "dq_layout_num_buckets", "dq_layout_packed_words", "dq_layout_bucket",
-    "dq_layout_table_bytes", "dq_layout_bind_device_table",
+    "dq_layout_shard_bounds", "dq_layout_slice", "dq_layout_table_bytes", "dq_layout_bind_device_table",
     "dq_bucket_norms", "dq_tensor_norms_scratch_bytes", "dq_tensor_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
     "dq_choose_bits_noalloc_max_norms", "dq_choose_bits_noalloc",
-    "dq_quantize_pack", "dq_norms_quantize_pack", "dq_unpack_dequant_average",
+    "dq_quantize_pack", "dq_quantize_pack_worker", "dq_norms_quantize_pack", "dq_norms_quantize_pack_worker", "dq_unpack_dequant_average",
     "dq_unpack_average_update", "dq_status_string",
 ]
 
@@ -86,6 +86,10 @@ def lib():
         L.dq_layout_packed_words.argtypes = [vp, i32]
         L.dq_layout_bucket.restype = C.c_int
         L.dq_layout_bucket.argtypes = [vp, i64, C.POINTER(i64), C.POINTER(i64)]
+        L.dq_layout_shard_bounds.restype = C.c_int
+        L.dq_layout_shard_bounds.argtypes = [vp, i32, C.POINTER(i64)]
+        L.dq_layout_slice.restype = C.c_int
+        L.dq_layout_slice.argtypes = [vp, i64, i64, C.POINTER(vp), C.POINTER(i64)]
         L.dq_layout_table_bytes.restype = sz
         L.dq_layout_table_bytes.argtypes = [vp]
         L.dq_layout_bind_device_table.restype = C.c_int
@@ -106,6 +110,10 @@ def lib():
         L.dq_choose_bits_noalloc.argtypes = [vp, vp, i32, C.POINTER(Rule), vp, vp, vp]
         L.dq_quantize_pack.restype = C.c_int
         L.dq_quantize_pack.argtypes = [vp, vp, i64, i32, vp, vp, u64, u32, vp, i64, vp, vp]
+        L.dq_quantize_pack_worker.restype = C.c_int
+        L.dq_quantize_pack_worker.argtypes = [vp, vp, i64, i32, vp, vp, u64, u32, u32, vp, i64, vp, vp]
+        L.dq_norms_quantize_pack_worker.restype = C.c_int
+        L.dq_norms_quantize_pack_worker.argtypes = [vp, vp, i64, i32, vp, u64, u32, u32, vp, vp, i64, vp, vp]
         L.dq_norms_quantize_pack.restype = C.c_int
         L.dq_norms_quantize_pack.argtypes = [vp, vp, i64, i32, vp, u64, u32, vp, vp, i64, vp, vp]
         L.dq_unpack_dequant_average.restype = C.c_int
@@ -151,12 +159,15 @@ class Layout:
     ``bucket = BUCKET_WHOLE_TENSOR`` gives one norm per tensor (Eq. 5 as written);
     ``norm`` picks the member of the l_p family the norm calls compute."""
 
-    def __init__(self, seg_elems: Sequence[int], bucket: int, norm: int = NORM_L2):
-        arr = (C.c_int64 * len(seg_elems))(*[int(x) for x in seg_elems])
+    def __init__(self, seg_elems: Sequence[int], bucket: int, norm: int = NORM_L2, _handle=None):
         h = C.c_void_p()
-        if norm == NORM_L2 and bucket != BUCKET_WHOLE_TENSOR:
+        if _handle is not None:
+            h = _handle                     # a layout the library created (dq_layout_slice)
+        elif norm == NORM_L2 and bucket != BUCKET_WHOLE_TENSOR:
+            arr = (C.c_int64 * len(seg_elems))(*[int(x) for x in seg_elems])
             _check(lib().dq_layout_create(arr, len(seg_elems), int(bucket), C.byref(h)), "dq_layout_create")
         else:
+            arr = (C.c_int64 * len(seg_elems))(*[int(x) for x in seg_elems])
             _check(lib().dq_layout_create_ex(arr, len(seg_elems), int(bucket), int(norm), C.byref(h)),
                    "dq_layout_create_ex")
         self._h = h
@@ -188,6 +199,19 @@ class Layout:
 
     def table_bytes(self) -> int:
         return int(lib().dq_layout_table_bytes(self._h))
+
+    def shard_bounds(self, n_shards: int):
+        """First bucket of each of ``n_shards`` contiguous ranges, plus ``nb`` (``dq_layout_shard_bounds``)."""
+        out = (C.c_int64 * (int(n_shards) + 1))()
+        _check(lib().dq_layout_shard_bounds(self._h, int(n_shards), out), "dq_layout_shard_bounds")
+        return [int(x) for x in out]
+
+    def slice(self, k0: int, k1: int):
+        """Buckets [k0, k1) as a layout of their own and where it starts in this padded buffer
+        (``dq_layout_slice``); returns (Layout, first_elem)."""
+        h, first = C.c_void_p(), C.c_int64()
+        _check(lib().dq_layout_slice(self._h, int(k0), int(k1), C.byref(h), C.byref(first)), "dq_layout_slice")
+        return Layout(None, self.bucket, self.norm, _handle=h), int(first.value)
 
     def bind_device_table(self, dev_buf, nbytes: Optional[int] = None, stream=None) -> None:
         """dev_buf: a torch uint8/int32 CUDA tensor (kept alive by this object) or a raw address."""
@@ -245,6 +269,24 @@ def quantize_pack(layout: Layout, grads, worker_stride_elems: int, M: int, norms
     _check(lib().dq_quantize_pack(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(norms),
                                   _ptr(dev_b), int(seed) & (2 ** 64 - 1), int(step) & 0xFFFFFFFF, _ptr(packed),
                                   int(packed_stride_words), _ptr(status), _stream(stream)), "dq_quantize_pack")
+
+
+def quantize_pack_worker(layout: Layout, grads, worker_stride_elems: int, M: int, norms, dev_b, seed: int, step: int,
+                         first_worker: int, packed, packed_stride_words: int, status, stream=None) -> None:
+    _check(lib().dq_quantize_pack_worker(layout.handle, _ptr(grads), int(worker_stride_elems), int(M), _ptr(norms),
+                                         _ptr(dev_b), int(seed) & (2 ** 64 - 1), int(step) & 0xFFFFFFFF,
+                                         int(first_worker) & 0xFFFFFFFF, _ptr(packed), int(packed_stride_words),
+                                         _ptr(status), _stream(stream)), "dq_quantize_pack_worker")
+
+
+def norms_quantize_pack_worker(layout: Layout, grads, worker_stride_elems: int, M: int, dev_b, seed: int, step: int,
+                               first_worker: int, norms, packed, packed_stride_words: int, status,
+                               stream=None) -> None:
+    _check(lib().dq_norms_quantize_pack_worker(layout.handle, _ptr(grads), int(worker_stride_elems), int(M),
+                                               _ptr(dev_b), int(seed) & (2 ** 64 - 1), int(step) & 0xFFFFFFFF,
+                                               int(first_worker) & 0xFFFFFFFF, _ptr(norms), _ptr(packed),
+                                               int(packed_stride_words), _ptr(status), _stream(stream)),
+           "dq_norms_quantize_pack_worker")
 
 
 def norms_quantize_pack(layout: Layout, grads, worker_stride_elems: int, M: int, dev_b, seed: int, step: int,

@@ -156,3 +156,14 @@ def test_norm_family_layouts(dqlib):
     assert L.dq_tensor_norms(one.handle, A, 10016, 2, A, 0, need, A, 0) == dqlib.ERR_ARG
     assert L.dq_tensor_norms(one.handle, A, 10016, 2, A, A + 4, need, A, 0) == dqlib.ERR_ALIGN
     assert L.dq_tensor_norms(one.handle, A, 10016, 2, A, A, need - 1, A, 0) == dqlib.ERR_RANGE
+
+
+def test_worker_offset_calls_check_their_arguments(dqlib):
+    lay = dqlib.Layout([1000], 64)
+    A = 0x7f0000001000
+    L = dqlib.lib()
+    h = lay.handle
+    assert L.dq_quantize_pack_worker(h, A, 1024, 1, A, 0, 0, 0, 3, A, 1024, A, 0) == dqlib.ERR_ARG
+    assert L.dq_quantize_pack_worker(h, A, 1024, 1, A, A, 0, 0, 3, A, 1022, A, 0) == dqlib.ERR_ALIGN
+    assert L.dq_norms_quantize_pack_worker(h, A, 1024, 1, 0, 0, 0, 3, A, A, 1024, A, 0) == dqlib.ERR_ARG
+    assert L.dq_norms_quantize_pack_worker(h, A, 1024, 1, A, 0, 0, 3, A, A, 16, A, 0) == dqlib.ERR_RANGE
