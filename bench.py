@@ -53,7 +53,7 @@ def _peaks():
 KERNEL_SOURCES = {
     "norms_quantize_pack": ["dq_fused.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
     "quantize_pack": ["dq_quantize.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
-    "bucket_norms": ["dq_norms.cu", "dq_tma.cuh", "dq_common.cuh"],
+    "bucket_norms": ["dq_norms.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
     "unpack_dequant_average": ["dq_unpack.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
     "choose_bits": ["dq_bits.cu", "dq_common.cuh"],
 }

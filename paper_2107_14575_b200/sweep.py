@@ -3,7 +3,8 @@
     python -m paper_2107_14575_b200.sweep [--quick] [--out sweep.json]
 
 Sizes d = 2^20 ... 2^30 at M = 1 and d = 2^26 at M = 32, bit widths 1..16 at bucket 512
-and {2, 4, 8, 16} at buckets 128 and 4096.  Every kernel is timed alone with CUDA events
+and {2, 4, 8, 16} at buckets 128 and 4096; at bucket 512 also the l_inf norms (alone and fused
+with the quantizer) and one norm per tensor (``dq_tensor_norms``).  Every kernel is timed alone with CUDA events
 (3 warm-up launches, median of 8-20), over rotating inputs that together exceed the L2,
 and once more as a train of launches between two events (the sustained rate: launch latency
 overlaps the previous launch).  Each row gives both times, GB/s of algorithmic bytes (norms 4, quantizers 4 + b/8 per
@@ -73,7 +74,25 @@ def run(quick: bool = False):
             torch.cuda.synchronize()
             if rnd.read_status() != 0:
                 raise RuntimeError("device status %d" % rnd.read_status())
-            del gs, rnd
+            del rnd
+            if bucket == 512:
+                # the other members of the norm family on the same inputs: l_inf buckets, one norm per tensor
+                for norm, tag in ((dq.NORM_LINF, "_linf"),):
+                    alt = Round([d], bucket, M, norm=norm)
+                    add("bucket_norms" + tag, 0, *_time(lambda i: alt.norms_(gs[i % nbuf]), reps), 4.0 * M * D32)
+                    for b in (2, 4, 8, 16):
+                        alt.bits_(dq.Rule.fixed(b))
+                        add("norms_quantize_pack" + tag, b, *_time(lambda i: alt.norms_quantize_(gs[i % nbuf], 1, i), reps),
+                            (4.0 + b / 8.0) * M * D32)
+                    del alt
+                for norm, tag in ((dq.NORM_L2, ""), (dq.NORM_LINF, "_linf")):
+                    whole = Round([d], dq.BUCKET_WHOLE_TENSOR, M, max_bits=1, norm=norm)
+                    add("tensor_norms" + tag, 0, *_time(lambda i: whole.norms_(gs[i % nbuf]), reps), 4.0 * M * D32)
+                    torch.cuda.synchronize()
+                    if whole.read_status() != 0:
+                        raise RuntimeError("device status %d" % whole.read_status())
+                    del whole
+            del gs
             torch.cuda.empty_cache()
     return rows
 
