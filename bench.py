@@ -353,6 +353,7 @@ def run_cuda(args) -> dict:
         "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": (tr or {}).get("bytes_per_launch"),
         "peak_source": peak_src + "; of measured" if peak_src.startswith("measured") else peak_src + "; of fallback",
         "algorithmic_bytes_per_launch": kernels[dominant]["algorithmic_bytes_per_launch"], "mean_b": round(mean_b, 3),
+        "frac_of_nominal_8tbs": round(kernels[dominant]["achieved_gbs"] / 8000.0, 4),
         "kernels": kernels,
     }
     # The events that bracket a single launch also see its launch latency (the stream drains at
@@ -406,6 +407,9 @@ def run_cuda(args) -> dict:
                                     % (max(1, K // 12), len(range(0, K, max(1, K // 12)))),
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "roofline": roofline,
+        # what the workers would put on the wire per step (Eq. 7: d * b bits per worker, plus the fp32 norms)
+        "wire": {"bytes_per_step": M * (w.d * mean_b / 8.0 + 4.0 * L.nb), "fp32_bytes_per_step": 4.0 * M * w.d,
+                 "ratio": round((w.d * mean_b / 8.0 + 4.0 * L.nb) / (4.0 * w.d), 4)},
         "four_call_order": four, "with_parameter_update": upd,
         "host_submit_ms_per_step": round(host_ms["algorithm1"], 5),
     }
