@@ -43,6 +43,7 @@ __global__ void __launch_bounds__(kSumThreads, 8)
 norm_square_partials(const float* __restrict__ norms, const int64_t n, double* __restrict__ partial)
 {
     __shared__ double sh[kSumThreads / 32];
+    grid_dependency_wait();
     constexpr int kPer = kChunk / kSumThreads;     // 64 norms per thread, fetched 32 at a time
     constexpr int kBatch = 32;
     const int64_t base = (int64_t)blockIdx.x * kChunk + threadIdx.x;
@@ -71,6 +72,7 @@ apply_rule(const double* __restrict__ partial, const int npartial, const int M, 
            int32_t* __restrict__ dev_b, int32_t* __restrict__ status)
 {
     __shared__ double sh[kThreads / 32];
+    grid_dependency_wait();
     double acc = 0.0;
     for (int i = threadIdx.x; i < npartial; i += kThreads) acc += partial[i];
     const double sum = block_sum<kThreads>(acc, sh);
@@ -134,10 +136,10 @@ extern "C" int dq_choose_bits(const dq_layout_t* L, const float* dev_norms, int3
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     double* partial = static_cast<double*>(dev_scratch);
     if (rule->fixed_b == 0) {
-        norm_square_partials<<<(unsigned)chunks, kSumThreads, 0, st>>>(dev_norms, n, partial);
+        dq_launch(norm_square_partials, dim3((unsigned)chunks), dim3(kSumThreads), 0, st, dev_norms, n, partial);
         if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     }
-    apply_rule<<<1, kThreads, 0, st>>>(partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
+    dq_launch(apply_rule, dim3(1), dim3(kThreads), 0, st, partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
                                       rule->b_min, rule->b_max, rule->fixed_b, dev_b, dev_status);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
@@ -218,10 +220,10 @@ extern "C" int dq_choose_bits_noalloc(const dq_layout_t* L, const float* dev_nor
     // Nothing in the array has to start at zero: the first kernel writes every entry the
     // second one reads, so whatever an earlier call left behind is overwritten, never used.
     if (rule->fixed_b == 0) {
-        norm_square_partials<<<(unsigned)chunks, kSumThreads, 0, st>>>(dev_norms, n, partial);
+        dq_launch(norm_square_partials, dim3((unsigned)chunks), dim3(kSumThreads), 0, st, dev_norms, n, partial);
         if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     }
-    apply_rule<<<1, kThreads, 0, st>>>(partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
+    dq_launch(apply_rule, dim3(1), dim3(kThreads), 0, st, partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
                                       rule->b_min, rule->b_max, rule->fixed_b, dev_b, dev_status);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;

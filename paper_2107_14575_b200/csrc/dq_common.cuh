@@ -6,6 +6,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
 #include <vector>
 
 #include "dq.h"
@@ -82,6 +83,29 @@ int dq_check_common(const dq_layout* L, int32_t M);   // DQ_OK / DQ_ERR_*
 int dq_sm_count();                                    // SMs of the current device (cached per device)
 
 #ifdef __CUDACC__
+
+// Every kernel of the library is launched with programmatic stream serialization and begins
+// with grid_dependency_wait(): the grid may be set up while the previous kernel of the stream
+// is still draining (which hides the launch latency between the calls of a step), and the wait
+// returns once that kernel has completed and its writes are visible, so nothing is read or
+// written early.  No kernel signals its dependents ahead of its own end.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline void dq_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    (void)cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);   // the caller reads cudaGetLastError()
+}
 
 // Index of the last entry of starts[0..n] (n + 1 entries, non-decreasing) that is <= x.
 // Tensors of zero size repeat a start; the last repeat is the non-empty one.

@@ -587,6 +587,7 @@ template <int P>
 __global__ void __launch_bounds__(kThreads, 6)
 norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
+    grid_dependency_wait();
     const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
@@ -625,6 +626,7 @@ template <int P>
 __global__ void __launch_bounds__(kThreads, 5)
 norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
+    grid_dependency_wait();
     const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
@@ -728,7 +730,7 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
         const int64_t warp_tiles = (int64_t)M * ((L->nb + R - 1) / R);
         int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
         if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
-        kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
+        dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
     } else {
         const size_t smem_need = (size_t)kTblOffset + tbl_bytes;
         const auto kernel = (L->norm == DQ_NORM_LINF) ? norms_quantize_pack_kernel<DQ_NORM_LINF>
@@ -742,7 +744,7 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
         const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
         int64_t blocks = (int64_t)dq_sm_count() * 5;   // five 42 KB CTAs per SM
         if (blocks > tiles) blocks = tiles;
-        kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
+        dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
     }
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;

@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(kThreads)
 bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const int64_t worker_stride,
                     float* __restrict__ norms, int32_t* __restrict__ status)
 {
+    grid_dependency_wait();
     constexpr int kTeamsPerWarp = 32 / LANES;
     constexpr int kChunk = kRun * kTeamsPerWarp;          // buckets per run
     const int lane = threadIdx.x % LANES;
@@ -109,6 +110,7 @@ bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, co
                          float* __restrict__ norms, int32_t* __restrict__ status)
 {
     extern __shared__ int32_t tbl_s[];
+    grid_dependency_wait();
     const int lane = threadIdx.x & 31;
     const int m = blockIdx.y;
     const float4* gw4 = reinterpret_cast<const float4*>(grads + (int64_t)m * worker_stride);
@@ -253,6 +255,7 @@ template <int P, bool RAW>
 __global__ void __launch_bounds__(kTmaThreads)
 bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_constant__ CUtensorMap map)
 {
+    grid_dependency_wait();
     const int tid = threadIdx.x;
     if (tma::smem_addr(smem) & 1023u) {
         if (tid == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
@@ -403,6 +406,7 @@ tensor_norms_join_kernel(const int32_t n_seg, const int32_t* __restrict__ piece0
 {
     __shared__ double part_d[kJoinThreads / 32];
     __shared__ float part_f[kJoinThreads / 32];
+    grid_dependency_wait();
     const int seg = blockIdx.x, m = blockIdx.y;
     int c0 = 0, c1 = n_pieces, k = 0;
     if (n_seg > 1) {
@@ -475,7 +479,7 @@ int launch_tma(const dq_layout_t* L, const LayoutView& v, const float* dev_grads
     const int64_t tiles = (int64_t)M * ((v.nb + R - 1) / R);
     int64_t blocks = (int64_t)dq_sm_count() * 3;    // three 65 KB CTAs per SM
     if (blocks > tiles) blocks = tiles;
-    bucket_norms_tma_kernel<P, RAW><<<(unsigned)blocks, kTmaThreads, smem_need, st>>>(a, map);
+    dq_launch(bucket_norms_tma_kernel<P, RAW>, dim3((unsigned)blocks), dim3(kTmaThreads), smem_need, st, a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
@@ -497,12 +501,12 @@ int launch_plain(const dq_layout_t* L, const LayoutView& v, const float* dev_gra
     const dim3 grid((unsigned)bx, (unsigned)M);
     if (lanes == 32) {
         const size_t smem = (L->n_seg > 1 && (size_t)3 * (L->n_seg + 1) * 4 <= 12 * 1024) ? (size_t)3 * (L->n_seg + 1) * 4 : 0;
-        bucket_norms_warp_kernel<P><<<grid, kThreads, smem, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+        dq_launch(bucket_norms_warp_kernel<P>, grid, dim3(kThreads), smem, st, v, dev_grads, worker_stride_elems, dev_norms, dev_status);
     }
     else if (lanes == 16)
-        bucket_norms_kernel<16, P><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+        dq_launch(bucket_norms_kernel<16, P>, grid, dim3(kThreads), 0, st, v, dev_grads, worker_stride_elems, dev_norms, dev_status);
     else
-        bucket_norms_kernel<8, P><<<grid, kThreads, 0, st>>>(v, dev_grads, worker_stride_elems, dev_norms, dev_status);
+        dq_launch(bucket_norms_kernel<8, P>, grid, dim3(kThreads), 0, st, v, dev_grads, worker_stride_elems, dev_norms, dev_status);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
@@ -571,11 +575,11 @@ extern "C" int dq_tensor_norms(const dq_layout_t* L, const float* dev_grads, int
     const int32_t* bucket0 = L->n_seg > 1 ? L->dev_table + n1 : nullptr;
     const dim3 grid((unsigned)L->n_seg, (unsigned)M);
     if (linf)
-        tensor_norms_join_kernel<DQ_NORM_LINF><<<grid, kJoinThreads, 0, st>>>(L->n_seg, piece0, bucket0, (int32_t)L->n_pieces,
-                                                                             (int32_t)L->nb, partial, dev_norms, dev_status);
+        dq_launch(tensor_norms_join_kernel<DQ_NORM_LINF>, grid, dim3(kJoinThreads), 0, st, L->n_seg, piece0, bucket0,
+                  (int32_t)L->n_pieces, (int32_t)L->nb, partial, dev_norms, dev_status);
     else
-        tensor_norms_join_kernel<DQ_NORM_L2><<<grid, kJoinThreads, 0, st>>>(L->n_seg, piece0, bucket0, (int32_t)L->n_pieces,
-                                                                           (int32_t)L->nb, partial, dev_norms, dev_status);
+        dq_launch(tensor_norms_join_kernel<DQ_NORM_L2>, grid, dim3(kJoinThreads), 0, st, L->n_seg, piece0, bucket0,
+                  (int32_t)L->n_pieces, (int32_t)L->nb, partial, dev_norms, dev_status);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }

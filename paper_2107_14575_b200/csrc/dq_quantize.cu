@@ -203,6 +203,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
 __global__ void __launch_bounds__(kThreads, 6)
 quantize_pack_kernel(const __grid_constant__ QuantizeArgs a, const __grid_constant__ CUtensorMap map)
 {
+    grid_dependency_wait();
     const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {           // the swizzled tiles need a 1024-byte aligned base
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
@@ -305,7 +306,7 @@ extern "C" int dq_quantize_pack_worker(const dq_layout_t* L, const float* dev_gr
     const int64_t warp_tiles = (int64_t)M * ((a.v.total_groups + 31) / 32);
     int64_t blocks = (int64_t)dq_sm_count() * 6;       // six 33 KB CTAs fit one SM
     if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
-    quantize_pack_kernel<<<(unsigned)blocks, kThreads, smem_need, static_cast<cudaStream_t>(stream)>>>(a, map);
+    dq_launch(quantize_pack_kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }

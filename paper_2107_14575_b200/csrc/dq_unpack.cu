@@ -383,6 +383,7 @@ template <bool UPDATE>
 __global__ void __launch_bounds__(kBlock, 4)
 unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_constant__ CUtensorMap out_map)
 {
+    grid_dependency_wait();
     const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
     if (tma::smem_addr(smem) & 1023u) {           // the swizzled tile needs a 1024-byte aligned base
         if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
@@ -483,7 +484,8 @@ int launch_average(const dq_layout_t* L, const uint32_t* dev_packed, int64_t pac
     const int64_t tiles = ((int64_t)a.v.total_groups + kThreads - 1) / kThreads;
     int64_t blocks = (int64_t)dq_sm_count() * 4;       // four 53 KB CTAs per SM
     if (blocks > tiles) blocks = tiles;
-    unpack_average_kernel<UPDATE><<<(unsigned)blocks, kBlock, smem_need, static_cast<cudaStream_t>(stream)>>>(a, out_map);
+    dq_launch(unpack_average_kernel<UPDATE>, dim3((unsigned)blocks), dim3(kBlock), smem_need, static_cast<cudaStream_t>(stream), a,
+              out_map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
