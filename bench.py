@@ -428,6 +428,7 @@ def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> d
     host = [pool[p].cpu().pin_memory() for p in range(2)]
     for i in range(2):
         rnd.step_host(host[i % 2], rule_for(i + 1), SEED, i)
+    rnd.sync_host()
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -435,7 +436,9 @@ def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> d
     s2.record()
     for i in range(Ke):
         res = rnd.step_host(host[i % 2], rule_for(i + 1), SEED, i)
+    rnd.join_host()                        # the last download ends inside the timed region
     e2.record()
+    rnd.sync_host()
     torch.cuda.synchronize()
     checksum = float(res[:1024].double().abs().sum())        # the result is read on the host
     ms2 = s2.elapsed_time(e2)

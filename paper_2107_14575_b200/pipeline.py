@@ -152,16 +152,52 @@ class Round:
     def step_host(self, host_grads: torch.Tensor, next_rule: dq.Rule, seed: int, step: int) -> torch.Tensor:
         """``step_fused`` on pinned host gradients [M, stride]; returns a pinned host tensor [D32].
 
-        Copies the gradients to the device, runs the round and copies the
-        average back, all on the current stream; the caller synchronises.
+        The gradients travel to the device on a copy stream, the round runs on the current
+        stream and the average travels back on a second copy stream, with two device input
+        buffers and two host output buffers used in turn: in a loop of calls the upload of
+        step i + 1 runs beside the round and the download of step i (the link is full duplex).
+        The caller synchronises before it reads the returned tensor, leaves ``host_grads``
+        untouched until then, and finds the result of a call intact until the call after next.
         """
         if self._dev_in is None:
-            self._dev_in = torch.empty((self.M, self.stride), dtype=torch.float32, device=self.device)
-            self._host_out = torch.empty(self.layout.D32, dtype=torch.float32).pin_memory()
-        self._dev_in.copy_(host_grads, non_blocking=True)
-        self.step_fused(self._dev_in, next_rule, seed, step)
-        self._host_out.copy_(self.out, non_blocking=True)
-        return self._host_out
+            self._dev_in = [torch.empty((self.M, self.stride), dtype=torch.float32, device=self.device) for _ in range(2)]
+            self._host_out = [torch.empty(self.layout.D32, dtype=torch.float32).pin_memory() for _ in range(2)]
+            self._s_in = torch.cuda.Stream(self.device)
+            self._s_out = torch.cuda.Stream(self.device)
+            self._ev_in = [torch.cuda.Event() for _ in range(2)]       # upload into buffer i has landed
+            self._ev_used = [torch.cuda.Event() for _ in range(2)]     # the round that read buffer i is done
+            self._ev_avg = torch.cuda.Event()                           # this round's average is in self.out
+            self._ev_out = torch.cuda.Event()                           # the last download has left self.out
+            self._host_calls = 0
+        i = self._host_calls % 2
+        self._host_calls += 1
+        main = torch.cuda.current_stream(self.device)
+        self._s_in.wait_event(self._ev_used[i])          # (a wait on an event never recorded returns at once)
+        with torch.cuda.stream(self._s_in):
+            self._dev_in[i].copy_(host_grads, non_blocking=True)
+            self._ev_in[i].record(self._s_in)
+        main.wait_event(self._ev_in[i])
+        main.wait_event(self._ev_out)                    # the previous average has been read out of self.out
+        self.step_fused(self._dev_in[i], next_rule, seed, step)
+        self._ev_used[i].record(main)
+        self._ev_avg.record(main)
+        self._s_out.wait_event(self._ev_avg)
+        with torch.cuda.stream(self._s_out):
+            self._host_out[i].copy_(self.out, non_blocking=True)
+            self._ev_out.record(self._s_out)
+        return self._host_out[i]
+
+    def join_host(self) -> None:
+        """Makes the current stream wait (on the device) for the last download ``step_host`` queued."""
+        if self._dev_in is not None:
+            torch.cuda.current_stream(self.device).wait_event(self._ev_out)
+
+    def sync_host(self) -> None:
+        """Waits for everything ``step_host`` has queued (its copy streams included)."""
+        if self._dev_in is not None:
+            self._s_in.synchronize()
+            self._s_out.synchronize()
+        torch.cuda.current_stream(self.device).synchronize()
 
     def bits(self) -> int:
         """b chosen by the last bits_ call (synchronises)."""
