@@ -122,16 +122,16 @@ extern "C" int dq_layout_shard_bounds(const dq_layout_t* L, int32_t n_shards, in
 {
     if (!L || !bounds || n_shards < 1) return DQ_ERR_ARG;
     bounds[0] = 0;
-    int64_t k = 0;
     for (int32_t j = 1; j < n_shards; ++j) {
         const int64_t target = L->padded * j / n_shards;
-        while (k < L->nb) {
+        int64_t lo = bounds[j - 1], hi = L->nb;          // first bucket in [lo, nb] that starts at or after target
+        while (lo < hi) {
+            const int64_t mid = lo + (hi - lo) / 2;
             int64_t start = 0, len = 0;
-            dq_layout_bucket(L, k, &start, &len);
-            if (start >= target) break;
-            ++k;
+            dq_layout_bucket(L, mid, &start, &len);
+            if (start >= target) hi = mid; else lo = mid + 1;
         }
-        bounds[j] = k;
+        bounds[j] = lo;
     }
     bounds[n_shards] = L->nb;
     return DQ_OK;
