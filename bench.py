@@ -464,9 +464,21 @@ def _cpu_baseline(pool, w, eps_hat, alpha) -> dict:
         _oracle_round(oracle, np, w, ref, grads[steps % len(grads)], steps % w.T, eps_hat, alpha)
         dt += time.perf_counter() - t0
         steps += 1
-    return {"value": 4.0 * w.M * w.d * steps / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "%d full steps (all %d workers, all %d tensors, t = 0..%d), %.1f s"
-                      % (steps, w.M, len(w.segments), steps - 1, dt)}
+    out = {"value": 4.0 * w.M * w.d * steps / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": "%d full steps (all %d workers, all %d tensors, t = 0..%d), %.1f s"
+                     % (steps, w.M, len(w.segments), steps - 1, dt)}
+    # the same checker on one thread, on one worker's share of a step
+    import copy
+    w1 = copy.copy(w)
+    w1.M = 1
+    oracle.set_threads(1)
+    t0 = time.perf_counter()
+    _oracle_round(oracle, np, w1, ref, grads[0][:1], 0, eps_hat, alpha)
+    dt1 = time.perf_counter() - t0
+    oracle.set_threads(cores)
+    out["one_thread"] = {"value": 4.0 * w.d / dt1 / 1e9, "unit": UNIT, "cores": 1,
+                         "sample": "one step of one worker (all %d tensors), %.1f s" % (len(w.segments), dt1)}
+    return out
 
 
 def main():
