@@ -24,6 +24,12 @@
  *  - "dev" pointers are device pointers owned by the caller.  The library never
  *    allocates or frees device memory and never synchronises the host.
  *  - `stream` is a cudaStream_t passed as void* (NULL = legacy default stream).
+ *    Kernels are launched with programmatic stream serialization and start by
+ *    waiting for the previous kernel of the stream to complete: the usual
+ *    stream order holds for everything they read and write, whatever kernel
+ *    (the library's or the caller's) precedes them.  The calls of a round
+ *    (norms, bit rule with caller scratch, quantizer, average, update) can be
+ *    captured in a CUDA graph.
  *  - Return value: DQ_OK or a negative DQ_ERR_* for errors found on the host
  *    before anything is launched (nothing is written in that case).
  *  - Conditions only the device can see are OR-ed into *dev_status (DQ_STAT_*

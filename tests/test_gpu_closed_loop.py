@@ -27,8 +27,12 @@ def _lib(dqlib):
         pytest.fail("the gpu tests need a CUDA device")
 
 
-def test_quadratic_follows_theorem_3_and_the_error_budget():
-    d, bucket, M, lam, eta, T, b0 = 1 << 16, 512, 4, 1.0, 0.2, 30, 5
+@pytest.mark.parametrize("p,b0,x_first", [("l2", 5, 9.0), ("linf", 3, 2.0)])
+def test_quadratic_follows_theorem_3_and_the_error_budget(p, b0, x_first):
+    """l2: per-bucket l_2 norms, b = 5.  linf: the l_inf member of the family at b = 3 (its level
+    grid is ~sqrt(bucket) / 3.5 times finer, so a coarser b keeps the quantizer's share of F_T well
+    above the test's resolution); Lemma 1's variance formula is the same for both."""
+    d, bucket, M, lam, eta, T = 1 << 16, 512, 4, 1.0, 0.2, 30
     rho = 1.0 - eta * lam
     beta = rho * rho                                   # contraction of F per step: the alpha of Eq. 17
     rng = np.random.default_rng(2107)
@@ -37,11 +41,15 @@ def test_quadratic_follows_theorem_3_and_the_error_budget():
     xs = torch.from_numpy(x_star.astype(np.float32)).cuda()
     x = torch.from_numpy(x0.astype(np.float32)).cuda()
 
-    rnd = Round([d], bucket, M)
+    rnd = Round([d], bucket, M, norm=dq.NORM_L2 if p == "l2" else dq.NORM_LINF)
     g0 = lam * (x0 - x_star)
-    G0sq = float((g0 ** 2).sum())                      # (1/M) sum_m sum_k norm^2 with M identical workers
-    eps_hat = T * beta ** (T - 1) * G0sq / 9.0 ** 2    # Eq. 17: x = 9 at t = 0 and 9 / sqrt(alpha) = 11.25 when
-    #                                                     step t + 1 is sized from step t's norms: b = 5 (s = 15)
+    if p == "l2":
+        G0sq = float((g0 ** 2).sum())                  # (1/M) sum_m sum_k norm^2 with M identical workers
+    else:
+        G0sq = float((np.abs(g0).reshape(-1, bucket).max(axis=1) ** 2).sum())
+    # Eq. 17: x = x_first at t = 0 and x_first / sqrt(alpha) when step t + 1 is sized from step t's norms
+    # (9 -> 11.25: b = 5, s = 15; 2 -> 2.5: b = 3, s = 3)
+    eps_hat = T * beta ** (T - 1) * G0sq / x_first ** 2
     sched = schedule.BitSchedule(T, eps_hat, tau=1, alpha=beta, b0=b0)
     rnd.bits_(dq.Rule.fixed(b0))
 
