@@ -16,8 +16,9 @@
 // norm and the tile's words leave with 16-byte coalesced stores.
 //  * Buckets of up to 1024 elements (gpb <= 32): every WARP is a pipeline of its own
 //    over tiles of 32 / gpb buckets; no CTA barrier in the loop.
-//  * Larger buckets (up to 4096 elements): the CTA is the pipeline, tiles of
-//    128 / gpb buckets, partial sums of a bucket's warps meet in shared memory.
+//  * Buckets of 2048 elements: a warp takes a whole bucket through its two stages.
+//  * Buckets of 4096 elements: the CTA is the pipeline, tiles of 128 / gpb buckets,
+//    partial sums of a bucket's warps meet in shared memory.
 // HBM traffic: 4 + b/8 bytes per element.
 #include "dq_common.cuh"
 #include "dq_device.cuh"
@@ -621,6 +622,226 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
     }
 }
 
+// ---- buckets of 2048 elements: a warp takes a whole bucket through its two stages ------
+//
+// A bucket of 64 groups is two warp tiles.  The warp fetches them into its two stages, every
+// lane squares its row of each, the two halves are reduced by the same butterflies and added
+// in the same order as dq_bucket_norms does, and the rows are then encoded half by half: as
+// soon as a half has left for the packed stream, its stage is refilled with the matching half
+// of the warp's next bucket, so that the fetch runs beside the encoding of the other half.
+// Short buckets (a tensor's last) and padding take the same route with per-lane valid counts.
+template <int B, int P>
+__device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUtensorMap* map)
+{
+    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kWTblOffset);
+    constexpr int s = (1 << (B - 1)) - 1;
+    const float sf = (float)s;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n1 = a.v.n_seg + 1;
+    const int nb = a.v.nb;
+    constexpr int kBucket = 2048;
+    const int64_t total = (int64_t)a.M * nb;
+    const int64_t nwarps = (int64_t)gridDim.x * kWarps;
+    const int64_t gw = (int64_t)blockIdx.x * kWarps + warp;
+    const int64_t begin = gw * total / nwarps;
+    const int n_tiles = (int)((gw + 1) * total / nwarps - begin);
+    if (n_tiles <= 0) return;
+
+    int seg = 0;                                  // walking hint: buckets only move forward inside a worker
+    auto locate = [&](int k, int& g0, int& len) {
+        int local, n, gs;
+        if (a.v.n_seg == 1) {
+            local = k; n = a.v.seg0_elems; gs = 0;
+        } else {
+            while (k >= tbl_s[n1 + seg + 1]) ++seg;
+            local = k - tbl_s[n1 + seg];
+            n = tbl_s[2 * n1 + seg];
+            gs = tbl_s[seg];
+        }
+        g0 = gs + local * 64;
+        const int left = n - local * kBucket;
+        len = left < kBucket ? left : kBucket;
+    };
+    auto issue = [&](int st, int row0, int mm) {
+        tma::mbar_expect_tx(wbar(warp, st), kWTileBytes);
+        if (a.stream_reads)
+            tma::load_tile_3d_hint(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? mm : 0,
+                                   tma::policy_evict_first());
+        else
+            tma::load_tile_3d(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? mm : 0);
+    };
+
+    int m = (int)(begin / nb), k = (int)(begin - (int64_t)m * nb);
+    int g0, len;
+    locate(k, g0, len);
+    if (lane == 0) {
+        issue(0, g0, m);
+        if (len > 1024) issue(1, g0 + 32, m);
+    }
+    bool pend_a = true, pend_b = len > 1024;
+    uint32_t ph_a = 0, ph_b = 0;
+    bool timed_out = false, bad = false;
+    // byte offset of this lane's row inside a stage, swizzle phase folded in: chunk c sits at own ^ (c << 4)
+    const uint32_t own = (uint32_t)(lane * 128 + ((lane & 7) << 4));
+
+    // sum of squares (or maximum) of the lane's row of a stage, same operations and order as dq_bucket_norms
+    auto row_reduce = [&](const unsigned char* base, int valid) -> float {
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        if (valid == 32) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float4 x = *reinterpret_cast<const float4*>(base + (own ^ (uint32_t)(c << 4)));
+                a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
+            }
+        } else {
+            for (int e = 0; e < valid; ++e) {
+                const float x = *reinterpret_cast<const float*>(base + (own ^ (uint32_t)((e >> 2) << 4)) + ((e & 3) << 2));
+                a0 = take<P>(a0, x);
+            }
+        }
+        float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum = join<P>(sum, __shfl_xor_sync(0xffffffffu, sum, o));
+        return sum;
+    };
+    // encodes the lane's row of a stage against `inv`, stages the half's words in the stage itself and
+    // sends them to the packed stream; `row0` is the half's first group, `span` its number of groups
+    auto encode_half = [&](unsigned char* base, int row0, int valid, int span, float inv, int mm) {
+        uint32_t acc[B];
+        if (valid > 0) {
+            unsigned char* rowp = base + lane * 128;
+            const uint32_t sw = (uint32_t)(lane & 7);
+            if (valid < 32) {                    // padding after a tensor's end encodes as 0
+                for (int e = valid; e < 32; ++e)
+                    *reinterpret_cast<float*>(rowp + ((((e >> 2) ^ sw) << 4) | ((e & 3) << 2))) = 0.0f;
+            }
+            if constexpr (B == 1) {
+                acc[0] = 0u;
+            } else {
+                uint32_t cur = 0;
+                const uint32_t q0 = (uint32_t)(row0 + lane) * 4u;
+#define DQ_BLOCK(C)                                                                                             \
+                encode_block<B, C>(acc, cur,                                                                    \
+                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)), \
+                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
+                                   inv, q0 + (C), (uint32_t)mm + a.worker0, a.step, a.keys, a.one_bits);
+                DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
+#undef DQ_BLOCK
+            }
+        }
+        __syncwarp();                            // the warp has read all of its rows
+        uint32_t* out_words = reinterpret_cast<uint32_t*>(base);
+        const int off = (int)(((int64_t)row0 * B) & 3);      // staging keeps the stream's 16-byte phase
+        if (valid > 0) {
+#pragma unroll
+            for (int i = 0; i < B; ++i) out_words[off + lane * B + i] = acc[i];
+        }
+        tma::fence_proxy_async();                // these stores precede the bulk copy that refills the stage
+        __syncwarp();
+        const int jend = off + span * B;
+        uint32_t* aligned_dst = a.packed + (int64_t)mm * a.packed_stride + ((int64_t)row0 * B - off);
+        const int q0 = off ? 1 : 0, q1 = jend >> 2;          // full quads [q0, q1)
+        for (int q = q0 + lane; q < q1; q += 32)
+            reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
+        if (off && lane >= off && lane < 4 && lane < jend) aligned_dst[lane] = out_words[lane];   // head
+        int ts = q1 * 4;                                                                          // tail
+        if (off && ts < 4) ts = 4;
+        if (lane < jend - ts) aligned_dst[ts + lane] = out_words[ts + lane];
+        __syncwarp();
+    };
+
+    for (int it = 0; it < n_tiles; ++it) {
+        const int rows = (len + 31) >> 5;
+        // the warp's next bucket (its halves are fetched as this one's halves leave)
+        int nm = m, nk = k + 1, ng0 = 0, nlen = 0;
+        const bool has_next = it + 1 < n_tiles;
+        if (nk == nb) { nk = 0; ++nm; }
+        if (has_next) {
+            if (nm != m) seg = 0;
+            locate(nk, ng0, nlen);
+        }
+
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u))) { timed_out = true; break; }
+        pend_a = false; ++ph_a;
+        if (rows > 32) {
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 1), ph_b & 1u))) { timed_out = true; break; }
+            pend_b = false; ++ph_b;
+        }
+        int valid_a = len - lane * 32;
+        valid_a = valid_a < 0 ? 0 : (valid_a > 32 ? 32 : valid_a);
+        int valid_b = len - (lane + 32) * 32;
+        valid_b = valid_b < 0 ? 0 : (valid_b > 32 ? 32 : valid_b);
+
+        const float part_a = row_reduce(wstage(warp, 0), valid_a);
+        const float part_b = rows > 32 ? row_reduce(wstage(warp, 1), valid_b) : 0.0f;
+        const float nrm = finish<P>(join<P>(join<P>(0.0f, part_a), part_b));
+        if (lane == 0) {
+            a.norms[(int64_t)m * nb + k] = nrm;
+            bad |= !isfinite(nrm);
+        }
+        const float inv = inv_scale(sf, nrm);
+
+        encode_half(wstage(warp, 0), g0, valid_a, rows < 32 ? rows : 32, inv, m);
+        if (has_next) {
+            if (lane == 0) issue(0, ng0, nm);
+            pend_a = true;
+        }
+        if (rows > 32) {
+            encode_half(wstage(warp, 1), g0 + 32, valid_b, rows - 32, inv, m);
+        }
+        if (has_next && nlen > 1024) {
+            if (lane == 0) issue(1, ng0 + 32, nm);
+            pend_b = true;
+        }
+        m = nm; k = nk; g0 = ng0; len = nlen;
+    }
+    if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
+    if (timed_out) {
+        if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
+        // give copies still in flight a bounded chance to land before the CTA's shared memory is released
+        if (pend_a) (void)tma::mbar_wait(wbar(warp, 0), ph_a & 1u);
+        if (pend_b) (void)tma::mbar_wait(wbar(warp, 1), ph_b & 1u);
+    }
+}
+
+template <int P>
+__global__ void __launch_bounds__(kThreads, 6)
+norms_quantize_pack_bucket_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
+{
+    grid_dependency_wait();
+    const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
+    if (tma::smem_addr(smem) & 1023u) {
+        if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
+        return;
+    }
+    if (a.v.n_seg > 1) {
+        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kWTblOffset);
+        for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
+    }
+    if (threadIdx.x == 0) {
+        tma::prefetch_tensor_map(&map);
+        for (int i = 0; i < kWarps * kWStages; ++i) tma::mbar_init(wbar(0, i), 1);
+        tma::fence_barrier_init();
+    }
+    __syncthreads();
+    if (b < 1 || b > DQ_MAX_BITS) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
+        return;
+    }
+    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
+        return;
+    }
+
+    switch (b) {
+#define DQ_CASE(BB) case BB: fused_warp_buckets<BB, P>(a, &map); break;
+        DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
+        DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
+#undef DQ_CASE
+        default: break;
+    }
+}
+
 // ---- buckets that span several warps: the CTA is the pipeline -----------------------
 template <int P>
 __global__ void __launch_bounds__(kThreads, 5)
@@ -708,10 +929,11 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
     a.map_has_worker_dim = worker_dim ? 1 : 0;
 
     const bool per_warp = gpb <= 32;
+    const bool per_bucket = gpb == 64;          // 2048 elements: a warp takes a whole bucket through both stages
     CUtensorMap map;
     const uint64_t dims[3] = {32, (uint64_t)a.v.total_groups, worker_dim ? (uint64_t)M : 1};
     const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
-    const uint32_t box[3] = {32, per_warp ? 32u : (uint32_t)kThreads, 1};
+    const uint32_t box[3] = {32, (per_warp || per_bucket) ? 32u : (uint32_t)kThreads, 1};
     if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
                               CU_TENSOR_MAP_SWIZZLE_128B))
         return DQ_ERR_CUDA;
@@ -728,6 +950,19 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
         }
         const int R = 32 >> a.gpb_shift;
         const int64_t warp_tiles = (int64_t)M * ((L->nb + R - 1) / R);
+        int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
+        if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
+        dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
+    } else if (per_bucket) {
+        const size_t smem_need = (size_t)kWTblOffset + tbl_bytes;
+        const auto kernel = (L->norm == DQ_NORM_LINF) ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF>
+                                                      : norms_quantize_pack_bucket_kernel<DQ_NORM_L2>;
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem_need) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return DQ_ERR_CUDA;
+        }
+        const int64_t warp_tiles = (int64_t)M * L->nb;
         int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
         if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
         dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
