@@ -7,18 +7,16 @@
 // byte is read from HBM a single time.  The norms are written out as well: the
 // server needs them for the average and for the next bit width.
 //
-// Work is cut into tiles of R consecutive buckets of one worker (bucket = 32 * 2^k
-// elements = gpb groups).  In the padded layout such a run is one contiguous span
-// of at most R * gpb groups, fetched by a single TMA tensor copy into a ring of
-// swizzled shared-memory stages.  The thread that owns group l of bucket r of the
-// tile squares its 128-byte row, the gpb threads of a bucket combine by shuffles
-// exactly as dq_bucket_norms does, then the thread encodes its row against that
-// norm and the tile's words leave with 16-byte coalesced stores.
-//  * Buckets of up to 1024 elements (gpb <= 32): every WARP is a pipeline of its own
-//    over tiles of 32 / gpb buckets; no CTA barrier in the loop.
+// Every WARP is a pipeline of its own (two 4 KB stages filled by TMA tensor copies with the
+// 128-byte swizzle; no CTA barrier in any loop).  A lane owns one 128-byte row (32 elements)
+// of a stage: it squares the row, the lanes of a bucket combine by shuffles exactly as
+// dq_bucket_norms does, then the lane encodes its row against that norm and the words leave
+// with 16-byte coalesced stores through the consumed stage.
+//  * Buckets of up to 1024 elements (gpb = bucket / 32 <= 32): tiles of 32 / gpb buckets, fetched
+//    two tiles ahead.
 //  * Buckets of 2048 elements: a warp takes a whole bucket through its two stages.
-//  * Buckets of 4096 elements: the CTA is the pipeline, tiles of 128 / gpb buckets,
-//    partial sums of a bucket's warps meet in shared memory.
+//  * Buckets of 4096 elements: a pair of warps takes a bucket, 2048 elements each, and
+//    exchanges four partial results through shared memory.
 // HBM traffic: 4 + b/8 bytes per element.
 #include "dq_common.cuh"
 #include "dq_device.cuh"
@@ -27,29 +25,25 @@
 namespace {
 
 constexpr int kThreads = 128;
-constexpr int kStages = 2;
-constexpr int kTileBytes = kThreads * 128;          // 16 KB
 constexpr int kMaxSmemSegs = 1023;
 
-// Dynamic shared memory, addressed only through this symbol:
-//   [0, kStages * 16 KB)   input tiles (1024-byte aligned for the 128-byte swizzle)
-//   then 128 * 16 + 4 words of output staging, 4 partial sums, the stage barriers, per-stage tile
-//   geometry, the tensor table
+// Dynamic shared memory, addressed only through this symbol so that every access compiles to a
+// shared-memory instruction:
+//   [0, kWarps * kWStages * 4 KB)   input tiles, warp-major (1024-byte aligned for the swizzle); a
+//   consumed tile doubles as the staging area of its warp's output words; then the stage barriers
+//   and the tensor table
 extern __shared__ __align__(1024) unsigned char smem[];
-constexpr int kOutOffset = kStages * kTileBytes;
-constexpr int kPartOffset = kOutOffset + (kThreads * DQ_MAX_BITS + 4) * 4;
-constexpr int kBarOffset = kPartOffset + 16;
-constexpr int kMetaOffset = kBarOffset + kStages * 8;        // per stage: first group and span of the tile
-constexpr int kTblOffset = kMetaOffset + kStages * 8;
-
-// The per-warp pipelines use another carving of the same symbol:
-//   [0, kWarps * kWStages * 4 KB)   input tiles, warp-major; a consumed tile doubles as the staging
-//   area of its warp's output words; then the stage barriers and the tensor table
 constexpr int kWarps = kThreads / 32;
 constexpr int kWStages = 2;
 constexpr int kWTileBytes = 32 * 128;
 constexpr int kWBarOffset = kWarps * kWStages * kWTileBytes;
 constexpr int kWTblOffset = kWBarOffset + kWarps * kWStages * 8;
+
+// The whole-bucket kernel adds, between the stage barriers and the tensor table, one barrier and two
+// slots of four partial results for each pair of warps that share a bucket of 4096 elements.
+constexpr int kPairBarOffset = kWTblOffset;
+constexpr int kPairPartOffset = kPairBarOffset + (kWarps / 2) * 8;
+constexpr int kBTblOffset = kPairPartOffset + (kWarps / 2) * 2 * 4 * 4;
 
 __device__ __forceinline__ uint64_t* wbar(int warp, int st)
 {
@@ -59,8 +53,6 @@ __device__ __forceinline__ unsigned char* wstage(int warp, int st)
 {
     return smem + (warp * kWStages + st) * kWTileBytes;
 }
-
-__device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
 
 struct FusedArgs {
     LayoutView v;
@@ -78,193 +70,6 @@ struct FusedArgs {
     int32_t stream_reads;         // 1: the gradients exceed the L2, read them with the evict-first policy
     uint32_t one_bits;            // 0x3F800040, kept out of the compiler's sight (see and_or)
 };
-
-template <int B, int P>
-__device__ __forceinline__ void fused_tiles(const FusedArgs& a, const CUtensorMap* map)
-{
-    // the tensor table of a multi-tensor layout always sits in shared memory here (the host
-    // takes the two-pass route for layouts too large for that)
-    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kTblOffset);
-    auto tbl = [&](int i) -> int { return tbl_s[i]; };
-    constexpr int s = (1 << (B - 1)) - 1;
-    const float sf = (float)s;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int n1 = a.v.n_seg + 1;
-    const int gpb = 1 << a.gpb_shift;
-    const int R = kThreads >> a.gpb_shift;                    // buckets per tile
-    const int nb = a.v.nb;
-    const int tiles_per_worker = (nb + R - 1) / R;
-    const int total_tiles = a.M * tiles_per_worker;
-    const int bsz = gpb * 32;
-    const int tile_begin = (int)((int64_t)blockIdx.x * total_tiles / gridDim.x);
-    const int tile_end = (int)((int64_t)(blockIdx.x + 1) * total_tiles / gridDim.x);
-
-    // first group and valid elements of bucket k; `seg` is a walking hint (buckets only move forward)
-    auto locate = [&](int k, int& seg, int& first_group, int& len) {
-        int local, n, g0;
-        if (a.v.n_seg == 1) {
-            local = k; n = a.v.seg0_elems; g0 = 0;
-        } else {
-            while (k >= tbl(n1 + seg + 1)) ++seg;
-            local = k - tbl(n1 + seg);
-            n = tbl(2 * n1 + seg);
-            g0 = tbl(seg);
-        }
-        first_group = g0 + (local << a.gpb_shift);
-        const int left = n - local * bsz;
-        len = left < bsz ? left : bsz;
-    };
-    auto advance = [&](int& mm, int& rr) {
-        if (++rr == tiles_per_worker) { rr = 0; ++mm; }
-    };
-
-    int m = tile_begin / tiles_per_worker, kt = tile_begin - m * tiles_per_worker;
-    int pm = m, pkt = kt, ptile = tile_begin, pseg = 0, pseg_m = m;
-    const uint64_t policy = tma::policy_evict_first();
-    int* meta = reinterpret_cast<int*>(smem + kMetaOffset);
-    int pseg1 = 0;
-    // The issuing thread works out where the tile starts and how many groups it spans, and
-    // leaves both in shared memory for the consumers of that stage (they read them after the
-    // barrier that precedes the stage's next use, or after the prologue's barrier).
-    auto issue = [&](int st) {
-        if (pm != pseg_m) { pseg = 0; pseg1 = 0; pseg_m = pm; }
-        const int k0 = pkt * R;
-        const int k_last = (k0 + R < nb ? k0 + R : nb) - 1;
-        int row0, len0, first_last, len_last;
-        locate(k0, pseg, row0, len0);
-        locate(k_last, pseg1, first_last, len_last);
-        meta[2 * st] = row0;
-        meta[2 * st + 1] = first_last + ((len_last + 31) >> 5) - row0;
-        tma::mbar_expect_tx(full_bar(st), kTileBytes);
-        if (a.stream_reads)
-            tma::load_tile_3d_hint(smem + st * kTileBytes, map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0, policy);
-        else
-            tma::load_tile_3d(smem + st * kTileBytes, map, full_bar(st), 0, row0, a.map_has_worker_dim ? pm : 0);
-    };
-#pragma unroll
-    for (int st = 0; st < kStages; ++st) {
-        if (ptile < tile_end && tid == 0) issue(st);
-        ++ptile;
-        advance(pm, pkt);
-    }
-    __syncthreads();                             // the prologue's tile geometry is visible
-
-    const int r = tid >> a.gpb_shift;            // bucket of the tile this thread works on
-    const int l = tid & (gpb - 1);               // its group inside that bucket
-    float* part = reinterpret_cast<float*>(smem + kPartOffset);
-    uint32_t* out_words = reinterpret_cast<uint32_t*>(smem + kOutOffset);
-    int seg = 0, seg_m = -1;
-    int it = 0;
-    bool timed_out = false, bad = false;
-    for (int tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, kt)) {
-        const int st = it % kStages;
-        if (m != seg_m) { seg = 0; seg_m = m; }
-        const int k = kt * R + r;
-        const int row0 = meta[2 * st], span = meta[2 * st + 1];
-        int first = 0, len = 0;
-        if (k < nb) locate(k, seg, first, len);
-        const int row = first - row0 + l;        // this thread's row of the tile
-        int valid = len - l * 32;                // elements of its group that count
-        valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
-
-        if (!tma::mbar_wait(full_bar(st), (it / kStages) & 1)) { timed_out = true; break; }
-
-        // ---- norm of the bucket (same operations, same order as dq_bucket_norms)
-        unsigned char* base = smem + st * kTileBytes;
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        if (valid > 0) {
-            if (valid == 32) {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
-                    a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
-                }
-            } else {                             // last group of a tensor: what follows is padding
-                for (int e = 0; e < valid; ++e) {
-                    const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
-                    a0 = take<P>(a0, x);
-                }
-            }
-        }
-        float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
-        // butterfly over the threads of the bucket: the steps up to its size, smallest distance last
-        // (the same order as in dq_bucket_norms)
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float other = __shfl_xor_sync(0xffffffffu, sum, o);
-            if (o < gpb) sum = join<P>(sum, other);
-        }
-        if (gpb > 32) {
-            if (lane == 0) part[warp] = sum;
-            __syncthreads();
-            sum = 0.f;
-            const int w0 = (tid >> a.gpb_shift << a.gpb_shift) >> 5;        // first warp of this bucket
-            for (int i = 0; i < (gpb >> 5); ++i) sum = join<P>(sum, part[w0 + i]);
-        }
-        const float nrm = finish<P>(sum);
-        if (l == 0 && k < nb) {
-            a.norms[(int64_t)m * nb + k] = nrm;
-            bad |= !isfinite(nrm);
-        }
-
-        // ---- codes of this thread's group against that norm
-        const int off = (int)(((int64_t)row0 * B) & 3);      // staging keeps the stream's 16-byte phase
-        if (valid > 0) {
-            const float inv = inv_scale(sf, nrm);
-            unsigned char* rowp = base + row * 128;
-            const uint32_t sw = (uint32_t)(row & 7);
-            if (valid < 32) {                    // padding after a tensor's end encodes as 0
-                for (int e = valid; e < 32; ++e)
-                    *reinterpret_cast<float*>(rowp + ((((e >> 2) ^ sw) << 4) | ((e & 3) << 2))) = 0.0f;
-                tma::fence_proxy_async();        // these stores precede the next bulk copy into this stage
-            }
-            uint32_t acc[B];
-            if constexpr (B == 1) {
-                acc[0] = 0u;
-            } else {
-                uint32_t cur = 0;
-                const uint32_t q0 = (uint32_t)(row0 + row) * 4u;
-#define DQ_BLOCK(C)                                                                                             \
-                encode_block<B, C>(acc, cur,                                                                    \
-                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)), \
-                                   *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
-                                   inv, q0 + (C), (uint32_t)m + a.worker0, a.step, a.keys, a.one_bits);
-                DQ_BLOCK(0) DQ_BLOCK(1) DQ_BLOCK(2) DQ_BLOCK(3)
-#undef DQ_BLOCK
-            }
-#pragma unroll
-            for (int i = 0; i < B; ++i) out_words[off + row * B + i] = acc[i];
-        }
-        __syncthreads();
-
-        // ---- the tile's span * B words.  Word i of the tile sits at out_words[off + i] and goes to
-        //      aligned_dst[off + i]; whole quads move 16 bytes at a time, the ragged ends word by word.
-        {
-            const int jend = off + span * B;
-            uint32_t* aligned_dst = a.packed + (int64_t)m * a.packed_stride + ((int64_t)row0 * B - off);
-            const int q0 = off ? 1 : 0, q1 = jend >> 2;          // full quads [q0, q1)
-            for (int q = q0 + tid; q < q1; q += kThreads)
-                reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
-            if (off && tid >= off && tid < 4 && tid < jend) aligned_dst[tid] = out_words[tid];       // head
-            int ts = q1 * 4;                                                                         // tail
-            if (off && ts < 4) ts = 4;
-            if (tid < jend - ts) aligned_dst[ts + tid] = out_words[ts + tid];
-        }
-        __syncthreads();                         // everyone is done with this stage and with the staging area
-        if (ptile < tile_end && tid == 0) {
-            tma::fence_proxy_async();
-            issue(st);
-        }
-        ++ptile;
-        advance(pm, pkt);
-    }
-    if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
-    if (timed_out) {
-        if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
-        for (int j = it + 1; j < it + kStages; ++j)
-            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kStages), (j / kStages) & 1);
-    }
-}
 
 // ---- buckets that fit one warp: a tile that touches the end of a tensor ---------------
 // General route of the per-warp pipelines, kept out of line so that the common case does
@@ -622,7 +427,7 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
     }
 }
 
-// ---- buckets of 2048 elements: a warp takes a whole bucket through its two stages ------
+// ---- buckets of 2048 and 4096 elements: a warp takes 2048 elements through its two stages ----
 //
 // A bucket of 64 groups is two warp tiles.  The warp fetches them into its two stages, every
 // lane squares its row of each, the two halves are reduced by the same butterflies and added
@@ -630,21 +435,25 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
 // soon as a half has left for the packed stream, its stage is refilled with the matching half
 // of the warp's next bucket, so that the fetch runs beside the encoding of the other half.
 // Short buckets (a tensor's last) and padding take the same route with per-lane valid counts.
-template <int B, int P>
+// H = 2: a bucket of 128 groups belongs to a pair of warps, 64 groups each; the pair exchanges its
+// four partial results through shared memory (a barrier of its own, waited for with the usual
+// limit) and both warps add them in the order of dq_bucket_norms.
+template <int B, int P, int H>
 __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUtensorMap* map)
 {
-    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kWTblOffset);
+    const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kBTblOffset);
     constexpr int s = (1 << (B - 1)) - 1;
     const float sf = (float)s;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n1 = a.v.n_seg + 1;
     const int nb = a.v.nb;
-    constexpr int kBucket = 2048;
+    constexpr int kBucket = 2048 * H;
+    const int sub = warp % H;                     // which 2048 elements of the bucket this warp takes
     const int64_t total = (int64_t)a.M * nb;
-    const int64_t nwarps = (int64_t)gridDim.x * kWarps;
-    const int64_t gw = (int64_t)blockIdx.x * kWarps + warp;
-    const int64_t begin = gw * total / nwarps;
-    const int n_tiles = (int)((gw + 1) * total / nwarps - begin);
+    const int64_t nteams = (int64_t)gridDim.x * (kWarps / H);
+    const int64_t team = (int64_t)blockIdx.x * (kWarps / H) + warp / H;
+    const int64_t begin = team * total / nteams;
+    const int n_tiles = (int)((team + 1) * total / nteams - begin);
     if (n_tiles <= 0) return;
 
     int seg = 0;                                  // walking hint: buckets only move forward inside a worker
@@ -658,9 +467,10 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
             n = tbl_s[2 * n1 + seg];
             gs = tbl_s[seg];
         }
-        g0 = gs + local * 64;
-        const int left = n - local * kBucket;
-        len = left < kBucket ? left : kBucket;
+        g0 = gs + local * (64 * H) + 64 * sub;    // first group and valid elements of this warp's share
+        int left = n - local * kBucket - 2048 * sub;
+        left = left < 0 ? 0 : left;
+        len = left < 2048 ? left : 2048;
     };
     auto issue = [&](int st, int row0, int mm) {
         tma::mbar_expect_tx(wbar(warp, st), kWTileBytes);
@@ -675,11 +485,13 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
     int g0, len;
     locate(k, g0, len);
     if (lane == 0) {
-        issue(0, g0, m);
+        if (len > 0) issue(0, g0, m);
         if (len > 1024) issue(1, g0 + 32, m);
     }
-    bool pend_a = true, pend_b = len > 1024;
+    bool pend_a = len > 0, pend_b = len > 1024;
     uint32_t ph_a = 0, ph_b = 0;
+    uint64_t* pair_bar = reinterpret_cast<uint64_t*>(smem + kPairBarOffset) + warp / 2;
+    float* pair_part = reinterpret_cast<float*>(smem + kPairPartOffset) + (warp / 2) * 8;
     bool timed_out = false, bad = false;
     // byte offset of this lane's row inside a stage, swizzle phase folded in: chunk c sits at own ^ (c << 4)
     const uint32_t own = (uint32_t)(lane * 128 + ((lane & 7) << 4));
@@ -761,8 +573,10 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
             locate(nk, ng0, nlen);
         }
 
-        if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u))) { timed_out = true; break; }
-        pend_a = false; ++ph_a;
+        if (rows > 0) {
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u))) { timed_out = true; break; }
+            pend_a = false; ++ph_a;
+        }
         if (rows > 32) {
             if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 1), ph_b & 1u))) { timed_out = true; break; }
             pend_b = false; ++ph_b;
@@ -772,17 +586,29 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         int valid_b = len - (lane + 32) * 32;
         valid_b = valid_b < 0 ? 0 : (valid_b > 32 ? 32 : valid_b);
 
-        const float part_a = row_reduce(wstage(warp, 0), valid_a);
+        const float part_a = rows > 0 ? row_reduce(wstage(warp, 0), valid_a) : 0.0f;
         const float part_b = rows > 32 ? row_reduce(wstage(warp, 1), valid_b) : 0.0f;
-        const float nrm = finish<P>(join<P>(join<P>(0.0f, part_a), part_b));
-        if (lane == 0) {
+        float nrm;
+        if constexpr (H == 1) {
+            nrm = finish<P>(join<P>(join<P>(0.0f, part_a), part_b));
+        } else {
+            float* slot = pair_part + (it & 1) * 4;
+            if (lane == 0) {
+                slot[2 * sub] = part_a;
+                slot[2 * sub + 1] = part_b;
+                tma::mbar_arrive(pair_bar);
+            }
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(pair_bar, (uint32_t)it & 1u))) { timed_out = true; break; }
+            nrm = finish<P>(join<P>(join<P>(join<P>(join<P>(0.0f, slot[0]), slot[1]), slot[2]), slot[3]));
+        }
+        if (lane == 0 && sub == 0) {
             a.norms[(int64_t)m * nb + k] = nrm;
             bad |= !isfinite(nrm);
         }
         const float inv = inv_scale(sf, nrm);
 
-        encode_half(wstage(warp, 0), g0, valid_a, rows < 32 ? rows : 32, inv, m);
-        if (has_next) {
+        if (rows > 0) encode_half(wstage(warp, 0), g0, valid_a, rows < 32 ? rows : 32, inv, m);
+        if (has_next && nlen > 0) {
             if (lane == 0) issue(0, ng0, nm);
             pend_a = true;
         }
@@ -804,7 +630,7 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
     }
 }
 
-template <int P>
+template <int P, int H>
 __global__ void __launch_bounds__(kThreads, 6)
 norms_quantize_pack_bucket_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
@@ -815,12 +641,13 @@ norms_quantize_pack_bucket_kernel(const __grid_constant__ FusedArgs a, const __g
         return;
     }
     if (a.v.n_seg > 1) {
-        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kWTblOffset);
+        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kBTblOffset);
         for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
     }
     if (threadIdx.x == 0) {
         tma::prefetch_tensor_map(&map);
         for (int i = 0; i < kWarps * kWStages; ++i) tma::mbar_init(wbar(0, i), 1);
+        for (int i = 0; i < kWarps / 2; ++i) tma::mbar_init(reinterpret_cast<uint64_t*>(smem + kPairBarOffset) + i, 2);
         tma::fence_barrier_init();
     }
     __syncthreads();
@@ -834,47 +661,7 @@ norms_quantize_pack_bucket_kernel(const __grid_constant__ FusedArgs a, const __g
     }
 
     switch (b) {
-#define DQ_CASE(BB) case BB: fused_warp_buckets<BB, P>(a, &map); break;
-        DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
-        DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
-#undef DQ_CASE
-        default: break;
-    }
-}
-
-// ---- buckets that span several warps: the CTA is the pipeline -----------------------
-template <int P>
-__global__ void __launch_bounds__(kThreads, 5)
-norms_quantize_pack_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
-{
-    grid_dependency_wait();
-    const int b = __ldg(a.dev_b);       // issued first, looked at after the set-up below so that the loads overlap
-    if (tma::smem_addr(smem) & 1023u) {
-        if (threadIdx.x == 0) atomicOr(a.status, DQ_STAT_INTERNAL);
-        return;
-    }
-    if (a.v.n_seg > 1) {
-        int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
-        for (int i = threadIdx.x; i < 3 * (a.v.n_seg + 1); i += kThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
-    }
-    if (threadIdx.x == 0) {
-        tma::prefetch_tensor_map(&map);
-#pragma unroll
-        for (int st = 0; st < kStages; ++st) tma::mbar_init(full_bar(st), 1);
-        tma::fence_barrier_init();
-    }
-    __syncthreads();
-    if (b < 1 || b > DQ_MAX_BITS) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_BAD_BITS);
-        return;
-    }
-    if ((int64_t)b * a.v.total_groups > a.packed_stride) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(a.status, DQ_STAT_CAPACITY);
-        return;
-    }
-
-    switch (b) {
-#define DQ_CASE(BB) case BB: fused_tiles<BB, P>(a, &map); break;
+#define DQ_CASE(BB) case BB: fused_warp_buckets<BB, P, H>(a, &map); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -929,11 +716,11 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
     a.map_has_worker_dim = worker_dim ? 1 : 0;
 
     const bool per_warp = gpb <= 32;
-    const bool per_bucket = gpb == 64;          // 2048 elements: a warp takes a whole bucket through both stages
+    // otherwise gpb is 64 or 128: 2048 elements per warp through both of its stages
     CUtensorMap map;
     const uint64_t dims[3] = {32, (uint64_t)a.v.total_groups, worker_dim ? (uint64_t)M : 1};
     const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
-    const uint32_t box[3] = {32, (per_warp || per_bucket) ? 32u : (uint32_t)kThreads, 1};
+    const uint32_t box[3] = {32, 32, 1};                 // one warp tile
     if (!dq_encode_tensor_map(&map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, dev_grads, dims, strides, box,
                               CU_TENSOR_MAP_SWIZZLE_128B))
         return DQ_ERR_CUDA;
@@ -953,32 +740,21 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
         int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
         if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
         dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
-    } else if (per_bucket) {
-        const size_t smem_need = (size_t)kWTblOffset + tbl_bytes;
-        const auto kernel = (L->norm == DQ_NORM_LINF) ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF>
-                                                      : norms_quantize_pack_bucket_kernel<DQ_NORM_L2>;
+    } else {
+        const size_t smem_need = (size_t)kBTblOffset + tbl_bytes;
+        const bool linf = (L->norm == DQ_NORM_LINF);
+        const auto kernel = gpb == 64 ? (linf ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF, 1>
+                                              : norms_quantize_pack_bucket_kernel<DQ_NORM_L2, 1>)
+                                      : (linf ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF, 2>
+                                              : norms_quantize_pack_bucket_kernel<DQ_NORM_L2, 2>);
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem_need) != cudaSuccess) {
             (void)cudaGetLastError();
             return DQ_ERR_CUDA;
         }
-        const int64_t warp_tiles = (int64_t)M * L->nb;
+        const int64_t warp_tiles = (int64_t)M * L->nb * (gpb / 64);
         int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
         if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
-        dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
-    } else {
-        const size_t smem_need = (size_t)kTblOffset + tbl_bytes;
-        const auto kernel = (L->norm == DQ_NORM_LINF) ? norms_quantize_pack_kernel<DQ_NORM_LINF>
-                                                      : norms_quantize_pack_kernel<DQ_NORM_L2>;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem_need) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return DQ_ERR_CUDA;
-        }
-        const int R = kThreads >> a.gpb_shift;
-        const int64_t tiles = (int64_t)M * ((L->nb + R - 1) / R);
-        int64_t blocks = (int64_t)dq_sm_count() * 5;   // five 42 KB CTAs per SM
-        if (blocks > tiles) blocks = tiles;
         dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
     }
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
