@@ -76,6 +76,16 @@ __device__ __forceinline__ uint32_t div_gpb(const AverageArgs& a, uint32_t n)
     return (uint32_t)(((uint64_t)n * a.div_magic) >> 33);     // exact for n < 2^26, divisor <= 128
 }
 
+// A norm load that stays where it is written: the compiler may not sink it past the barrier wait and
+// the decode that follow (a volatile statement keeps its place among the other volatile statements),
+// so the value is on its way while the unit is decoded.
+__device__ __forceinline__ float load_norm_early(const float* p)
+{
+    float x;
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(x) : "l"(p));
+    return x;
+}
+
 // workers per stage: as many as fit 16 KB with 128 groups of B words each, at most kMaxChunk
 template <int B>
 struct ChunkOf {
@@ -299,7 +309,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                     const float* nrm = a.norms + (int64_t)nm0 * a.v.nb + nbucket;
 #pragma unroll
                     for (int j = 0; j < MC; ++j)
-                        nxt[j] = (has_next && j < nmc && nvalid > 0) ? __ldg(nrm + (int64_t)j * a.v.nb) : 0.0f;
+                        nxt[j] = (has_next && j < nmc && nvalid > 0) ? load_norm_early(nrm + (int64_t)j * a.v.nb) : 0.0f;
                 }
 
                 if constexpr (UPDATE) {
