@@ -67,6 +67,16 @@ __device__ __forceinline__ uint32_t div_gpb(const QuantizeArgs& a, uint32_t n)
     return (uint32_t)(((uint64_t)n * a.div_magic) >> 33);     // exact for n < 2^26, divisor <= 128
 }
 
+// A norm load that stays where it is written (a volatile statement keeps its place among the other
+// volatile statements, the barrier wait among them): the norm of the warp's next tile is requested
+// before this tile's wait and encoding, not after them.
+__device__ __forceinline__ float load_norm_early(const float* p)
+{
+    float x;
+    asm volatile("ld.global.nc.f32 %0, [%1];" : "=f"(x) : "l"(p));
+    return x;
+}
+
 template <int B>
 __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUtensorMap* map, const bool tbl_in_smem)
 {
@@ -112,23 +122,19 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
     }
 
     int seg = 0, seg_m = -1;
-    int it = 0;
-    bool timed_out = false;
-    for (int64_t tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, rt)) {
-        const int st = it % kStages;
-        const uint32_t parity = (it / kStages) & 1;
-        const int row0 = rt * 32;
-        const int g = row0 + lane;
-        const bool active = g < G;
-
-        // where this group lives: tensor, bucket, valid elements (independent of the tile's data)
-        int bucket = 0, valid = 32;
-        if (active) {
+    // Valid elements and bucket norm of this lane's group in tile (mm, rr); the norm is only requested
+    // here.  Groups beyond the layout (the last tile's tail) encode zeros that are never stored.
+    auto prepare = [&](int mm, int rr, int& valid_o, float& norm_o) {
+        const int g = rr * 32 + lane;
+        int bucket = 0;
+        valid_o = 32;
+        norm_o = 0.0f;
+        if (g < G) {
             int local, n, b0;
             if (a.v.n_seg == 1) {
                 local = g; n = a.v.seg0_elems; b0 = 0;
             } else {
-                if (m != seg_m) { seg = 0; seg_m = m; }
+                if (mm != seg_m) { seg = 0; seg_m = mm; }
                 while (g >= tbl(seg + 1)) ++seg;                 // groups only move forward within a worker
                 local = g - tbl(seg);
                 b0 = tbl(n1 + seg);
@@ -136,9 +142,27 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
             }
             bucket = b0 + (int)div_gpb(a, (uint32_t)local);
             const int left = n - local * 32;
-            valid = left < 32 ? left : 32;
+            valid_o = left < 32 ? left : 32;
+            norm_o = load_norm_early(a.norms + (int64_t)mm * a.v.nb + bucket);
         }
-        const float norm = active ? __ldg(a.norms + (int64_t)m * a.v.nb + bucket) : 0.0f;
+    };
+    int next_valid = 32;
+    float next_norm = 0.0f;
+    if (tile_begin < tile_end) prepare(m, rt, next_valid, next_norm);
+    int it = 0;
+    bool timed_out = false;
+    for (int64_t tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, rt)) {
+        const int st = it % kStages;
+        const uint32_t parity = (it / kStages) & 1;
+        const int row0 = rt * 32;
+        const int g = row0 + lane;
+        const int valid = next_valid;
+        const float norm = next_norm;
+        if (tile + 1 < tile_end) {              // the next tile's norm travels while this tile is encoded
+            int m2 = m, rt2 = rt;
+            advance(m2, rt2);
+            prepare(m2, rt2, next_valid, next_norm);
+        }
         const float inv = inv_scale(sf, norm);
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
