@@ -324,22 +324,12 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                 const int st = u % kStages;
                 if (!tma::mbar_wait(full_bar(st), (u / kStages) & 1)) { timed_out = true; break; }
                 const uint32_t* base = stage_words(st) + tid * B;
-                if (mc == MC) {                  // a full unit: unrolled over its workers
-#pragma unroll
-                    for (int j = 0; j < MC; ++j) {
-                        uint32_t wd[B], hi[B];
-                        load_words<B>(base + j * (kThreads * B), wd);
-                        UpperHalves<B, 0>::run(wd, hi);
-                        AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
-                    }
-                } else {
 #pragma unroll 2
-                    for (int j = 0; j < mc; ++j) {
-                        uint32_t wd[B], hi[B];
-                        load_words<B>(base + j * (kThreads * B), wd);
-                        UpperHalves<B, 0>::run(wd, hi);
-                        AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
-                    }
+                for (int j = 0; j < mc; ++j) {
+                    uint32_t wd[B], hi[B];
+                    load_words<B>(base + j * (kThreads * B), wd);
+                    UpperHalves<B, 0>::run(wd, hi);
+                    AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
                 }
 #pragma unroll
                 for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j] * unit;
