@@ -4,12 +4,18 @@
 One step = one communication round of Algorithm 1 on one batch of synthetic
 gradients, all through the C-ABI library: bucket norms and quantize+pack in one
 pass with the bit width chosen after the previous round, unpack+dequantize+average,
-and the bit rule for the next round beside the average.  The same steps as four
-separate calls (norms -> bit rule -> quantize+pack -> average) and with the
-parameter update folded into the average are timed as secondary figures.
-The workload is the ResNet-18-shaped gradient
-(62 tensors, 11,173,962 fp32 per worker, M = 8 workers, bucket 512, Laplace
-values, dynamic b over T = 100 steps, norms shrinking by 0.98 per step).
+and the bit rule for the next round beside the average.
+
+The workload is the largest single-GPU point of the bandwidth sweep: one flat
+N(0,1) fp32 gradient of d = 2^26 elements per worker, M = 32 workers (8 GiB of
+gradients per step), bucket 512.  The headline step runs at the paper's operating
+point b = 4 (chosen on the device by the rule of Eq. 17, calibrated so); the
+``per_b`` table repeats the three hot kernels -- quantize+pack, norms+quantize+pack
+in one pass, unpack+average -- for a list of bit widths, each as a train of launches
+and as single event-bracketed launches, with achieved GB/s of algorithmic bytes, the
+fraction of the measured copy bandwidth and of 8 TB/s, and which roof binds.
+The model-shaped workloads (ResNet-18 M = 8, VGG-16 M = 16, text classifier M = 16)
+are timed as secondary figures.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
@@ -35,21 +41,26 @@ if ROOT not in sys.path:
 
 METRIC = "quantize+pack and unpack+average GB/s of fp32 gradient"
 UNIT = "GB/s"
-WORKLOAD = "resnet18-cifar10 gradient, 62 tensors, d=11173962 fp32/worker, M=8, bucket=512, Laplace, dynamic b, T=100"
+MAIN_D, MAIN_M, MAIN_BUCKET = 1 << 26, 32, 512
+HEADLINE_B = 4
+PER_B = (2, 3, 4, 5, 6, 8, 12, 16)
+WORKLOAD = ("bandwidth sweep point: flat N(0,1) gradient, d=2^26 fp32/worker, M=32 workers (8 GiB/step), bucket=512, "
+            "l2 norms, b=%d chosen on the device by the rule of Eq. 17" % HEADLINE_B)
 SEED = 2107
-POOL_BYTES = 40 << 30          # device memory the pre-generated inputs may take
+NOMINAL_HBM_GBS = 8000.0
+SCHEDULERS_PER_SM = 4          # one warp instruction per scheduler and cycle is the issue roof
 
 
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as fh:
-            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
-    return 6650.0, "fallback (earlier measurement on this pool)"
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs); of measured"
+    return 6650.0, "fallback (earlier measurement on this pool); of fallback"
 
 
-# Sources whose text decides what each timed call moves through DRAM: a counter capture
-# stays valid only while their digest is the one stored beside it.
+# Sources whose text decides what each timed call moves through DRAM and how many instructions
+# it issues: a counter capture stays valid only while their digest is the one stored beside it.
 KERNEL_SOURCES = {
     "norms_quantize_pack": ["dq_fused.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
     "quantize_pack": ["dq_quantize.cu", "dq_device.cuh", "dq_tma.cuh", "dq_common.cuh"],
@@ -67,10 +78,10 @@ def _sources_digest(kernel_key: str) -> str:
     return h.hexdigest()
 
 
-def _traffic(kernel_key: str):
-    """DRAM bytes per launch from the committed ncu capture, or None if one of the
-    kernel's sources changed since the capture."""
-    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+def _counters(kernel_key: str):
+    """The committed ncu counters of a kernel (DRAM bytes and warp instructions per unit of work), or
+    None if one of the kernel's sources changed since the capture."""
+    path = os.path.join(ROOT, "profiles", "counters.json")
     if not os.path.exists(path):
         return None
     with open(path) as fh:
@@ -78,6 +89,19 @@ def _traffic(kernel_key: str):
     if not rec or rec.get("sha256") != _sources_digest(kernel_key):
         return None
     return rec
+
+
+def _interp(table: dict, b: int):
+    """Value at bit width b of a {"b": value} table measured at a few b (linear between neighbours)."""
+    if not table:
+        return None
+    pts = sorted((int(k), float(v)) for k, v in table.items())
+    if b <= pts[0][0]:
+        return pts[0][1]
+    for (b0, v0), (b1, v1) in zip(pts, pts[1:]):
+        if b <= b1:
+            return v0 + (v1 - v0) * (b - b0) / (b1 - b0)
+    return pts[-1][1]
 
 
 class ClockSampler:
@@ -141,44 +165,62 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------
-# reference arm: the CPU checker, as it stands, on the host cores
+# the CPU checker on the host cores (reference arm and cpu_baseline leg)
 # --------------------------------------------------------------------------
 
-def _oracle_round(oracle, np, w, ref, g, t, eps_hat, alpha):
+def _calibrated_eps(G2: float, T: int, x: float) -> float:
+    """eps_hat for which the rule's x = sqrt(T / eps_hat) * G-bar equals `x` at alpha = 1."""
+    return T * G2 / (x * x)
+
+
+def _x_for(b: int) -> float:
+    """A value of x that the rule rounds up to exactly b bits: half a level below s(b) = 2^(b-1) - 1."""
+    return ((1 << (b - 1)) - 1) - 0.5
+
+
+def _oracle_round(oracle, ref, g, T, t, eps_hat):
     norms = oracle.bucket_norms(ref, g)
-    b, s, _ = oracle.choose_bits(norms, w.T, t, eps_hat, alpha)
+    b, s, _ = oracle.choose_bits(norms, T, t, eps_hat, 1.0)
     packed = oracle.quantize_pack(ref, g, norms, b, SEED, t)
     out = oracle.unpack_dequant_average(ref, packed, norms, b)
     return b, out
 
 
-def run_reference(args) -> dict:
+def _oracle_rate(grads, seconds: float, min_steps: int, max_steps: int, fixed_steps=None, warmup: int = 0):
+    """Times whole rounds of the CPU checker on `grads` [M, d] (numpy); returns (GB/s, steps, s, b, cores)."""
     import numpy as np
 
     import oracle
-    from paper_2107_14575_b200 import workloads
-    factor = 16
-    full = workloads.config_resnet18()
-    w = workloads.scaled_down(full, factor)
-    ref = oracle.Layout(w.segments, w.bucket)
+    M, d = grads.shape
+    ref = oracle.Layout([d], MAIN_BUCKET)
     cores = os.cpu_count() or 1
     oracle.set_threads(cores)
-    pool = [workloads.make_grads(w, ref.offsets, ref.D32, step=t) for t in range(4)]
-    n0 = oracle.bucket_norms(ref, pool[0])
-    G2 = float((n0.astype(np.float64) ** 2).sum() / w.M)
-    alpha = full.alpha
-    eps_hat = full.T * alpha ** (full.T - 1) * G2 / full.x0 ** 2
-    for i in range(args.warmup):
-        _oracle_round(oracle, np, w, ref, pool[i % 4], i % full.T, eps_hat, alpha)
-    t0 = time.perf_counter()
-    for i in range(args.steps):
-        _oracle_round(oracle, np, w, ref, pool[i % 4], i % full.T, eps_hat, alpha)
-    dt = time.perf_counter() - t0
-    gbs = 4.0 * w.M * w.d * args.steps / dt / 1e9
-    sample = "every tensor of the workload cut to 1/%d of its size (d=%d per worker), all M=8 workers" % (factor, w.d)
+    n0 = oracle.bucket_norms(ref, grads)
+    G2 = float((n0.astype(np.float64) ** 2).sum() / M)
+    eps_hat = _calibrated_eps(G2, 100, _x_for(HEADLINE_B))
+    b = 0
+    for i in range(warmup):
+        b, _ = _oracle_round(oracle, ref, grads, 100, i % 100, eps_hat)
+    steps, dt = 0, 0.0
+    while (steps < fixed_steps) if fixed_steps is not None else (steps < min_steps or (dt < seconds and steps < max_steps)):
+        t0 = time.perf_counter()
+        b, _ = _oracle_round(oracle, ref, grads, 100, steps % 100, eps_hat)
+        dt += time.perf_counter() - t0
+        steps += 1
+    return 4.0 * M * d * steps / dt / 1e9, steps, dt, b, cores
+
+
+def run_reference(args) -> dict:
+    import numpy as np
+    d_sample = 1 << 21
+    rng = np.random.Generator(np.random.PCG64(SEED))
+    g = rng.standard_normal((MAIN_M, d_sample), dtype=np.float32)
+    gbs, steps, dt, b, cores = _oracle_rate(g, 0.0, 0, 0, fixed_steps=args.steps, warmup=args.warmup)
+    sample = ("each step = one whole round of the CPU checker on a prefix of the workload: the first 2^21 of the 2^26 "
+              "elements of all M=32 workers (268 MB of gradients), b=%d from its own bit rule" % b)
     return {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(steps, 1) * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": WORKLOAD, "sample": sample},
         "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
@@ -190,16 +232,141 @@ def run_reference(args) -> dict:
 # CUDA arm
 # --------------------------------------------------------------------------
 
-def _gen_step(torch, gen, scale_vec, M, D32, step):
+class Timer:
+    """CUDA-event timing on torch's current stream (the stream every library call is launched on)."""
+
+    def __init__(self, torch, warmup: int):
+        self.torch, self.warmup = torch, max(3, warmup)
+
+    def train(self, fn, n: int) -> float:
+        """ms per call of `n` calls launched back to back between two events."""
+        torch = self.torch
+        for i in range(self.warmup):
+            fn(i)
+        torch.cuda.synchronize()
+        s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s.record()
+        for i in range(n):
+            fn(i)
+        e.record()
+        torch.cuda.synchronize()
+        return s.elapsed_time(e) / n
+
+    def single(self, fn, n: int) -> float:
+        """mean ms of `n` calls each bracketed by its own pair of events (sees the launch latency too)."""
+        torch = self.torch
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        torch.cuda.synchronize()
+        for i, (s, e) in enumerate(ev):
+            s.record()
+            fn(i)
+            e.record()
+        torch.cuda.synchronize()
+        return sum(s.elapsed_time(e) for s, e in ev) / n
+
+
+def _bound(kernel_key, b, alg_bytes, units, ms, peak_gbs, sm_count, sm_mhz):
+    """Which roof binds a launch that took `ms`: the time its algorithmic bytes need at the measured copy
+    bandwidth, or the time its warp instructions need at one instruction per scheduler and cycle
+    (instructions per unit from the committed ncu counters x units, at the sampled SM clock)."""
+    gbs = alg_bytes / (ms * 1e-3) / 1e9
+    rec = {"ms": round(ms, 5), "achieved_gbs": round(gbs, 1), "frac_of_measured": round(gbs / peak_gbs, 4),
+           "frac_of_8tbs": round(gbs / NOMINAL_HBM_GBS, 4), "algorithmic_bytes": alg_bytes, "bound": "hbm",
+           "issue": None}
+    c = _counters(kernel_key)
+    ipu = _interp((c or {}).get("warp_instructions_per_group"), b)
+    if ipu is not None and sm_mhz:
+        issue_peak = sm_count * SCHEDULERS_PER_SM * sm_mhz * 1e6            # warp instructions per second
+        inst = ipu * units
+        t_issue_ms = inst / issue_peak * 1e3
+        t_hbm_ms = alg_bytes / (peak_gbs * 1e9) * 1e3
+        rec["issue"] = {"warp_instructions_per_group": round(ipu, 1), "warp_instructions": inst,
+                        "roof_ms": round(t_issue_ms, 5), "hbm_roof_ms": round(t_hbm_ms, 5),
+                        "frac_of_issue_roof": round(t_issue_ms / ms, 4),
+                        "lane_instructions_per_element": round(ipu, 1),     # 32 lanes x instructions / 32 elements
+                        "sm_mhz": sm_mhz}
+        if t_issue_ms > t_hbm_ms:
+            rec["bound"] = "alu"
+    return rec
+
+
+def _gen_resnet(torch, gen, w, L, dev, step):
     """Laplace(0, scale_l * 0.98^step) per tensor l, zero on padding; [M, D32] fp32 on the device."""
-    u = torch.rand((M, D32), generator=gen, device=scale_vec.device, dtype=torch.float32) - 0.5
+    nseg = len(w.segments)
+    scale_vec = torch.zeros(L.D32, dtype=torch.float32, device=dev)
+    for i, n in enumerate(w.segments):
+        scale_vec[L.offsets[i]: L.offsets[i] + n] = 1e-2 * 10.0 ** (-i / (nseg - 1))
+    u = torch.rand((w.M, L.D32), generator=gen, device=dev, dtype=torch.float32) - 0.5
     g = -torch.sign(u) * torch.log1p(-2.0 * u.abs().clamp_(max=0.4999999))
     g.mul_(scale_vec * (0.98 ** step))
     return g
 
 
+def _gen_vgg(torch, gen, w, L, dev, step):
+    """Gaussian values, 1% of the entries scaled x100; zero on padding."""
+    mask = torch.zeros(L.D32, dtype=torch.float32, device=dev)
+    for i, n in enumerate(w.segments):
+        mask[L.offsets[i]: L.offsets[i] + n] = 1.0
+    g = torch.randn((w.M, L.D32), generator=gen, device=dev, dtype=torch.float32) * 1e-2
+    big = torch.rand((w.M, L.D32), generator=gen, device=dev, dtype=torch.float32) < 0.01
+    g = torch.where(big, g * 100.0, g)
+    return g * mask
+
+
+def _gen_text(torch, gen, w, L, dev, step):
+    """Embedding 30000 x 300 with 97% of the rows exactly zero (fresh subset per worker), dense LSTM and head."""
+    g = torch.randn((w.M, L.D32), generator=gen, device=dev, dtype=torch.float32) * 1e-2
+    mask = torch.zeros(L.D32, dtype=torch.float32, device=dev)
+    for i, n in enumerate(w.segments):
+        mask[L.offsets[i]: L.offsets[i] + n] = 1.0
+    g = g * mask
+    rows, cols = 30000, 300
+    emb = g[:, L.offsets[0]: L.offsets[0] + rows * cols].view(w.M, rows, cols)
+    keep = torch.rand((w.M, rows, 1), generator=gen, device=dev) < 0.03
+    emb.mul_(keep.to(torch.float32))
+    return g
+
+
+def _model_workload(torch, dq, Round, timer, w, gen_fn, dev, K, peak):
+    """Algorithm-1 steps of a model-shaped workload with the dynamic schedule of its config; returns the
+    per-step time, the bit widths seen, and the event-bracketed time of each call."""
+    rnd = Round(w.segments, w.bucket, w.M, device=str(dev))
+    L = rnd.layout
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(SEED + 17)
+    npool = 3
+    pool = [gen_fn(torch, gen, w, L, dev, p) for p in range(npool)]
+    rnd.norms_(pool[0])
+    G2 = float((rnd.norms.double() ** 2).sum().item() / w.M)
+    T, alpha = w.T, w.alpha
+    eps_hat = T * alpha ** (T - 1) * G2 / w.x0 ** 2
+
+    def rule_for(i):
+        return dq.Rule.dynamic(T, i % T, eps_hat, alpha)
+
+    rnd.bits_(rule_for(0))
+    b0 = rnd.bits()
+    ms = timer.train(lambda i: rnd.step_fused(pool[i % npool], rule_for(i + 1), SEED, i), K)
+    b1 = rnd.bits()
+    # per call, event-bracketed, at the b the schedule has reached
+    elems = w.M * L.D32
+    t_f = timer.single(lambda i: rnd.norms_quantize_(pool[i % npool], SEED, i), min(K, 10))
+    t_a = timer.single(lambda i: rnd.average_(), min(K, 10))
+    assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
+    out = {"workload": "%s: %d tensors, d=%d fp32/worker, M=%d, bucket=%d, dynamic b over T=%d"
+                       % (w.name, len(w.segments), w.d, w.M, w.bucket, w.T),
+           "ms_per_step": round(ms, 5), "value": round(4.0 * w.M * w.d / (ms * 1e-3) / 1e9, 1),
+           "bits_first_last": [b0, b1], "mb_per_step": (4 * elems) >> 20,
+           "norms_quantize_pack": {"b": b1, "ms": round(t_f, 5),
+                                   "frac_of_measured": round((4.0 + b1 / 8.0) * elems / (t_f * 1e-3) / 1e9 / peak, 4)},
+           "unpack_dequant_average": {"b": b1, "ms": round(t_a, 5),
+                                      "frac_of_measured": round((w.M * b1 / 8.0 + 4.0) * L.D32 / (t_a * 1e-3) / 1e9 / peak, 4)}}
+    del pool, rnd
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_cuda(args) -> dict:
-    import numpy as np
     import torch
     import torch.distributed as dist
 
@@ -214,220 +381,178 @@ def run_cuda(args) -> dict:
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    w = workloads.config_resnet18()
-    rnd = Round(w.segments, w.bucket, w.M, device=str(dev))
+    K, W = args.steps, max(3, args.warmup)
+    M, d = MAIN_M, MAIN_D
+    rnd = Round([d], MAIN_BUCKET, M, device=str(dev))
     L = rnd.layout
-    M, D32, T = w.M, L.D32, w.T
-    nseg = len(w.segments)
-
-    scale_vec = torch.zeros(D32, dtype=torch.float32, device=dev)
-    for i, n in enumerate(w.segments):
-        scale_vec[L.offsets[i]: L.offsets[i] + n] = 1e-2 * 10.0 ** (-i / (nseg - 1))
-
-    K, W = args.steps, args.warmup
-    step_bytes = 4 * M * D32
-    npool = max(2, min(K + W, POOL_BYTES // step_bytes))
-    if npool > T:
-        npool = T                              # one input set per schedule step: set i % T belongs to step t = i % T
+    D32 = L.D32
+    elems = M * D32
+    groups = elems // 32
     gen = torch.Generator(device=dev)
     gen.manual_seed(SEED + 1000 * rank)
-    # pool entry p is the input of every step i with i % npool == p; it carries the
-    # norm decay of schedule step t = p % T
-    pool = [_gen_step(torch, gen, scale_vec, M, D32, p % T) for p in range(npool)]
-
-    # calibrate eps_hat so that x(t = 0) = x0 (b = 4 at the start of the schedule)
-    rnd.norms_(pool[0])
+    grads = torch.randn((M, D32), generator=gen, device=dev, dtype=torch.float32)      # 8 GiB: far larger than the L2
+    rnd.norms_(grads)
     G2 = float((rnd.norms.double() ** 2).sum().item() / M)
-    alpha = w.alpha
-    eps_hat = T * alpha ** (T - 1) * G2 / w.x0 ** 2
+    T = 100
 
-    def rule_for(i):
-        return dq.Rule.dynamic(T, i % T, eps_hat, alpha)
+    def rule_b(b, t=0):
+        """The dynamic rule of Eq. 17 with eps_hat calibrated so that it lands on b for these norms."""
+        return dq.Rule.dynamic(T, t % T, _calibrated_eps(G2, T, _x_for(b)), 1.0)
+
+    def set_b(b):
+        rnd.bits_(rule_b(b))
+        got = rnd.bits()
+        assert got == b, "the device rule chose b=%d where the calibration aims at %d" % (got, b)
 
     peak, peak_src = _peaks()
-    elems = M * D32
-
-    def b_of(norm_set, t):
-        """b the rule gives at schedule step t for the norms of input set `norm_set` (synchronises)."""
-        rnd.norms_(pool[norm_set % npool])
-        rnd.bits_(dq.Rule.dynamic(T, t % T, eps_hat, alpha))
-        return rnd.bits()
-
-    # Two orders of the same four steps (both supported by the library):
-    #  "algorithm1": as Algorithm 1 of the paper runs -- quantize with b_t, which was chosen from the
-    #     previous step's norms, in ONE pass together with the norms (dq_norms_quantize_pack), average,
-    #     then choose b_{t+1} from this step's norms.  This is the timed headline.
-    #  "four_call": norms, bit rule on this step's own norms, quantize (second pass), average.
-    host_ms = {}
-
-    def run_order(order, sampler=None):
-        if order in ("algorithm1", "algorithm1_update"):
-            names = ["norms_quantize_pack", "unpack_dequant_average" if order == "algorithm1" else "unpack_average_update",
-                     "choose_bits"]
-            bits = [b_of(0, 0)] + [b_of(i - 1, i) for i in range(1, K)]          # untimed: b of every step
-        else:
-            names = ["bucket_norms", "choose_bits", "quantize_pack", "unpack_dequant_average"]
-            bits = [b_of(i, i) for i in range(K)]
-
-        def one_step(i, e):
-            g = pool[i % npool]
-            if order == "algorithm1":
-                rnd.step_fused(g, rule_for(i + 1), SEED, i, overlap=not args.no_overlap, events=e)
-            elif order == "algorithm1_update":
-                rnd.step_fused(g, rule_for(i + 1), SEED, i, overlap=not args.no_overlap, events=e, params=params,
-                               lr=1e-3)
-            else:
-                rec = (lambda j: e[j].record()) if e else (lambda j: None)
-                rec(0); rnd.norms_(g)
-                rec(1); rnd.bits_(rule_for(i))
-                rec(2); rnd.quantize_(g, SEED, i)
-                rec(3); rnd.average_()
-                rec(4)
-
-        nev = 5
-        b_of(0, 0)                                  # dev_b holds b_0 before the first step
-        dummy = [torch.cuda.Event(enable_timing=True) for _ in range(nev)]
-        for i in range(max(W, 3)):
-            one_step(i, dummy)
-        b_of(0, 0)
-        torch.cuda.synchronize()
-        assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
-        # Per-call events cost about 3 us of device time each (the stream drains around them), so only
-        # every `ev_stride`-th timed step carries them; the others run as a user's steps do.
-        ev_stride = max(1, K // 12)
-        ev = {i: [torch.cuda.Event(enable_timing=True) for _ in range(nev)] for i in range(0, K, ev_stride)}
-        start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-        if sampler:
-            sampler.start()
-        start.record()
-        h0 = time.perf_counter()
-        for i in range(K):
-            one_step(i, ev.get(i))
-        end.record()
-        host_ms[order] = (time.perf_counter() - h0) * 1e3 / K      # host time to submit one step
-        torch.cuda.synchronize()
-        clk = sampler.stop() if sampler else None
-        t_ms = start.elapsed_time(end)
-        assert rnd.read_status() == 0
-        t_ms = replicas.max_over_ranks(t_ms, dev)
-        # algorithm1: events 0-1 bracket the fused call, 1-2 the average, 3-4 the bit rule (on its own
-        # stream when it overlaps the average); four_call: 0-1-2-3-4 in sequence
-        spans = [(0, 1), (1, 2), (3, 4)] if order != "four_call" else [(0, 1), (1, 2), (2, 3), (3, 4)]
-        totals = {n: sum(e[p].elapsed_time(e[q]) for e in ev.values()) for n, (p, q) in zip(names, spans)}
-        nsamp = len(ev)
-        mean_b = sum(bits) / len(bits)
-        mean_bs = sum(bits[i] for i in ev) / nsamp                 # of the steps that carried events
-        alg_bytes = {
-            "bucket_norms": 4.0 * elems,
-            "choose_bits": 4.0 * M * L.nb,
-            "quantize_pack": (4.0 + mean_bs / 8.0) * elems,
-            "norms_quantize_pack": (4.0 + mean_bs / 8.0) * elems,
-            "unpack_dequant_average": (M * mean_bs / 8.0 + 4.0) * D32,
-            "unpack_average_update": (M * mean_bs / 8.0 + 8.0) * D32,
-        }
-        # shares are of the time on the main stream; a bit rule that runs beside the average on the
-        # second stream is not on that path (its interval there includes waiting for room on the SMs)
-        beside = order != "four_call" and not args.no_overlap
-        on_path = [n for n in names if not (beside and n == "choose_bits")]
-        path_total = sum(totals[n] for n in on_path)
-        kernels = {}
-        for n in names:
-            avg_ms = totals[n] / nsamp
-            gbs = alg_bytes[n] / (avg_ms * 1e-3) / 1e9
-            kernels[n] = {"avg_ms": round(avg_ms, 5), "achieved_gbs": round(gbs, 1), "frac": round(gbs / peak, 4),
-                          "share": round(totals[n] / path_total, 4) if n in on_path else None,
-                          "algorithmic_bytes_per_launch": alg_bytes[n]}
-            if n not in on_path:
-                kernels[n]["runs_beside"] = names[1]
-        return t_ms, bits, mean_b, kernels, clk, len(names) + (1 if "choose_bits" in names else 0)
-
+    sm_count = torch.cuda.get_device_properties(dev).multi_processor_count
+    timer = Timer(torch, W)
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", ""))
-    ms, bits, mean_b, kernels, clocks, launches_per_step = run_order("algorithm1", sampler)
-    dominant = max(kernels, key=lambda n: kernels[n]["avg_ms"])
-    tr = _traffic(dominant)
-    roofline = {
-        "kernel": dominant, "bound": "hbm", "achieved": kernels[dominant]["achieved_gbs"], "peak": peak,
-        "unit": "GB/s", "frac": kernels[dominant]["frac"], "traffic": (tr or {}).get("bytes_per_launch"),
-        "peak_source": peak_src + "; of measured" if peak_src.startswith("measured") else peak_src + "; of fallback",
-        "algorithmic_bytes_per_launch": kernels[dominant]["algorithmic_bytes_per_launch"], "mean_b": round(mean_b, 3),
-        "frac_of_nominal_8tbs": round(kernels[dominant]["achieved_gbs"] / 8000.0, 4),
-        "kernels": kernels,
+
+    # ---- headline: K steps in the order of Algorithm 1 at b = 4
+    set_b(HEADLINE_B)
+    for i in range(W):
+        rnd.step_fused(grads, rule_b(HEADLINE_B, i + 1), SEED, i, overlap=not args.no_overlap)
+    torch.cuda.synchronize()
+    assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
+    nev = 5
+    ev_stride = max(1, K // 12)
+    ev = {i: [torch.cuda.Event(enable_timing=True) for _ in range(nev)] for i in range(0, K, ev_stride)}
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record()
+    h0 = time.perf_counter()
+    for i in range(K):
+        rnd.step_fused(grads, rule_b(HEADLINE_B, i + 1), SEED, i, overlap=not args.no_overlap, events=ev.get(i))
+    end.record()
+    host_submit_ms = (time.perf_counter() - h0) * 1e3 / K
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_total = replicas.max_over_ranks(start.elapsed_time(end), dev)
+    assert rnd.read_status() == 0 and rnd.bits() == HEADLINE_B
+    sm_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz")
+    spans = {"norms_quantize_pack": (0, 1), "unpack_dequant_average": (1, 2), "choose_bits": (3, 4)}
+    step_ms = {n: sum(e[p].elapsed_time(e[q]) for e in ev.values()) / len(ev) for n, (p, q) in spans.items()}
+    alg_bytes = {
+        "bucket_norms": lambda b: 4.0 * elems,
+        "quantize_pack": lambda b: (4.0 + b / 8.0) * elems,
+        "norms_quantize_pack": lambda b: (4.0 + b / 8.0) * elems,
+        "unpack_dequant_average": lambda b: (M * b / 8.0 + 4.0) * D32,
     }
-    # The events that bracket a single launch also see its launch latency (the stream drains at
-    # every record).  For context, the same kernel launched back to back between two events:
-    if dominant == "norms_quantize_pack":
-        nb2b = 10
-        b_last = bits[-1]
-        rnd.bits_(dq.Rule.fixed(b_last))
-        for i in range(3):
-            rnd.norms_quantize_(pool[i % npool], SEED, i)
-        torch.cuda.synchronize()
-        s3, e3 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        s3.record()
-        for i in range(nb2b):
-            rnd.norms_quantize_(pool[i % npool], SEED, i)
-        e3.record()
-        torch.cuda.synchronize()
-        b2b_ms = s3.elapsed_time(e3) / nb2b
-        b2b_bytes = (4.0 + b_last / 8.0) * elems
-        roofline["back_to_back"] = {"launches": nb2b, "b": b_last, "avg_ms": round(b2b_ms, 5),
-                                    "achieved": round(b2b_bytes / (b2b_ms * 1e-3) / 1e9, 1),
-                                    "frac": round(b2b_bytes / (b2b_ms * 1e-3) / 1e9 / peak, 4)}
-    upd = None
-    if not args.no_four_call:
-        # the same order with the parameter update of Eq. 2 folded into the server step
-        params = torch.zeros(D32, dtype=torch.float32, device=dev)
-        msu, _, mean_bu, kernelsu, _, _ = run_order("algorithm1_update")
-        upd = {"ms_per_step": msu / K, "value": replicas.whole_job_rate(4.0 * M * w.d * K, world, msu) / 1e9,
-               "mean_bits": round(mean_bu, 3), "kernels": kernelsu}
-    four = None
-    if not args.no_four_call:
-        ms4, bits4, mean_b4, kernels4, _, _ = run_order("four_call")
-        four = {"ms_per_step": ms4 / K, "value": replicas.whole_job_rate(4.0 * M * w.d * K, world, ms4) / 1e9,
-                "mean_bits": round(mean_b4, 3), "kernels": kernels4}
+    # units of the instruction model: 32-element groups a launch processes (per worker for the
+    # quantizers; for the average a group of M x 32 codes)
+    units = {"bucket_norms": groups, "quantize_pack": groups, "norms_quantize_pack": groups,
+             "unpack_dequant_average": D32 // 32}
+    kernels = {n: _bound(n, HEADLINE_B, alg_bytes[n](HEADLINE_B), units[n], step_ms[n], peak, sm_count, sm_mhz)
+               for n in ("norms_quantize_pack", "unpack_dequant_average")}
+    path_ms = sum(step_ms[n] for n in kernels)
+    for n in kernels:
+        kernels[n]["share"] = round(step_ms[n] / path_ms, 4)
+    kernels["choose_bits"] = {"ms": round(step_ms["choose_bits"], 5), "share": None,
+                              "runs_beside": "unpack_dequant_average (second stream)" if not args.no_overlap else None,
+                              "algorithmic_bytes": 4.0 * M * L.nb}
+    dominant = max(("norms_quantize_pack", "unpack_dequant_average"), key=lambda n: step_ms[n])
+    dk = kernels[dominant]
+    cnt = _counters(dominant)
+    traffic = _interp((cnt or {}).get("dram_bytes_per_group"), HEADLINE_B)
+    roofline = {"kernel": dominant, "b": HEADLINE_B, "bound": dk["bound"], "unit": "GB/s", "achieved": dk["achieved_gbs"],
+                "peak": peak, "frac": dk["frac_of_measured"], "peak_source": peak_src,
+                "traffic": traffic * units[dominant] if traffic is not None else None,
+                "algorithmic_bytes_per_launch": dk["algorithmic_bytes"], "frac_of_nominal_8tbs": dk["frac_of_8tbs"],
+                "hbm": {"achieved_gbs": dk["achieved_gbs"], "frac_of_measured": dk["frac_of_measured"]},
+                "kernels": kernels,
+                "timing": "CUDA events on the launching stream around each call of every %d-th timed step (%d samples)"
+                          % (ev_stride, len(ev))}
+    if dk["bound"] == "alu":
+        # the instruction roof binds: report against it (lane instructions per second; peak = SMs x 128 lanes x
+        # sampled SM clock), the HBM figures stay beside it under "hbm"
+        iss = dk["issue"]
+        roofline.update({"unit": "Ginst/s", "achieved": round(iss["warp_instructions"] * 32 / (dk["ms"] * 1e-3) / 1e9, 1),
+                         "peak": round(sm_count * SCHEDULERS_PER_SM * 32 * sm_mhz * 1e6 / 1e9, 1),
+                         "frac": iss["frac_of_issue_roof"],
+                         "peak_source": "SMs x 4 schedulers x 32 lanes x sampled SM clock (one warp instruction per "
+                                        "scheduler and cycle); instructions per group from profiles/counters.json"})
 
-    value = replicas.whole_job_rate(4.0 * M * w.d * K, world, ms) / 1e9
+    # ---- per b: the three hot kernels, trains of K launches and single event-bracketed launches
+    per_b = {}
+    n_single = min(K, 8)
+    norms_ms = timer.train(lambda i: rnd.norms_(grads), K)
+    for b in PER_B:
+        set_b(b)
+        rec = {}
+        rnd.norms_(grads)
+        for name, fn in (("quantize_pack", lambda i: rnd.quantize_(grads, SEED, i)),
+                         ("norms_quantize_pack", lambda i: rnd.norms_quantize_(grads, SEED, i)),
+                         ("unpack_dequant_average", lambda i: rnd.average_())):
+            t_train = timer.train(fn, K)
+            t_single = timer.single(fn, n_single)
+            r = _bound(name, b, alg_bytes[name](b), units[name], t_train, peak, sm_count, sm_mhz)
+            r["single_launch_ms"] = round(t_single, 5)
+            r["single_launch_frac_of_measured"] = round(alg_bytes[name](b) / (t_single * 1e-3) / 1e9 / peak, 4)
+            r["gradient_gbs"] = round(4.0 * M * d / (t_train * 1e-3) / 1e9, 1)
+            rec[name] = r
+        step = timer.train(lambda i: rnd.step_fused(grads, rule_b(b, i + 1), SEED, i, overlap=not args.no_overlap), K)
+        rec["step_ms"] = round(step, 5)
+        rec["step_gradient_gbs"] = round(4.0 * M * d / (step * 1e-3) / 1e9, 1)
+        per_b[str(b)] = rec
+        assert rnd.read_status() == 0 and rnd.bits() == b
+    set_b(HEADLINE_B)
 
-    # ---- end to end: pinned host gradients in, averaged gradient out, copies timed ----
+    value = replicas.whole_job_rate(4.0 * M * d * K, world, ms_total) / 1e9
+
+    # ---- end to end: pinned host gradients in, averaged gradient out, copies timed
     e2e = None
     if not args.no_e2e:
-        e2e = _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, w.d, D32)
+        e2e = _end_to_end(torch, dist, rnd, grads, rule_b, K, world, dev, M, d, D32)
+
+    # ---- the model-shaped workloads (secondary)
+    other = None
+    if not args.no_models:
+        del grads
+        rnd = None
+        torch.cuda.empty_cache()
+        other = {}
+        for w, gen_fn in ((workloads.config_resnet18(), _gen_resnet), (workloads.config_vgg16(), _gen_vgg),
+                          (workloads.config_text(), _gen_text)):
+            other[w.name] = _model_workload(torch, dq, Round, timer, w, gen_fn, dev, K, peak)
+
     out = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": max(W, 3),
-        "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_total / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "bits_first_last": [bits[0], bits[-1]], "mean_bits": round(mean_b, 3),
+        "config": {"workload": WORKLOAD,
                    "order": "Algorithm 1: norms+quantize+pack in one pass with b_t, average, b_{t+1} from this step's norms"
                             + ("" if args.no_overlap else " (bit rule on a second stream beside the average)"),
-                   "l2": "inputs larger than L2 (%d MB per step, %d rotating input sets)" % (step_bytes >> 20, npool),
-                   "kernel_events": "CUDA events around each call on every %d-th timed step (%d samples)"
-                                    % (max(1, K // 12), len(range(0, K, max(1, K // 12)))),
+                   "l2": "inputs larger than L2 (%d MB of gradients per step)" % ((4 * elems) >> 20),
+                   "per_b": "b in %s: trains of %d launches and %d single event-bracketed launches per kernel"
+                            % (list(PER_B), K, n_single),
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
-        "clocks": clocks, "e2e": e2e, "gpu_launches": launches_per_step * K, "roofline": roofline,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * K, "roofline": roofline,
+        "per_b": per_b, "bucket_norms": _bound("bucket_norms", 0, 4.0 * elems, groups, norms_ms, peak, sm_count, sm_mhz),
         # what the workers would put on the wire per step (Eq. 7: d * b bits per worker, plus the fp32 norms)
-        "wire": {"bytes_per_step": M * (w.d * mean_b / 8.0 + 4.0 * L.nb), "fp32_bytes_per_step": 4.0 * M * w.d,
-                 "ratio": round((w.d * mean_b / 8.0 + 4.0 * L.nb) / (4.0 * w.d), 4)},
-        "four_call_order": four, "with_parameter_update": upd,
-        "host_submit_ms_per_step": round(host_ms["algorithm1"], 5),
+        "wire": {"bytes_per_step": M * (d * HEADLINE_B / 8.0 + 4.0 * L.nb), "fp32_bytes_per_step": 4.0 * M * d,
+                 "ratio": round((d * HEADLINE_B / 8.0 + 4.0 * L.nb) / (4.0 * d), 4)},
+        "model_workloads": other, "host_submit_ms_per_step": round(host_submit_ms, 5),
     }
-
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = _cpu_baseline(pool, w, eps_hat, alpha)
+        out["cpu_baseline"] = _cpu_baseline(torch, gen, dev)
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
     return out if rank == 0 else {}
 
 
-def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> dict:
+def _end_to_end(torch, dist, rnd, grads, rule_b, K, world, dev, M, d, D32) -> dict:
     from paper_2107_14575_b200 import replicas
-    Ke = min(K, 10)
-    host = [pool[p].cpu().pin_memory() for p in range(2)]
+    Ke = max(2, min(K, 4))
+    host = torch.empty((M, D32), dtype=torch.float32, pin_memory=True)
+    host.copy_(grads)
+    torch.cuda.synchronize()
     for i in range(2):
-        rnd.step_host(host[i % 2], rule_for(i + 1), SEED, i)
+        rnd.step_host(host, rule_b(HEADLINE_B, i + 1), SEED, i)
     rnd.sync_host()
     torch.cuda.synchronize()
     if world > 1:
@@ -435,61 +560,39 @@ def _end_to_end(torch, dist, rnd, pool, rule_for, K, world, dev, M, d, D32) -> d
     s2, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s2.record()
     for i in range(Ke):
-        res = rnd.step_host(host[i % 2], rule_for(i + 1), SEED, i)
+        res = rnd.step_host(host, rule_b(HEADLINE_B, i + 1), SEED, i)
     rnd.join_host()                        # the last download ends inside the timed region
     e2.record()
     rnd.sync_host()
     torch.cuda.synchronize()
     checksum = float(res[:1024].double().abs().sum())        # the result is read on the host
-    ms2 = s2.elapsed_time(e2)
-    ms2 = replicas.max_over_ranks(ms2, dev)
+    ms2 = replicas.max_over_ranks(s2.elapsed_time(e2), dev)
     return {"value": replicas.whole_job_rate(4.0 * M * d * Ke, world, ms2) / 1e9, "unit": UNIT,
             "h2d_bytes_per_step": 4 * M * D32, "d2h_bytes_per_step": 4 * D32, "steps": Ke,
-            "ms_per_step": ms2 / Ke, "checksum": checksum}
+            "ms_per_step": ms2 / Ke, "checksum": checksum,
+            "api": "pipeline.Round.step_host: pinned host gradients in, averaged gradient back in pinned host memory"}
 
 
-def _cpu_baseline(pool, w, eps_hat, alpha) -> dict:
-    """The CPU checker timed on full steps of the same workload (same arrays): as many steps as
-    fit about twelve seconds, at least two."""
-    import numpy as np
-
-    import oracle
-    ref = oracle.Layout(w.segments, w.bucket)
-    cores = os.cpu_count() or 1
-    oracle.set_threads(cores)
-    grads = [pool[p].cpu().numpy() for p in range(min(4, len(pool)))]
-    steps, dt = 0, 0.0
-    while steps < 2 or (dt < 12.0 and steps < 64):
-        t0 = time.perf_counter()
-        _oracle_round(oracle, np, w, ref, grads[steps % len(grads)], steps % w.T, eps_hat, alpha)
-        dt += time.perf_counter() - t0
-        steps += 1
-    out = {"value": 4.0 * w.M * w.d * steps / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
-           "sample": "%d full steps (all %d workers, all %d tensors, t = 0..%d), %.1f s"
-                     % (steps, w.M, len(w.segments), steps - 1, dt)}
-    # the same checker on one thread, on one worker's share of a step
-    import copy
-    w1 = copy.copy(w)
-    w1.M = 1
-    oracle.set_threads(1)
-    t0 = time.perf_counter()
-    _oracle_round(oracle, np, w1, ref, grads[0][:1], 0, eps_hat, alpha)
-    dt1 = time.perf_counter() - t0
-    oracle.set_threads(cores)
-    out["one_thread"] = {"value": 4.0 * w.d / dt1 / 1e9, "unit": UNIT, "cores": 1,
-                         "sample": "one step of one worker (all %d tensors), %.1f s" % (len(w.segments), dt1)}
-    return out
+def _cpu_baseline(torch, gen, dev) -> dict:
+    """The CPU checker timed on whole rounds over a prefix of the same workload (drawn by the same
+    generator): about twelve seconds of work, at least two rounds."""
+    d_sample = 1 << 23
+    g = torch.randn((MAIN_M, d_sample), generator=gen, device=dev, dtype=torch.float32).cpu().numpy()
+    gbs, steps, dt, b, cores = _oracle_rate(g, 12.0, 2, 16)
+    return {"value": gbs, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d whole rounds (norms, bit rule, quantize+pack, unpack+average; b=%d) on 2^23 of the 2^26 elements "
+                      "of all %d workers (1 GiB of gradients per round), %.1f s" % (steps, b, MAIN_M, dt)}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
-    ap.add_argument("--no-four-call", action="store_true", help="skip the secondary timing of the four separate calls")
+    ap.add_argument("--no-models", action="store_true", help="skip the secondary timing of the model-shaped workloads")
     ap.add_argument("--no-overlap", action="store_true",
                     help="run the bit rule after the average on the same stream instead of beside it")
     ap.add_argument("--source-digests", action="store_true",

@@ -35,7 +35,10 @@
  *  - Conditions only the device can see are OR-ed into *dev_status (DQ_STAT_*
  *    bits, a caller-owned int32 the caller zeroes and reads when it wants).
  *    A kernel that raises DQ_STAT_BAD_BITS or DQ_STAT_CAPACITY writes no
- *    output.  No kernel traps or spins without bound.
+ *    output.  No kernel traps or spins without bound: every wait has a time
+ *    limit, a decision to leave after one ran out is taken by all threads that
+ *    later meet at a barrier (a vote or a barrier reduction, never a thread's own
+ *    view), and whoever issued copies waits for them before the CTA ends.
  *  - Data layout ("padded layout"): tensor i of n_i elements starts at element
  *    offset P_i = sum_{j<i} roundup32(n_j) of a worker's fp32 buffer; the
  *    buffer holds D32 = sum_i roundup32(n_i) elements.  Buckets of `bucket`
@@ -333,6 +336,18 @@ int dq_unpack_average_update(const dq_layout_t* layout, const uint32_t* dev_pack
 
 /* Text for a DQ_ERR_* return value (static storage). */
 const char* dq_status_string(int code);
+
+/* Test hook for the bounded waits (no counterpart in the paper).  Every wait of a
+ * kernel for one of its own asynchronous copies is bounded by `limit_ns` of the GPU's
+ * global timer (default 2e9; 0 restores the default).  `first_wait_limit_ns` bounds,
+ * instead, the first such wait of every warp or CTA that consumes copies (UINT64_MAX:
+ * the same as limit_ns).  Setting it to 0 declares those first waits lost at once
+ * although their copies are valid and land a moment later, which exercises what a kernel
+ * does after a time-out -- raise DQ_STAT_WAIT, stop producing output, wait (with
+ * limit_ns) for every copy it has issued, return -- without anything being lost, faulting
+ * or hanging.  Host state of the library, read when a call is made; not for production
+ * use (outputs of a call made under it are incomplete). */
+void dq_debug_set_wait_limits(uint64_t limit_ns, uint64_t first_wait_limit_ns);
 
 #ifdef __cplusplus
 }

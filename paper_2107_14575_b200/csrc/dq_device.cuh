@@ -80,6 +80,52 @@ __device__ __forceinline__ float finish(const float a)
     else return a;
 }
 
+// ---- l2 norms of buckets whose squares leave the fp32 range ---------------------------------
+// The sum of squares S of a bucket, accumulated with fused multiply-adds, is taken as it is when
+// 2^-100 <= S < inf: no square overflowed, every term that fell into the subnormal range (or
+// vanished) is below 2^-126 and so below 2^-26 of S, and sqrt(S) >= 2^-50 dominates each of
+// those entries while sqrt(fl(g^2)) = |g| for the others.  Outside that range (a bucket of tiny
+// entries, an overflowed square, a NaN) the bucket is reduced again: first its largest magnitude
+// (exact), then the squares of the entries scaled by the power of two that brings that magnitude
+// into [1, 2), in the same order as before, and the square root is scaled back.  The functors
+// below are the three reductions; the kernels supply the loads and the joins between threads.
+__device__ __forceinline__ bool l2_sum_in_range(const float sum)
+{
+    return sum >= 0x1p-100f && sum <= 3.402823466e38f;       // false for a NaN as well
+}
+struct SumSquares {
+    __device__ __forceinline__ float take(const float acc, const float x) const { return fmaf(x, x, acc); }
+    __device__ __forceinline__ float join(const float a, const float b) const { return a + b; }
+};
+struct MaxMagnitude {
+    __device__ __forceinline__ float take(const float acc, const float x) const { return max_nan(acc, fabsf(x)); }
+    __device__ __forceinline__ float join(const float a, const float b) const { return max_nan(a, b); }
+};
+struct ScaledSquares {
+    int e;                          // the entries are multiplied by 2^-e first (exact, or negligible when it underflows)
+    __device__ __forceinline__ float take(const float acc, const float x) const
+    {
+        const float y = scalbnf(x, -e);
+        return fmaf(y, y, acc);
+    }
+    __device__ __forceinline__ float join(const float a, const float b) const { return a + b; }
+};
+// the reduction a member of the family starts with
+template <int P> struct FamilyReduction { using type = SumSquares; };
+template <> struct FamilyReduction<DQ_NORM_LINF> { using type = MaxMagnitude; };
+// Exponent to scale by, from the bucket's largest magnitude (0 when there is nothing to scale:
+// an all-zero bucket, an infinity or a NaN, for which rescaled_l2 returns the magnitude itself).
+__device__ __forceinline__ bool magnitude_scalable(const float mx) { return mx > 0.0f && mx <= 3.402823466e38f; }
+__device__ __forceinline__ int scale_exponent(const float mx) { return magnitude_scalable(mx) ? ilogbf(mx) : 0; }
+// The norm from the largest magnitude and the scaled sum of squares.  An overflow of the
+// result (entries near the top of the fp32 range) gives infinity, as the fp64 definition
+// rounded to fp32 does.
+__device__ __forceinline__ float rescaled_l2(const float mx, const float scaled_sum, const int e)
+{
+    if (!magnitude_scalable(mx)) return mx;                  // 0, infinity or NaN
+    return scalbnf(sqrtf(scaled_sum), e);
+}
+
 // (a & mask) | c as one three-input logic operation.  `c` must come from a register the
 // compiler cannot fold (callers pass the exponent pattern of 2^23 from a kernel
 // argument), otherwise two immediates would cost two instructions.

@@ -69,7 +69,48 @@ struct FusedArgs {
     int32_t gpb_shift;            // log2(groups per bucket)
     int32_t stream_reads;         // 1: the gradients exceed the L2, read them with the evict-first policy
     uint32_t one_bits;            // 0x3F800040, kept out of the compiler's sight (see and_or)
+    WaitLimits wait;
 };
+
+// ---- l2 norm of a bucket whose fp32 sum of squares is out of range (see l2_sum_in_range) ----
+// One reduction of the row at byte offset `own` of the shared memory (swizzle phase folded in:
+// chunk c sits at own ^ (c << 4)) over the `gpb` lanes of the row's bucket, in the order of the
+// sum of squares it replaces: four accumulators per row, a pairwise join, the xor butterfly.
+template <class R>
+__device__ __forceinline__ float reduce_row_team(const R& red, const uint32_t own, const int valid, const int gpb)
+{
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    if (valid == 32) {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            const float4 x = *reinterpret_cast<const float4*>(smem + (own ^ (uint32_t)(c << 4)));
+            a0 = red.take(a0, x.x); a1 = red.take(a1, x.y); a2 = red.take(a2, x.z); a3 = red.take(a3, x.w);
+        }
+    } else {
+        for (int e = 0; e < valid; ++e) {
+            const float x = *reinterpret_cast<const float*>(smem + (own ^ (uint32_t)((e >> 2) << 4)) + ((e & 3) << 2));
+            a0 = red.take(a0, x);
+        }
+    }
+    float v = red.join(red.join(a0, a1), red.join(a2, a3));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float other = __shfl_xor_sync(0xffffffffu, v, o);
+        if (o < gpb) v = red.join(v, other);
+    }
+    return v;
+}
+
+// Called by the whole warp when some bucket of its tile is out of range; a lane whose own bucket
+// was in range keeps `nrm`.  Out of line: the common case does not pay for its registers.
+__device__ __noinline__ float rescaled_team_norm(const uint32_t own, const int valid, const int gpb, const float sum,
+                                                 const float nrm)
+{
+    const float mx = reduce_row_team(MaxMagnitude{}, own, valid, gpb);
+    const int e = scale_exponent(mx);
+    const float scaled = reduce_row_team(ScaledSquares{e}, own, valid, gpb);
+    return l2_sum_in_range(sum) ? nrm : rescaled_l2(mx, scaled, e);
+}
 
 // ---- buckets that fit one warp: a tile that touches the end of a tensor ---------------
 // General route of the per-warp pipelines, kept out of line so that the common case does
@@ -138,7 +179,12 @@ __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* ba
         const float other = __shfl_xor_sync(0xffffffffu, sum, o);
         if (o < gpb) sum = join<P>(sum, other);
     }
-    const float nrm = finish<P>(sum);
+    float nrm = finish<P>(sum);
+    if constexpr (P == DQ_NORM_L2) {
+        if (__any_sync(0xffffffffu, !l2_sum_in_range(sum)))
+            nrm = rescaled_team_norm((uint32_t)(base - smem) + (uint32_t)(row * 128 + ((row & 7) << 4)), valid, gpb, sum,
+                                     nrm);
+    }
     int bad = 0;
     if (l == 0 && k < nb) {
         a.norms[(int64_t)m * nb + k] = nrm;
@@ -276,8 +322,12 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
         // warp-level synchronisations below are always reached by all lanes or by none
-        if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, st), (it / kWStages) & 1))) { timed_out = true; break; }
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, st), (it / kWStages) & 1, it == 0 ? a.wait.first_ns : a.wait.ns))) {
+            timed_out = true;
+            break;
+        }
 
+        bool done = false;
         if (regular) {
             // ---- norm of the bucket (same operations, same order as dq_bucket_norms)
             const uint32_t own = own_row0 + (uint32_t)(st * kWTileBytes);
@@ -294,6 +344,10 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 if (o < gpb) sum = join<P>(sum, other);
             }
             const float nrm = finish<P>(sum);
+            // a tile with an l2 sum out of range (see l2_sum_in_range) goes to the general route, which
+            // reduces such buckets a second time; the vote keeps the warp together
+            if (P == DQ_NORM_L2 && __any_sync(0xffffffffu, !l2_sum_in_range(sum))) goto general_route;
+            done = true;
             if (l == 0) {
                 a.norms[(int64_t)m * nb + (kt * R + r)] = nrm;
                 bad |= !isfinite(nrm);
@@ -345,7 +399,9 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 }
                 span = 0;
             }
-        } else {
+        }
+    general_route:
+        if (!done) {
             const int res = irregular_tile<B, P>(a, base, row0, m, kt);
             span = res & 0xff;
             bad |= (res >> 8) != 0;
@@ -383,9 +439,10 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
     if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
     if (timed_out) {
         if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
-        // give copies still in flight a bounded chance to land before the CTA's shared memory is released
-        for (int j = it + 1; j < it + kWStages; ++j)
-            if (j < n_tiles) (void)tma::mbar_wait(wbar(warp, j % kWStages), (j / kWStages) & 1);
+        // every copy the warp has issued and not seen land, the one whose wait ran out included, gets the
+        // full limit before the CTA's shared memory is released
+        for (int j = it; j < it + kWStages; ++j)
+            if (j < n_tiles) (void)tma::mbar_wait(wbar(warp, j % kWStages), (j / kWStages) & 1, a.wait.ns);
     }
 }
 
@@ -497,24 +554,46 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
     const uint32_t own = (uint32_t)(lane * 128 + ((lane & 7) << 4));
 
     // sum of squares (or maximum) of the lane's row of a stage, same operations and order as dq_bucket_norms
-    auto row_reduce = [&](const unsigned char* base, int valid) -> float {
+    auto row_reduce = [&](const auto& red, const unsigned char* base, int valid) -> float {
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         if (valid == 32) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const float4 x = *reinterpret_cast<const float4*>(base + (own ^ (uint32_t)(c << 4)));
-                a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
+                a0 = red.take(a0, x.x); a1 = red.take(a1, x.y); a2 = red.take(a2, x.z); a3 = red.take(a3, x.w);
             }
         } else {
             for (int e = 0; e < valid; ++e) {
                 const float x = *reinterpret_cast<const float*>(base + (own ^ (uint32_t)((e >> 2) << 4)) + ((e & 3) << 2));
-                a0 = take<P>(a0, x);
+                a0 = red.take(a0, x);
             }
         }
-        float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
+        float sum = red.join(red.join(a0, a1), red.join(a2, a3));
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sum = join<P>(sum, __shfl_xor_sync(0xffffffffu, sum, o));
+        for (int o = 16; o > 0; o >>= 1) sum = red.join(sum, __shfl_xor_sync(0xffffffffu, sum, o));
         return sum;
+    };
+    // One reduction of the bucket: the warp's two halves and, for a pair of warps, the exchange of
+    // the four partial results (every exchange is one phase of the pair's barrier and uses the
+    // slot of that phase's parity).  False if the wait for the other warp ran out.
+    uint32_t exchanges = 0;
+    auto bucket_reduce = [&](const auto& red, int rows, int valid_a, int valid_b, float& result) -> bool {
+        const float part_a = rows > 0 ? row_reduce(red, wstage(warp, 0), valid_a) : 0.0f;
+        const float part_b = rows > 32 ? row_reduce(red, wstage(warp, 1), valid_b) : 0.0f;
+        if constexpr (H == 1) {
+            result = red.join(red.join(0.0f, part_a), part_b);
+        } else {
+            float* slot = pair_part + (exchanges & 1u) * 4;
+            if (lane == 0) {
+                slot[2 * sub] = part_a;
+                slot[2 * sub + 1] = part_b;
+                tma::mbar_arrive(pair_bar);
+            }
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(pair_bar, exchanges & 1u, a.wait.ns))) return false;
+            ++exchanges;
+            result = red.join(red.join(red.join(red.join(0.0f, slot[0]), slot[1]), slot[2]), slot[3]);
+        }
+        return true;
     };
     // encodes the lane's row of a stage against `inv`, stages the half's words in the stage itself and
     // sends them to the packed stream; `row0` is the half's first group, `span` its number of groups
@@ -574,11 +653,14 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         }
 
         if (rows > 0) {
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u, it == 0 ? a.wait.first_ns : a.wait.ns))) {
+                timed_out = true;
+                break;
+            }
             pend_a = false; ++ph_a;
         }
         if (rows > 32) {
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 1), ph_b & 1u))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait.ns))) { timed_out = true; break; }
             pend_b = false; ++ph_b;
         }
         int valid_a = len - lane * 32;
@@ -586,20 +668,18 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         int valid_b = len - (lane + 32) * 32;
         valid_b = valid_b < 0 ? 0 : (valid_b > 32 ? 32 : valid_b);
 
-        const float part_a = rows > 0 ? row_reduce(wstage(warp, 0), valid_a) : 0.0f;
-        const float part_b = rows > 32 ? row_reduce(wstage(warp, 1), valid_b) : 0.0f;
-        float nrm;
-        if constexpr (H == 1) {
-            nrm = finish<P>(join<P>(join<P>(0.0f, part_a), part_b));
-        } else {
-            float* slot = pair_part + (it & 1) * 4;
-            if (lane == 0) {
-                slot[2 * sub] = part_a;
-                slot[2 * sub + 1] = part_b;
-                tma::mbar_arrive(pair_bar);
+        float sum;
+        if (!bucket_reduce(typename FamilyReduction<P>::type{}, rows, valid_a, valid_b, sum)) { timed_out = true; break; }
+        float nrm = finish<P>(sum);
+        if constexpr (P == DQ_NORM_L2) {
+            // every lane of the warp, and both warps of a pair, hold the same sum: the verdict is uniform
+            if (!l2_sum_in_range(sum)) {
+                float mx, scaled;
+                if (!bucket_reduce(MaxMagnitude{}, rows, valid_a, valid_b, mx)) { timed_out = true; break; }
+                const int e = scale_exponent(mx);
+                if (!bucket_reduce(ScaledSquares{e}, rows, valid_a, valid_b, scaled)) { timed_out = true; break; }
+                nrm = rescaled_l2(mx, scaled, e);
             }
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(pair_bar, (uint32_t)it & 1u))) { timed_out = true; break; }
-            nrm = finish<P>(join<P>(join<P>(join<P>(join<P>(0.0f, slot[0]), slot[1]), slot[2]), slot[3]));
         }
         if (lane == 0 && sub == 0) {
             a.norms[(int64_t)m * nb + k] = nrm;
@@ -624,9 +704,10 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
     if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
     if (timed_out) {
         if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
-        // give copies still in flight a bounded chance to land before the CTA's shared memory is released
-        if (pend_a) (void)tma::mbar_wait(wbar(warp, 0), ph_a & 1u);
-        if (pend_b) (void)tma::mbar_wait(wbar(warp, 1), ph_b & 1u);
+        // every copy the warp has issued and not seen land, the one whose wait ran out included, gets the
+        // full limit before the CTA's shared memory is released
+        if (pend_a) (void)tma::mbar_wait(wbar(warp, 0), ph_a & 1u, a.wait.ns);
+        if (pend_b) (void)tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait.ns);
     }
 }
 
@@ -709,6 +790,7 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
     a.worker0 = first_worker;
     a.M = M;
     a.one_bits = 0x3F800040u;
+    a.wait = dq_wait_limits();
     a.gpb_shift = 0;
     while ((1u << a.gpb_shift) < gpb) ++a.gpb_shift;
     a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;

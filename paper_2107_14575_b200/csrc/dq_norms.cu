@@ -17,6 +17,26 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kRun = 8;            // bucket rows a warp handles per run
 
+// l2 norm of a bucket whose fp32 sum of squares is out of range (see l2_sum_in_range), read
+// again with plain loads by its team of LANES lanes: largest magnitude first, then the squares of
+// the scaled entries.  Called by all lanes of the warp; out of line, it is rarely needed.
+template <int LANES>
+__device__ __noinline__ float rescaled_norm_global(const float* __restrict__ g, const int len, const int lane)
+{
+    const MaxMagnitude mag;
+    float mx = 0.f;
+    for (int i = lane; i < len; i += LANES) mx = mag.take(mx, __ldg(g + i));
+#pragma unroll
+    for (int o = LANES / 2; o > 0; o >>= 1) mx = mag.join(mx, __shfl_xor_sync(0xffffffffu, mx, o, LANES));
+    const int e = scale_exponent(mx);
+    const ScaledSquares sq{e};
+    float ss = 0.f;
+    for (int i = lane; i < len; i += LANES) ss = sq.take(ss, __ldg(g + i));
+#pragma unroll
+    for (int o = LANES / 2; o > 0; o >>= 1) ss = sq.join(ss, __shfl_xor_sync(0xffffffffu, ss, o, LANES));
+    return rescaled_l2(mx, ss, e);
+}
+
 template <int LANES, int P>
 __global__ void __launch_bounds__(kThreads)
 bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const int64_t worker_stride,
@@ -88,8 +108,14 @@ bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const i
             float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
 #pragma unroll
             for (int o = LANES / 2; o > 0; o >>= 1) sum = join<P>(sum, __shfl_xor_sync(0xffffffffu, sum, o, LANES));
+            float nrm = finish<P>(sum);
+            if constexpr (P == DQ_NORM_L2) {
+                if (__any_sync(0xffffffffu, active && !l2_sum_in_range(sum))) {
+                    const float again = rescaled_norm_global<LANES>(g, len, lane);
+                    if (!l2_sum_in_range(sum)) nrm = again;
+                }
+            }
             if (lane == 0 && active) {
-                const float nrm = finish<P>(sum);
                 nw[k] = nrm;
                 bad |= !isfinite(nrm);
             }
@@ -207,8 +233,21 @@ bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, co
         }
         t = join<P>(t, __shfl_xor_sync(0xffffffffu, t, 8));
         t = join<P>(t, __shfl_xor_sync(0xffffffffu, t, 16));
+        float nrm = finish<P>(t);
+        if constexpr (P == DQ_NORM_L2) {
+            // lane r holds bucket r of the run: the buckets out of range are taken again one by one
+            const unsigned need = __ballot_sync(0xffffffffu, lane < kRun && k0 + lane < v.nb && !l2_sum_in_range(t));
+            if (need) {
+#pragma unroll
+                for (int r = 0; r < kRun; ++r) {
+                    if ((need >> r) & 1u) {
+                        const float again = rescaled_norm_global<32>(gw + (int64_t)first[r] * 4, len[r], lane);
+                        if (lane == r) nrm = again;
+                    }
+                }
+            }
+        }
         if (lane < kRun && k0 + lane < v.nb) {
-            const float nrm = finish<P>(t);
             nw[k0 + lane] = nrm;
             bad |= !isfinite(nrm);
         }
@@ -231,8 +270,9 @@ constexpr int kTmaTileBytes = kTmaThreads * 128;
 constexpr int kTmaMaxSmemSegs = 1023;
 
 extern __shared__ __align__(1024) unsigned char smem[];
-constexpr int kPartOffset = kTmaStages * kTmaTileBytes;          // 4 floats: per-warp partial sums
-constexpr int kBarOffset = kPartOffset + 16;
+constexpr int kPartOffset = kTmaStages * kTmaTileBytes;          // 4 floats: per-warp partial results
+constexpr int kAbortOffset = kPartOffset + 16;                   // set by a thread whose wait ran out
+constexpr int kBarOffset = kPartOffset + 32;
 constexpr int kTblOffset = kBarOffset + kTmaStages * 8;
 
 __device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
@@ -246,12 +286,10 @@ struct NormsArgs {
     int32_t map_has_worker_dim;
     int32_t gpb_shift;           // log2(groups per bucket)
     int32_t stream_reads;        // 1: the gradients exceed the L2, read them with the evict-first policy
+    WaitLimits wait;
 };
 
-// RAW: the kernel writes the unfinished reduction (sum of squares, or maximum) of every
-// bucket instead of its norm -- the first step of dq_tensor_norms, whose "buckets" are the
-// 4096-element pieces of the tensors.
-template <int P, bool RAW>
+template <int P>
 __global__ void __launch_bounds__(kTmaThreads)
 bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_constant__ CUtensorMap map)
 {
@@ -266,11 +304,13 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
     int32_t* tbl_s = reinterpret_cast<int32_t*>(smem + kTblOffset);
     if (tbl_in_smem)
         for (int i = tid; i < 3 * n1; i += kTmaThreads) tbl_s[i] = __ldg(a.v.seg_group0 + i);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kAbortOffset);
     if (tid == 0) {
         tma::prefetch_tensor_map(&map);
 #pragma unroll
         for (int st = 0; st < kTmaStages; ++st) tma::mbar_init(full_bar(st), 1);
         tma::fence_barrier_init();
+        *abort_flag = 0;
     }
     __syncthreads();
     auto tbl = [&](int i) -> int { return tbl_in_smem ? tbl_s[i] : __ldg(a.v.seg_group0 + i); };
@@ -343,42 +383,73 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
         int valid = len - l * 32;                // elements of its group that count
         valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
 
-        if (!tma::mbar_wait(full_bar(st), (it / kTmaStages) & 1)) { timed_out = true; break; }
+        // A thread whose wait runs out says so in shared memory and goes on (what it reads from the
+        // stage is then arbitrary, and unused): every thread reaches the barriers below, after which all
+        // of them see the flag and leave together.
+        const bool landed = tma::mbar_wait(full_bar(st), (it / kTmaStages) & 1, it == 0 ? a.wait.first_ns : a.wait.ns);
+        if (!landed) *abort_flag = 1;
 
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        if (valid > 0) {
-            const unsigned char* base = smem + st * kTmaTileBytes;
-            if (valid == 32) {
+        // One reduction of the tile: the gpb threads of a bucket combine inside a warp by shuffles and
+        // across the warps of a bucket through shared memory; the result counts in the threads with l == 0
+        // (in all threads of the bucket when it lies inside one warp).
+        const unsigned char* base = smem + st * kTmaTileBytes;
+        auto tile_reduce = [&](const auto& red) -> float {
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            if (valid > 0) {
+                if (valid == 32) {
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
-                    a0 = take<P>(a0, x.x); a1 = take<P>(a1, x.y); a2 = take<P>(a2, x.z); a3 = take<P>(a3, x.w);
-                }
-            } else {                             // last group of a tensor: what follows is padding
-                for (int e = 0; e < valid; ++e) {
-                    const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
-                    a0 = take<P>(a0, x);
+                    for (int c = 0; c < 8; ++c) {
+                        const float4 x = *reinterpret_cast<const float4*>(base + tma::swizzle128(row, c));
+                        a0 = red.take(a0, x.x); a1 = red.take(a1, x.y); a2 = red.take(a2, x.z); a3 = red.take(a3, x.w);
+                    }
+                } else {                             // last group of a tensor: what follows is padding
+                    for (int e = 0; e < valid; ++e) {
+                        const float x = *reinterpret_cast<const float*>(base + tma::swizzle128(row, e >> 2) + ((e & 3) << 2));
+                        a0 = red.take(a0, x);
+                    }
                 }
             }
-        }
-        float sum = join<P>(join<P>(a0, a1), join<P>(a2, a3));
-        // combine the gpb threads of a bucket: inside a warp by shuffles ...
-        const int w = gpb < 32 ? gpb : 32;
-        for (int o = w >> 1; o > 0; o >>= 1) sum = join<P>(sum, __shfl_xor_sync(0xffffffffu, sum, o));
-        if (gpb > 32) {                          // ... and across the warps of a bucket through shared memory
-            if (lane == 0) part[warp] = sum;
-            __syncthreads();
-            if (l == 0) {
-                sum = 0.f;
-                for (int i = 0; i < (gpb >> 5); ++i) sum = join<P>(sum, part[(tid >> 5) + i]);
+            float v = red.join(red.join(a0, a1), red.join(a2, a3));
+            const int w = gpb < 32 ? gpb : 32;
+            for (int o = w >> 1; o > 0; o >>= 1) v = red.join(v, __shfl_xor_sync(0xffffffffu, v, o));
+            if (gpb > 32) {
+                if (lane == 0) part[warp] = v;
+                __syncthreads();
+                if (l == 0) {
+                    v = 0.f;
+                    for (int i = 0; i < (gpb >> 5); ++i) v = red.join(v, part[(tid >> 5) + i]);
+                }
+            }
+            return v;
+        };
+        const float sum = tile_reduce(typename FamilyReduction<P>::type{});
+        float nrm = finish<P>(sum);
+        const bool writes = (l == 0 && k < nb);
+        const bool out_of_range = (P == DQ_NORM_L2) && writes && !l2_sum_in_range(sum);
+        // after this barrier everyone is done with the stage and with part[]
+        if (__syncthreads_or(out_of_range || !landed)) {
+            if (*abort_flag) { timed_out = true; break; }
+            if constexpr (P == DQ_NORM_L2) {
+                // some bucket of the tile needs the rescaled reduction (see l2_sum_in_range): the whole
+                // CTA takes it, the buckets that were in range keep their norm
+                float mx = tile_reduce(MaxMagnitude{});
+                if (gpb > 32) {                  // the bucket's largest magnitude, for all of its threads
+                    __syncthreads();
+                    if (l == 0) part[warp] = mx;
+                    __syncthreads();
+                    mx = part[(tid >> a.gpb_shift) << (a.gpb_shift - 5)];
+                    __syncthreads();
+                }
+                const int e = scale_exponent(mx);
+                const float scaled = tile_reduce(ScaledSquares{e});
+                if (out_of_range) nrm = rescaled_l2(mx, scaled, e);
+                __syncthreads();
             }
         }
-        if (l == 0 && k < nb) {
-            const float nrm = RAW ? sum : finish<P>(sum);
+        if (writes) {
             a.norms[(int64_t)m * nb + k] = nrm;
             bad |= !isfinite(nrm);
         }
-        __syncthreads();                         // everyone is done with this stage (and with part[])
         if (ptile < tile_end && tid == 0) issue(st);
         ++ptile;
         advance(pm, pkt);
@@ -386,16 +457,19 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
     if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
     if (timed_out) {
         if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
-        for (int j = it + 1; j < it + kTmaStages; ++j)
-            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kTmaStages), (j / kTmaStages) & 1);
+        // every copy already issued, the one whose wait ran out included, gets the full limit to land
+        // before the CTA's shared memory is released
+        for (int j = it; j < it + kTmaStages; ++j)
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kTmaStages), (j / kTmaStages) & 1, a.wait.ns);
     }
 }
 
-// Second step of dq_tensor_norms: block (tensor, worker) reduces the unfinished results of the
-// tensor's pieces in a fixed order -- thread t takes pieces t, t + 256, ..., then a tree over the
-// block -- and writes the tensor's norm.  Sums of squares are added in fp64 and rounded to fp32
-// before the square root, which keeps norm >= |g_j| for every entry (each piece's sum is at
-// least fl(g_j^2), rounding is monotone, and sqrtf(fl(g^2)) = |g|).
+// Second step of dq_tensor_norms: block (tensor, worker) joins the norms of the tensor's pieces in
+// a fixed order -- thread t takes pieces t, t + 256, ..., then a tree over the block -- and writes
+// the tensor's norm.  l2: the squares of the piece norms are exact in fp64 and cannot leave its
+// range; their sum is at least p^2 for every piece norm p, the fp64 square root is monotone and
+// gives back p for p^2, and so is the rounding to fp32, which has p among its values: the tensor's
+// norm is at least every piece norm, which in turn is at least every entry of the piece.
 constexpr int kJoinThreads = 256;
 
 template <int P>
@@ -420,7 +494,10 @@ tensor_norms_join_kernel(const int32_t n_seg, const int32_t* __restrict__ piece0
     float nrm;
     if constexpr (P == DQ_NORM_L2) {
         double acc = 0.0;
-        for (int i = c0 + tid; i < c1; i += kJoinThreads) acc += (double)__ldg(src + i);
+        for (int i = c0 + tid; i < c1; i += kJoinThreads) {
+            const double p = (double)__ldg(src + i);
+            acc = fma(p, p, acc);
+        }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (lane == 0) part_d[warp] = acc;
@@ -428,7 +505,7 @@ tensor_norms_join_kernel(const int32_t n_seg, const int32_t* __restrict__ piece0
         if (tid != 0) return;
         double total = 0.0;
         for (int w = 0; w < kJoinThreads / 32; ++w) total += part_d[w];
-        nrm = sqrtf((float)total);
+        nrm = (float)sqrt(total);
     } else {
         float acc = 0.0f;
         for (int i = c0 + tid; i < c1; i += kJoinThreads) acc = max_nan(acc, __ldg(src + i));
@@ -446,7 +523,7 @@ tensor_norms_join_kernel(const int32_t n_seg, const int32_t* __restrict__ piece0
 }
 
 // Launch of the bulk-copy kernel over view `v` (groups per bucket a power of two, at most 128).
-template <int P, bool RAW>
+template <int P>
 int launch_tma(const dq_layout_t* L, const LayoutView& v, const float* dev_grads, int64_t worker_stride_elems, int32_t M,
                float* dev_out, int32_t* dev_status, cudaStream_t st)
 {
@@ -460,6 +537,7 @@ int launch_tma(const dq_layout_t* L, const LayoutView& v, const float* dev_grads
     a.gpb_shift = 0;
     while ((1u << a.gpb_shift) < gpb) ++a.gpb_shift;
     a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
+    a.wait = dq_wait_limits();
     const bool worker_dim = (M > 1 && worker_stride_elems != 0);
     a.map_has_worker_dim = worker_dim ? 1 : 0;
     CUtensorMap map;
@@ -471,7 +549,7 @@ int launch_tma(const dq_layout_t* L, const LayoutView& v, const float* dev_grads
         return DQ_ERR_CUDA;
     size_t smem_need = (size_t)kTblOffset;
     if (L->n_seg > 1 && L->n_seg <= kTmaMaxSmemSegs) smem_need += (size_t)3 * (L->n_seg + 1) * 4;
-    if (cudaFuncSetAttribute(bucket_norms_tma_kernel<P, RAW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
+    if (cudaFuncSetAttribute(bucket_norms_tma_kernel<P>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_need) != cudaSuccess) {
         (void)cudaGetLastError();
         return DQ_ERR_CUDA;
     }
@@ -479,7 +557,7 @@ int launch_tma(const dq_layout_t* L, const LayoutView& v, const float* dev_grads
     const int64_t tiles = (int64_t)M * ((v.nb + R - 1) / R);
     int64_t blocks = (int64_t)dq_sm_count() * 3;    // three 65 KB CTAs per SM
     if (blocks > tiles) blocks = tiles;
-    dq_launch(bucket_norms_tma_kernel<P, RAW>, dim3((unsigned)blocks), dim3(kTmaThreads), smem_need, st, a, map);
+    dq_launch(bucket_norms_tma_kernel<P>, dim3((unsigned)blocks), dim3(kTmaThreads), smem_need, st, a, map);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
 }
@@ -539,8 +617,8 @@ extern "C" int dq_bucket_norms(const dq_layout_t* L, const float* dev_grads, int
     const bool linf = (L->norm == DQ_NORM_LINF);
     if ((gpb & (gpb - 1)) == 0) {
         // bucket = 32 * 2^k: bulk-copy kernel
-        return linf ? launch_tma<DQ_NORM_LINF, false>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st)
-                    : launch_tma<DQ_NORM_L2, false>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st);
+        return linf ? launch_tma<DQ_NORM_LINF>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st)
+                    : launch_tma<DQ_NORM_L2>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st);
     }
     return linf ? launch_plain<DQ_NORM_LINF>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st)
                 : launch_plain<DQ_NORM_L2>(L, v, dev_grads, worker_stride_elems, M, dev_norms, dev_status, st);
@@ -567,8 +645,8 @@ extern "C" int dq_tensor_norms(const dq_layout_t* L, const float* dev_grads, int
     float* partial = static_cast<float*>(dev_scratch);
     const LayoutView pv = make_piece_view(L);
     const bool linf = (L->norm == DQ_NORM_LINF);
-    const int r1 = linf ? launch_tma<DQ_NORM_LINF, true>(L, pv, dev_grads, worker_stride_elems, M, partial, dev_status, st)
-                        : launch_tma<DQ_NORM_L2, true>(L, pv, dev_grads, worker_stride_elems, M, partial, dev_status, st);
+    const int r1 = linf ? launch_tma<DQ_NORM_LINF>(L, pv, dev_grads, worker_stride_elems, M, partial, dev_status, st)
+                        : launch_tma<DQ_NORM_L2>(L, pv, dev_grads, worker_stride_elems, M, partial, dev_status, st);
     if (r1 != DQ_OK) return r1;
     const int32_t n1 = L->n_seg + 1;
     const int32_t* piece0 = L->n_seg > 1 ? L->dev_table + 4 * n1 : nullptr;

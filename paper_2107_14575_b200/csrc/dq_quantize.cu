@@ -59,6 +59,7 @@ struct QuantizeArgs {
     int32_t div_shift;            // >= 0: power of two, shift; < 0: use div_magic with a 33-bit shift
     int32_t stream_reads;         // 1: the gradients exceed the L2, read them with the evict-first policy
     uint32_t one_bits;            // 0x3F800040 = bits of 1 + 2^-17, kept out of the compiler's sight (see and_or)
+    WaitLimits wait;
 };
 
 __device__ __forceinline__ uint32_t div_gpb(const QuantizeArgs& a, uint32_t n)
@@ -167,7 +168,10 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
         // warp-level synchronisations below are always reached by all lanes or by none
-        if (!__all_sync(0xffffffffu, tma::mbar_wait(full_bar(warp, st), parity))) { timed_out = true; break; }
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(full_bar(warp, st), parity, it == 0 ? a.wait.first_ns : a.wait.ns))) {
+            timed_out = true;
+            break;
+        }
 
         unsigned char* tile_base = stage_ptr(warp, st);
         unsigned char* row = tile_base + lane * 128;
@@ -216,10 +220,11 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
 
     if (timed_out) {
         if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
-        // give copies still in flight a bounded chance to land before the CTA's shared memory is released
-        for (int k = 1; k < kStages; ++k) {
+        // every copy the warp has issued and not seen land, the one whose wait ran out included, gets the
+        // full limit before the CTA's shared memory is released
+        for (int k = 0; k < kStages; ++k) {
             const int j = it + k;
-            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(warp, j % kStages), (j / kStages) & 1);
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(warp, j % kStages), (j / kStages) & 1, a.wait.ns);
         }
     }
 }
@@ -299,6 +304,7 @@ extern "C" int dq_quantize_pack_worker(const dq_layout_t* L, const float* dev_gr
     a.worker0 = first_worker;
     a.M = M;
     a.one_bits = 0x3F800040u;
+    a.wait = dq_wait_limits();
     a.stream_reads = ((int64_t)M * L->padded * 4 > (int64_t(64) << 20)) ? 1 : 0;
     const bool worker_dim = (M > 1 && worker_stride_elems != 0);
     a.map_has_worker_dim = worker_dim ? 1 : 0;

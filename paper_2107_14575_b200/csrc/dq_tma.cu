@@ -42,3 +42,22 @@ bool dq_encode_tensor_map(CUtensorMap* map, CUtensorMapDataType type, uint32_t r
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return rc == CUDA_SUCCESS;
 }
+
+// ---- wait limits (see WaitLimits) ----
+namespace {
+std::mutex g_limits_mu;
+WaitLimits g_limits = {2000000000ull, 2000000000ull};
+}  // namespace
+
+WaitLimits dq_wait_limits()
+{
+    std::lock_guard<std::mutex> lock(g_limits_mu);
+    return g_limits;
+}
+
+extern "C" void dq_debug_set_wait_limits(uint64_t limit_ns, uint64_t first_wait_limit_ns)
+{
+    std::lock_guard<std::mutex> lock(g_limits_mu);
+    g_limits.ns = limit_ns ? limit_ns : 2000000000ull;
+    g_limits.first_ns = first_wait_limit_ns == UINT64_MAX ? g_limits.ns : first_wait_limit_ns;
+}

@@ -1,6 +1,6 @@
 // Asynchronous-copy plumbing for sm_100a: mbarriers, bulk copies (TMA) from
 // global to shared memory, and the 128-byte swizzle that TMA tensor copies
-// apply.  No copy here uses cluster multicast.
+// apply.  Every copy here is addressed to the issuing CTA alone.
 #pragma once
 
 #include <cuda.h>
@@ -15,13 +15,22 @@ bool dq_encode_tensor_map(CUtensorMap* map, CUtensorMapDataType type, uint32_t r
                           const uint64_t* dims, const uint64_t* strides_bytes /*rank-1*/, const uint32_t* box,
                           CUtensorMapSwizzle swizzle);
 
+// Upper bounds on the waits for asynchronous copies, in nanoseconds of the global timer; every
+// kernel that waits receives them as an argument.  `ns` bounds every wait (2 s unless
+// dq_debug_set_wait_limits changed it).  `first_ns` bounds the FIRST wait of every consumer
+// (a warp or a CTA, as the kernel is organised) instead: it equals `ns` in normal use, and a test
+// sets it to 0 so that this wait is declared lost at once while its copy is valid and lands a
+// moment later -- the path taken after a time-out then runs with nothing actually lost.  A wait that
+// runs out raises DQ_STAT_WAIT, the CTA waits (with `ns`) for every copy it has issued, and leaves.
+struct WaitLimits {
+    unsigned long long ns;
+    unsigned long long first_ns;
+};
+WaitLimits dq_wait_limits();     // host: the limits the next launches get
+
 #ifdef __CUDACC__
 
 namespace tma {
-
-// Upper bound on any wait for an asynchronous copy, in nanoseconds of the
-// global timer.  A wait that runs out raises DQ_STAT_WAIT and the CTA leaves.
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p)
 {
@@ -79,16 +88,18 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 
-// Waits for the phase with the given parity; false if the time limit ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
+// Waits for the phase with the given parity; false if `limit_ns` ran out.  A limit of 0 declares the
+// wait lost without a look at the barrier (the test hook's deterministic time-out).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const unsigned long long limit_ns)
 {
+    if (limit_ns == 0) return false;
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+        if (global_timer_ns() - t0 > limit_ns) return false;
     }
 }
 

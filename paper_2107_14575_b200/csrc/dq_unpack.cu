@@ -46,13 +46,45 @@ constexpr int kScaleOffset = kStageOffset + kStages * kStageWords * 4;          
 // barriers: kStages "stage filled" (copies landed), kStages "stage drained" (one arrival per
 // consumer warp), then the one of the x tile
 constexpr int kBarOffset = kScaleOffset + kMaxChunk * kThreads * 4;
-constexpr int kTblOffset = kBarOffset + (2 * kStages + 1) * 8;
+// one word that says "a wait ran out": written by whoever notices, read by the copy warp (so that it
+// stops issuing) and fed into the consumers' barrier reductions
+constexpr int kAbortOffset = kBarOffset + (2 * kStages + 1) * 8;
+constexpr int kTblOffset = kAbortOffset + 8;
 
 __device__ __forceinline__ uint64_t* full_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + st; }
 __device__ __forceinline__ uint64_t* empty_bar(int st) { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + kStages + st; }
 __device__ __forceinline__ uint64_t* x_bar() { return reinterpret_cast<uint64_t*>(smem + kBarOffset) + 2 * kStages; }
+__device__ __forceinline__ volatile int* abort_flag() { return reinterpret_cast<volatile int*>(smem + kAbortOffset); }
 // barrier among the consumer warps only (the copy warp runs ahead on its own)
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kThreads) : "memory"); }
+// The same barrier with an OR over the consumers' predicates: every consumer gets the same answer,
+// so a decision to leave taken from it is taken by all of them or by none.
+__device__ __forceinline__ bool consumer_sync_or(const bool pred)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 q, %1, 0;\n\t"
+        "bar.red.or.pred p, 1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "n"(kThreads)
+        : "memory");
+    return r != 0;
+}
+// Wait of the copy warp for a drained stage: as mbar_wait, but it also gives up when the
+// consumers have said that they are leaving.
+__device__ __forceinline__ bool wait_unless_aborted(uint64_t* bar, const uint32_t parity, const unsigned long long limit_ns)
+{
+    if (tma::mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = tma::global_timer_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (tma::mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag() != 0 || tma::global_timer_ns() - t0 > limit_ns) return false;
+    }
+}
 __device__ __forceinline__ uint32_t* stage_words(int st) { return reinterpret_cast<uint32_t*>(smem + kStageOffset) + st * kStageWords; }
 
 struct AverageArgs {
@@ -68,6 +100,7 @@ struct AverageArgs {
     int32_t div_shift;
     uint32_t magic;               // 0x4B000000, kept out of the compiler's sight (see and_or)
     float neg_lr;                 // -eta of the parameter update (update kernel only)
+    WaitLimits wait;
 };
 
 __device__ __forceinline__ uint32_t div_gpb(const AverageArgs& a, uint32_t n)
@@ -198,16 +231,27 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         // the copy warp: unit u goes into stage u % kStages as soon as the consumers have drained
         // what was there (unit u - kStages)
         if (tid == kThreads) {
+            int issued = 0;
             for (int u = 0; u < my_units; ++u) {
                 const int st = u % kStages;
-                if (u >= kStages && !tma::mbar_wait(empty_bar(st), (uint32_t)(u / kStages - 1) & 1u)) {
-                    atomicOr(a.status, DQ_STAT_WAIT);
+                if (u >= kStages && !wait_unless_aborted(empty_bar(st), (uint32_t)(u / kStages - 1) & 1u, a.wait.ns)) {
+                    if (*abort_flag() == 0) {            // nobody drained the stage in time
+                        atomicOr(a.status, DQ_STAT_WAIT);
+                        *abort_flag() = 1;
+                    }
                     break;
                 }
                 const int tile = tile_begin + u / nchunk;
                 const int m0 = (u % nchunk) * MC;
                 issue_unit<B>(a, st, tile * kThreads, m0, (M - m0) < MC ? (M - m0) : MC);
+                issued = u + 1;
             }
+            // Whoever issues copies sees them land: the last copy into each stage is the only one the
+            // consumers may not have waited for (when they left early), and the CTA's shared memory
+            // must not be released under a copy in flight.
+            for (int u = issued > kStages ? issued - kStages : 0; u < issued; ++u)
+                if (!tma::mbar_wait(full_bar(u % kStages), (uint32_t)(u / kStages) & 1u, a.wait.ns))
+                    atomicOr(a.status, DQ_STAT_WAIT);
         }
         return;
     }
@@ -282,11 +326,14 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
             for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j] * unit;
         }
 
+        // A warp whose wait for a stage ran out raises the flag, decodes no more and releases no more
+        // stages; it walks on to the barrier at the tile's end, where all consumers learn of it together
+        // and leave.  (Warps that were still waiting for later stages run into their own limit first.)
         float acc[32];
-        bool timed_out = false;
+        bool timed_out = false, warp_out = false, x_pending = false;
         int u = 0;
         int tiles_done = 0;
-        for (int tile = tile_begin; tile < tile_end && !timed_out; ++tile) {
+        for (int tile = tile_begin; tile < tile_end; ++tile) {
 #pragma unroll
             for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
             for (int c = 0; c < nchunk; ++c, ++u) {
@@ -315,35 +362,45 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                 if constexpr (UPDATE) {
                     // the tile of x travels into the output tile while the codes are decoded; the
                     // previous tile's store must have drained it first
-                    if (c == 0 && tid == 0) {
-                        tma::store_wait_read();
-                        tma::mbar_expect_tx(x_bar(), kOutBytes);
-                        tma::load_tile_2d(smem, out_map, x_bar(), 0, tile * kThreads);
+                    if (c == 0) {
+                        if (tid == 0) {
+                            tma::store_wait_read();
+                            tma::mbar_expect_tx(x_bar(), kOutBytes);
+                            tma::load_tile_2d(smem, out_map, x_bar(), 0, tile * kThreads);
+                        }
+                        x_pending = true;
                     }
                 }
                 const int st = u % kStages;
-                if (!tma::mbar_wait(full_bar(st), (u / kStages) & 1)) { timed_out = true; break; }
-                const uint32_t* base = stage_words(st) + tid * B;
+                if (!warp_out &&
+                    !__all_sync(0xffffffffu, tma::mbar_wait(full_bar(st), (u / kStages) & 1, u == 0 ? a.wait.first_ns : a.wait.ns))) {
+                    warp_out = true;
+                    *abort_flag() = 1;
+                }
+                if (!warp_out) {
+                    const uint32_t* base = stage_words(st) + tid * B;
 #pragma unroll 2
-                for (int j = 0; j < mc; ++j) {
-                    uint32_t wd[B], hi[B];
-                    load_words<B>(base + j * (kThreads * B), wd);
-                    UpperHalves<B, 0>::run(wd, hi);
-                    AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
+                    for (int j = 0; j < mc; ++j) {
+                        uint32_t wd[B], hi[B];
+                        load_words<B>(base + j * (kThreads * B), wd);
+                        UpperHalves<B, 0>::run(wd, hi);
+                        AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
+                    }
                 }
 #pragma unroll
                 for (int j = 0; j < MC; ++j) my_scales[j * kThreads] = nxt[j] * unit;
 
                 // this warp is done with the stage: once all four have said so the copy warp refills it
+                // (a warp whose wait ran out says nothing: the stage's copy may still be on its way, and the
+                // copy warp, which watches the flag, issues no more)
                 __syncwarp();
-                if ((tid & 31) == 0) tma::mbar_arrive(empty_bar(st));
+                if ((tid & 31) == 0 && !warp_out) tma::mbar_arrive(empty_bar(st));
             }
-            if (timed_out) break;
             // the previous tile's bulk store must have drained the output tile before it is rewritten below
             if constexpr (!UPDATE) {
                 if (tid == 0) tma::store_wait_read();
             }
-            consumer_sync();
+            if (consumer_sync_or(warp_out || *abort_flag() != 0)) { timed_out = true; break; }
             Normalise<B, 0>::run(acc);
             if (valid < 32) {
 #pragma unroll
@@ -351,15 +408,18 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                     if (e >= valid) acc[e] = 0.0f;
             }
             // own row of the swizzled output tile (conflict-free), then one bulk tensor store per tile
+            bool x_landed = true;
             if constexpr (UPDATE) {
-                if (!tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u)) { timed_out = true; break; }
-                const float neg_lr = a.neg_lr;
+                x_landed = tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u, a.wait.ns);
+                if (x_landed) {
+                    const float neg_lr = a.neg_lr;
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    float4* p = reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c));
-                    const float4 x = *p;
-                    *p = make_float4(fmaf(neg_lr, acc[4 * c], x.x), fmaf(neg_lr, acc[4 * c + 1], x.y),
-                                     fmaf(neg_lr, acc[4 * c + 2], x.z), fmaf(neg_lr, acc[4 * c + 3], x.w));
+                    for (int c = 0; c < 8; ++c) {
+                        float4* p = reinterpret_cast<float4*>(smem + tma::swizzle128(tid, c));
+                        const float4 x = *p;
+                        *p = make_float4(fmaf(neg_lr, acc[4 * c], x.x), fmaf(neg_lr, acc[4 * c + 1], x.y),
+                                         fmaf(neg_lr, acc[4 * c + 2], x.z), fmaf(neg_lr, acc[4 * c + 3], x.w));
+                    }
                 }
             } else {
 #pragma unroll
@@ -368,7 +428,13 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                         make_float4(acc[4 * c], acc[4 * c + 1], acc[4 * c + 2], acc[4 * c + 3]);
             }
             tma::fence_proxy_async();
-            consumer_sync();
+            if constexpr (UPDATE) {
+                // nothing is stored from a tile whose parameters did not arrive
+                if (consumer_sync_or(!x_landed)) { timed_out = true; break; }
+                x_pending = false;
+            } else {
+                consumer_sync();
+            }
             if (tid == 0) {
                 tma::store_tile_2d(out_map, smem, 0, tile * kThreads);
                 tma::store_commit();
@@ -380,11 +446,13 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
 
         if (tid == 0) tma::store_wait_read();         // shared memory must outlive the last store's reads
         if (timed_out) {
+            // The copy warp stops issuing and sees its own copies land; the consumers' only copy is the
+            // tile of x, which gets the full limit before the shared memory is released.
+            *abort_flag() = 1;
             if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
-            // give copies still in flight a bounded chance to land before the shared memory is released
-            for (int k = 1; k < kStages; ++k)
-                if (u + k < my_units) (void)tma::mbar_wait(full_bar((u + k) % kStages), ((u + k) / kStages) & 1);
-            if constexpr (UPDATE) (void)tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u);
+            if constexpr (UPDATE) {
+                if (x_pending) (void)tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u, a.wait.ns);
+            }
         }
     }
 }
@@ -413,6 +481,7 @@ unpack_average_kernel(const __grid_constant__ AverageArgs a, const __grid_consta
         }
         tma::mbar_init(x_bar(), 1);
         tma::fence_barrier_init();
+        *abort_flag() = 0;
     }
     __syncthreads();
     if (b < 1 || b > DQ_MAX_BITS) {
@@ -467,6 +536,7 @@ int launch_average(const dq_layout_t* L, const uint32_t* dev_packed, int64_t pac
     a.M = M;
     a.magic = 0x4B000000u;
     a.neg_lr = -lr;
+    a.wait = dq_wait_limits();
     const uint32_t gpb = (uint32_t)a.v.groups_per_bucket;
     if ((gpb & (gpb - 1)) == 0) {
         a.div_shift = 0;

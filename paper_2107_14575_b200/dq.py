@@ -27,7 +27,7 @@ SYMBOLS = [
     "dq_bucket_norms", "dq_tensor_norms_scratch_bytes", "dq_tensor_norms", "dq_choose_bits_scratch_bytes", "dq_choose_bits",
     "dq_choose_bits_noalloc_max_norms", "dq_choose_bits_noalloc",
     "dq_quantize_pack", "dq_quantize_pack_worker", "dq_norms_quantize_pack", "dq_norms_quantize_pack_worker", "dq_unpack_dequant_average",
-    "dq_unpack_average_update", "dq_status_string",
+    "dq_unpack_average_update", "dq_status_string", "dq_debug_set_wait_limits",
 ]
 
 
@@ -122,12 +122,19 @@ def lib():
         L.dq_unpack_average_update.argtypes = [vp, vp, i64, vp, i32, vp, C.c_float, vp, vp, vp]
         L.dq_status_string.restype = C.c_char_p
         L.dq_status_string.argtypes = [C.c_int]
+        L.dq_debug_set_wait_limits.restype = None
+        L.dq_debug_set_wait_limits.argtypes = [u64, u64]
         _lib = L
     return _lib
 
 
 def status_string(code: int) -> str:
     return lib().dq_status_string(int(code)).decode()
+
+
+def debug_set_wait_limits(limit_ns: int = 0, first_wait_limit_ns: int = 2 ** 64 - 1) -> None:
+    """``dq_debug_set_wait_limits`` (test hook); the defaults restore normal operation."""
+    lib().dq_debug_set_wait_limits(int(limit_ns), int(first_wait_limit_ns))
 
 
 def _check(rc: int, where: str) -> None:
