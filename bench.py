@@ -484,6 +484,7 @@ def run_cuda(args) -> dict:
         set_b(b)
         rec = {}
         rnd.norms_(grads)
+        sampler.start()
         for name, fn in (("quantize_pack", lambda i: rnd.quantize_(grads, SEED, i)),
                          ("norms_quantize_pack", lambda i: rnd.norms_quantize_(grads, SEED, i)),
                          ("unpack_dequant_average", lambda i: rnd.average_())):
@@ -495,6 +496,7 @@ def run_cuda(args) -> dict:
             r["gradient_gbs"] = round(4.0 * M * d / (t_train * 1e-3) / 1e9, 1)
             rec[name] = r
         step = timer.train(lambda i: rnd.step_fused(grads, rule_b(b, i + 1), SEED, i, overlap=not args.no_overlap), K)
+        rec["clocks"] = sampler.stop()
         rec["step_ms"] = round(step, 5)
         rec["step_gradient_gbs"] = round(4.0 * M * d / (step * 1e-3) / 1e9, 1)
         per_b[str(b)] = rec

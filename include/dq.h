@@ -47,8 +47,12 @@
  *    padding: ignored on input, the code of 0 in the packed stream, +0 in the
  *    output.
  *  - Codes: s = 2^(b-1) - 1 levels per sign (Sec. IV-A).  A b-bit code holds
- *    s + sgn * level, a number in 0 .. 2s: the paper's sign bit and b-1 bits of
- *    zeta folded into one field (0 has a single code, s).
+ *    s + sgn * level, a number in 0 .. 2s (excess-s; 0 has a single code, s).
+ *    THIS IS NOT THE WIRE FORMAT SEC. IV-A DESCRIBES, which spends one bit on the
+ *    sign and b-1 bits on the level zeta: the information and the b bits per
+ *    element of Eq. 7 are the same, the bit patterns are not, so a peer that
+ *    follows the paper's layout literally cannot read these words (and has a
+ *    second code, -0, that this format does not).
  *  - Packed stream of one worker: group q (padded elements 32q .. 32q+31) owns
  *    words b*q .. b*q+b-1; element e of the group owns bits [e*b, e*b+b) of
  *    that little-endian bit string.
@@ -339,17 +343,17 @@ const char* dq_status_string(int code);
 
 /* Test hook for the bounded waits (no counterpart in the paper).  Every wait of a
  * kernel for one of its own asynchronous copies is bounded by `limit_ns` of the GPU's
- * global timer (default 2e9; 0 restores the default).  `first_wait_limit_ns` bounds,
- * instead, the first such wait of every warp or CTA that consumes copies (UINT64_MAX:
- * the same as limit_ns).  Setting it to 0 declares those first waits lost at once
- * although their copies are valid and land a moment later, which exercises what a kernel
- * does after a time-out -- raise DQ_STAT_WAIT, stop producing output, wait (with
- * limit_ns) for every copy it has issued, return -- without anything being lost, faulting
- * or hanging.  Host state of the library, read when a call is made; not for production
- * use (outputs of a call made under it are incomplete). */
-void dq_debug_set_wait_limits(uint64_t limit_ns, uint64_t first_wait_limit_ns);
+ * global timer (default 2e9; 0 restores the default).  With `lose_first_wait` != 0 the
+ * first such wait of every warp or CTA that consumes copies is declared lost at once,
+ * although its copy is valid and lands a moment later: this exercises what a kernel does
+ * after a time-out -- raise DQ_STAT_WAIT, stop producing output, wait (with limit_ns)
+ * for every copy it has issued, return -- without anything being lost, faulting or
+ * hanging.  Host state of the library, read when a call is made; not for production use
+ * (the outputs of a call made under it are incomplete). */
+void dq_debug_set_wait_limits(uint64_t limit_ns, int32_t lose_first_wait);
 
 #ifdef __cplusplus
 }
 #endif
+
 #endif /* DQ_H */

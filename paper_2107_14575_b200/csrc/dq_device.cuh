@@ -207,6 +207,28 @@ __device__ __forceinline__ void push_code(uint32_t (&acc)[B], uint32_t& cur, con
     }
 }
 
+// The B words of a group whose 32 codes all equal s: what a zero scale gives (x = 0 and
+// floor(0 + v) = 0 for every draw v in (0, 1)), so such a group needs neither uniforms nor
+// arithmetic.  Everything here folds to constants.
+template <int B, int E>
+struct PushSame {
+    static __device__ __forceinline__ void run(uint32_t (&acc)[B], uint32_t& cur, const uint32_t code)
+    {
+        push_code<B, E>(acc, cur, code);
+        PushSame<B, E + 1>::run(acc, cur, code);
+    }
+};
+template <int B>
+struct PushSame<B, 32> {
+    static __device__ __forceinline__ void run(uint32_t (&)[B], uint32_t&, const uint32_t) {}
+};
+template <int B>
+__device__ __forceinline__ void zero_group_words(uint32_t (&acc)[B])
+{
+    uint32_t cur = 0;
+    PushSame<B, 0>::run(acc, cur, (1u << (B - 1)) - 1u);
+}
+
 // Stores the B words of one group into the warp's staging area (stride B words
 // between lanes; the widest access the alignment allows keeps bank conflicts low).
 template <int B>

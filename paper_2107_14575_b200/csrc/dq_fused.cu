@@ -107,6 +107,8 @@ __device__ __noinline__ float rescaled_team_norm(const uint32_t own, const int v
                                                  const float nrm)
 {
     const float mx = reduce_row_team(MaxMagnitude{}, own, valid, gpb);
+    // zero buckets (and those with an infinity or a NaN) are settled by the magnitude alone
+    if (!__any_sync(0xffffffffu, !l2_sum_in_range(sum) && magnitude_scalable(mx))) return l2_sum_in_range(sum) ? nrm : mx;
     const int e = scale_exponent(mx);
     const float scaled = reduce_row_team(ScaledSquares{e}, own, valid, gpb);
     return l2_sum_in_range(sum) ? nrm : rescaled_l2(mx, scaled, e);
@@ -203,6 +205,8 @@ __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* ba
         }
         if constexpr (B == 1) {
             acc[0] = 0u;
+        } else if (inv == 0.0f) {                // a zero bucket (sparse gradients are full of them): every code is s
+            zero_group_words<B>(acc);
         } else {
             uint32_t cur = 0;
             const uint32_t q0 = (uint32_t)(row0 + row) * 4u;
@@ -312,22 +316,24 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
     const uint32_t own_row0 = (uint32_t)(warp * kWStages * kWTileBytes + lane * 128 + ((lane & 7) << 4));
     int it = 0;
     bool timed_out = false, bad = false;
-    for (; it < n_tiles; ++it, advance(m, kt)) {
+    // (test hook: with lose_first the warp's first wait counts as lost: no tile is taken and the warp
+    // goes straight to what follows a time-out)
+    const int n_loop = a.wait.lose_first != 0u ? 0 : n_tiles;
+    for (; it < n_loop; ++it, advance(m, kt)) {
         const int st = it % kWStages;
         const int row0 = (int)(d_cur & 0x7fffffffu);
         const bool regular = (d_cur >> 31) != 0;
         unsigned char* base = wstage(warp, st);
         uint32_t* out_words = reinterpret_cast<uint32_t*>(base);
-        int span = 32;
+        int span = regular ? 32 : -1;            // groups whose words wait in the staging area; -1: the general route decides
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
         // warp-level synchronisations below are always reached by all lanes or by none
-        if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, st), (it / kWStages) & 1, it == 0 ? a.wait.first_ns : a.wait.ns))) {
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, st), (it / kWStages) & 1, a.wait))) {
             timed_out = true;
             break;
         }
 
-        bool done = false;
         if (regular) {
             // ---- norm of the bucket (same operations, same order as dq_bucket_norms)
             const uint32_t own = own_row0 + (uint32_t)(st * kWTileBytes);
@@ -344,10 +350,13 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 if (o < gpb) sum = join<P>(sum, other);
             }
             const float nrm = finish<P>(sum);
-            // a tile with an l2 sum out of range (see l2_sum_in_range) goes to the general route, which
-            // reduces such buckets a second time; the vote keeps the warp together
-            if (P == DQ_NORM_L2 && __any_sync(0xffffffffu, !l2_sum_in_range(sum))) goto general_route;
-            done = true;
+            // Rarely, for the l2 norm, a bucket's sum of squares is out of range (see l2_sum_in_range): all
+            // zeros, tiny entries, an overflowed square.  The general route takes such a tile: it reduces
+            // the bucket a second time where that is needed and skips the encoding of zero buckets.
+            if (P == DQ_NORM_L2 && __any_sync(0xffffffffu, !l2_sum_in_range(sum))) {
+                span = -1;
+                goto general_route;
+            }
             if (l == 0) {
                 a.norms[(int64_t)m * nb + (kt * R + r)] = nrm;
                 bad |= !isfinite(nrm);
@@ -401,7 +410,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
             }
         }
     general_route:
-        if (!done) {
+        if (span < 0) {
             const int res = irregular_tile<B, P>(a, base, row0, m, kt);
             span = res & 0xff;
             bad |= (res >> 8) != 0;
@@ -437,17 +446,20 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
         advance(pm, pkt);
     }
     if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
-    if (timed_out) {
+    if (timed_out || n_loop < n_tiles) {
         if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
         // every copy the warp has issued and not seen land, the one whose wait ran out included, gets the
         // full limit before the CTA's shared memory is released
         for (int j = it; j < it + kWStages; ++j)
-            if (j < n_tiles) (void)tma::mbar_wait(wbar(warp, j % kWStages), (j / kWStages) & 1, a.wait.ns);
+            if (j < n_tiles) (void)tma::mbar_wait(wbar(warp, j % kWStages), (j / kWStages) & 1, a.wait);
     }
 }
 
+// Five CTAs per SM (up to 102 registers per thread): at six (80 registers) the widest bit widths
+// spill in the tile loop, and the kernel, bound by instruction issue, loses nothing at 20 warps per SM.
+constexpr int kWarpKernelCtasPerSm = 5;
 template <int P>
-__global__ void __launch_bounds__(kThreads, 6)
+__global__ void __launch_bounds__(kThreads, kWarpKernelCtasPerSm)
 norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
     grid_dependency_wait();
@@ -589,7 +601,7 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
                 slot[2 * sub + 1] = part_b;
                 tma::mbar_arrive(pair_bar);
             }
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(pair_bar, exchanges & 1u, a.wait.ns))) return false;
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(pair_bar, exchanges & 1u, a.wait))) return false;
             ++exchanges;
             result = red.join(red.join(red.join(red.join(0.0f, slot[0]), slot[1]), slot[2]), slot[3]);
         }
@@ -608,6 +620,8 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
             }
             if constexpr (B == 1) {
                 acc[0] = 0u;
+            } else if (inv == 0.0f) {            // a zero bucket (the whole warp works on one bucket)
+                zero_group_words<B>(acc);
             } else {
                 uint32_t cur = 0;
                 const uint32_t q0 = (uint32_t)(row0 + lane) * 4u;
@@ -641,7 +655,9 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         __syncwarp();
     };
 
-    for (int it = 0; it < n_tiles; ++it) {
+    // test hook: the warp's first wait counts as lost, and the warp goes straight to what follows a time-out
+    timed_out = a.wait.lose_first != 0u;
+    for (int it = 0; it < n_tiles && !timed_out; ++it) {
         const int rows = (len + 31) >> 5;
         // the warp's next bucket (its halves are fetched as this one's halves leave)
         int nm = m, nk = k + 1, ng0 = 0, nlen = 0;
@@ -653,14 +669,14 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         }
 
         if (rows > 0) {
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u, it == 0 ? a.wait.first_ns : a.wait.ns))) {
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u, a.wait))) {
                 timed_out = true;
                 break;
             }
             pend_a = false; ++ph_a;
         }
         if (rows > 32) {
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait.ns))) { timed_out = true; break; }
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait))) { timed_out = true; break; }
             pend_b = false; ++ph_b;
         }
         int valid_a = len - lane * 32;
@@ -706,8 +722,8 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
         // every copy the warp has issued and not seen land, the one whose wait ran out included, gets the
         // full limit before the CTA's shared memory is released
-        if (pend_a) (void)tma::mbar_wait(wbar(warp, 0), ph_a & 1u, a.wait.ns);
-        if (pend_b) (void)tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait.ns);
+        if (pend_a) (void)tma::mbar_wait(wbar(warp, 0), ph_a & 1u, a.wait);
+        if (pend_b) (void)tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait);
     }
 }
 
@@ -819,7 +835,7 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
         }
         const int R = 32 >> a.gpb_shift;
         const int64_t warp_tiles = (int64_t)M * ((L->nb + R - 1) / R);
-        int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
+        int64_t blocks = (int64_t)dq_sm_count() * kWarpKernelCtasPerSm;
         if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
         dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
     } else {

@@ -386,7 +386,8 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
         // A thread whose wait runs out says so in shared memory and goes on (what it reads from the
         // stage is then arbitrary, and unused): every thread reaches the barriers below, after which all
         // of them see the flag and leave together.
-        const bool landed = tma::mbar_wait(full_bar(st), (it / kTmaStages) & 1, it == 0 ? a.wait.first_ns : a.wait.ns);
+        bool landed = tma::mbar_wait(full_bar(st), (it / kTmaStages) & 1, a.wait);
+        if (it == 0 && a.wait.lose_first != 0u) landed = false;      // test hook: the first wait counts as lost
         if (!landed) *abort_flag = 1;
 
         // One reduction of the tile: the gpb threads of a bucket combine inside a warp by shuffles and
@@ -460,7 +461,7 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
         // every copy already issued, the one whose wait ran out included, gets the full limit to land
         // before the CTA's shared memory is released
         for (int j = it; j < it + kTmaStages; ++j)
-            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kTmaStages), (j / kTmaStages) & 1, a.wait.ns);
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(j % kTmaStages), (j / kTmaStages) & 1, a.wait);
     }
 }
 

@@ -151,8 +151,9 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
     float next_norm = 0.0f;
     if (tile_begin < tile_end) prepare(m, rt, next_valid, next_norm);
     int it = 0;
-    bool timed_out = false;
-    for (int64_t tile = tile_begin; tile < tile_end; ++tile, ++it, advance(m, rt)) {
+    // test hook: the warp's first wait counts as lost, and the warp goes straight to what follows a time-out
+    bool timed_out = a.wait.lose_first != 0u && tile_begin < tile_end;
+    for (int64_t tile = tile_begin; tile < tile_end && !timed_out; ++tile, ++it, advance(m, rt)) {
         const int st = it % kStages;
         const uint32_t parity = (it / kStages) & 1;
         const int row0 = rt * 32;
@@ -168,7 +169,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
 
         // every lane polls the barrier itself; the verdict is made warp-uniform so that the
         // warp-level synchronisations below are always reached by all lanes or by none
-        if (!__all_sync(0xffffffffu, tma::mbar_wait(full_bar(warp, st), parity, it == 0 ? a.wait.first_ns : a.wait.ns))) {
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(full_bar(warp, st), parity, a.wait))) {
             timed_out = true;
             break;
         }
@@ -182,6 +183,8 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
         uint32_t acc[B];
         if constexpr (B == 1) {
             acc[0] = 0u;                        // s = 0: every code is 0
+        } else if (__all_sync(0xffffffffu, inv == 0.0f)) {
+            zero_group_words<B>(acc);           // a tile of zero buckets: every code is s, whatever the draw
         } else {
             uint32_t cur = 0;
             const uint32_t q0 = (uint32_t)g * 4u;
@@ -224,7 +227,7 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
         // full limit before the CTA's shared memory is released
         for (int k = 0; k < kStages; ++k) {
             const int j = it + k;
-            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(warp, j % kStages), (j / kStages) & 1, a.wait.ns);
+            if (tile_begin + j < tile_end) (void)tma::mbar_wait(full_bar(warp, j % kStages), (j / kStages) & 1, a.wait);
         }
     }
 }

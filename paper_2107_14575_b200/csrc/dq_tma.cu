@@ -45,8 +45,9 @@ bool dq_encode_tensor_map(CUtensorMap* map, CUtensorMapDataType type, uint32_t r
 
 // ---- wait limits (see WaitLimits) ----
 namespace {
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;
 std::mutex g_limits_mu;
-WaitLimits g_limits = {2000000000ull, 2000000000ull};
+WaitLimits g_limits = {kDefaultWaitNs, 0u, 0u};
 }  // namespace
 
 WaitLimits dq_wait_limits()
@@ -55,9 +56,9 @@ WaitLimits dq_wait_limits()
     return g_limits;
 }
 
-extern "C" void dq_debug_set_wait_limits(uint64_t limit_ns, uint64_t first_wait_limit_ns)
+extern "C" void dq_debug_set_wait_limits(uint64_t limit_ns, int32_t lose_first_wait)
 {
     std::lock_guard<std::mutex> lock(g_limits_mu);
-    g_limits.ns = limit_ns ? limit_ns : 2000000000ull;
-    g_limits.first_ns = first_wait_limit_ns == UINT64_MAX ? g_limits.ns : first_wait_limit_ns;
+    g_limits.ns = limit_ns ? limit_ns : kDefaultWaitNs;
+    g_limits.lose_first = lose_first_wait ? 1u : 0u;
 }

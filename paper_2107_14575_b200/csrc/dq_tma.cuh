@@ -15,16 +15,18 @@ bool dq_encode_tensor_map(CUtensorMap* map, CUtensorMapDataType type, uint32_t r
                           const uint64_t* dims, const uint64_t* strides_bytes /*rank-1*/, const uint32_t* box,
                           CUtensorMapSwizzle swizzle);
 
-// Upper bounds on the waits for asynchronous copies, in nanoseconds of the global timer; every
-// kernel that waits receives them as an argument.  `ns` bounds every wait (2 s unless
-// dq_debug_set_wait_limits changed it).  `first_ns` bounds the FIRST wait of every consumer
-// (a warp or a CTA, as the kernel is organised) instead: it equals `ns` in normal use, and a test
-// sets it to 0 so that this wait is declared lost at once while its copy is valid and lands a
-// moment later -- the path taken after a time-out then runs with nothing actually lost.  A wait that
-// runs out raises DQ_STAT_WAIT, the CTA waits (with `ns`) for every copy it has issued, and leaves.
+// Limits of the waits for asynchronous copies; every kernel that waits receives them as part of
+// its (constant-bank) arguments.  `ns` bounds every wait, in nanoseconds of the global timer (2 s
+// unless dq_debug_set_wait_limits changed it).  `lose_first` is the test hook: when set, the FIRST
+// wait of every consumer (a warp or a CTA, as the kernel is organised) is declared lost without a
+// look at its barrier, while its copy is valid and lands a moment later -- the path taken after a
+// time-out then runs with nothing actually lost.  The kernels look at the hook outside their tile
+// loops (inside them it cost the quantizers 4 % of their time).  A wait that runs out raises DQ_STAT_WAIT, the
+// CTA waits (with `ns`) for every copy it has issued, and leaves.
 struct WaitLimits {
     unsigned long long ns;
-    unsigned long long first_ns;
+    uint32_t lose_first;
+    uint32_t reserved;
 };
 WaitLimits dq_wait_limits();     // host: the limits the next launches get
 
@@ -88,21 +90,19 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 
-// Waits for the phase with the given parity; false if `limit_ns` ran out.  A limit of 0 declares the
-// wait lost without a look at the barrier (the test hook's deterministic time-out).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const unsigned long long limit_ns)
+// Waits for the phase with the given parity; false if the limit ran out.  The limit is only read
+// on the slow path, so that a wait that succeeds at once costs one instruction and no registers.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const WaitLimits& lim)
 {
-    if (limit_ns == 0) return false;
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > limit_ns) return false;
+        if (global_timer_ns() - t0 > lim.ns) return false;
     }
 }
-
 // 3-D tiled tensor copy global -> shared, completion counted on `bar`.
 __device__ __forceinline__ void load_tile_3d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2)
 {

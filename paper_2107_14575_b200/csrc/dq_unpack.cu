@@ -74,7 +74,7 @@ __device__ __forceinline__ bool consumer_sync_or(const bool pred)
 }
 // Wait of the copy warp for a drained stage: as mbar_wait, but it also gives up when the
 // consumers have said that they are leaving.
-__device__ __forceinline__ bool wait_unless_aborted(uint64_t* bar, const uint32_t parity, const unsigned long long limit_ns)
+__device__ __forceinline__ bool wait_unless_aborted(uint64_t* bar, const uint32_t parity, const WaitLimits& lim)
 {
     if (tma::mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = tma::global_timer_ns();
@@ -82,7 +82,7 @@ __device__ __forceinline__ bool wait_unless_aborted(uint64_t* bar, const uint32_
 #pragma unroll 1
         for (int i = 0; i < 64; ++i)
             if (tma::mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag() != 0 || tma::global_timer_ns() - t0 > limit_ns) return false;
+        if (*abort_flag() != 0 || tma::global_timer_ns() - t0 > lim.ns) return false;
     }
 }
 __device__ __forceinline__ uint32_t* stage_words(int st) { return reinterpret_cast<uint32_t*>(smem + kStageOffset) + st * kStageWords; }
@@ -234,7 +234,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
             int issued = 0;
             for (int u = 0; u < my_units; ++u) {
                 const int st = u % kStages;
-                if (u >= kStages && !wait_unless_aborted(empty_bar(st), (uint32_t)(u / kStages - 1) & 1u, a.wait.ns)) {
+                if (u >= kStages && !wait_unless_aborted(empty_bar(st), (uint32_t)(u / kStages - 1) & 1u, a.wait)) {
                     if (*abort_flag() == 0) {            // nobody drained the stage in time
                         atomicOr(a.status, DQ_STAT_WAIT);
                         *abort_flag() = 1;
@@ -250,7 +250,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
             // consumers may not have waited for (when they left early), and the CTA's shared memory
             // must not be released under a copy in flight.
             for (int u = issued > kStages ? issued - kStages : 0; u < issued; ++u)
-                if (!tma::mbar_wait(full_bar(u % kStages), (uint32_t)(u / kStages) & 1u, a.wait.ns))
+                if (!tma::mbar_wait(full_bar(u % kStages), (uint32_t)(u / kStages) & 1u, a.wait))
                     atomicOr(a.status, DQ_STAT_WAIT);
         }
         return;
@@ -330,7 +330,9 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         // stages; it walks on to the barrier at the tile's end, where all consumers learn of it together
         // and leave.  (Warps that were still waiting for later stages run into their own limit first.)
         float acc[32];
-        bool timed_out = false, warp_out = false, x_pending = false;
+        // (test hook: every warp's first wait counts as lost, so the warps start out that way)
+        bool timed_out = false, warp_out = a.wait.lose_first != 0u, x_pending = false;
+        if (warp_out) *abort_flag() = 1;
         int u = 0;
         int tiles_done = 0;
         for (int tile = tile_begin; tile < tile_end; ++tile) {
@@ -373,7 +375,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                 }
                 const int st = u % kStages;
                 if (!warp_out &&
-                    !__all_sync(0xffffffffu, tma::mbar_wait(full_bar(st), (u / kStages) & 1, u == 0 ? a.wait.first_ns : a.wait.ns))) {
+                    !__all_sync(0xffffffffu, tma::mbar_wait(full_bar(st), (u / kStages) & 1, a.wait))) {
                     warp_out = true;
                     *abort_flag() = 1;
                 }
@@ -410,7 +412,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
             // own row of the swizzled output tile (conflict-free), then one bulk tensor store per tile
             bool x_landed = true;
             if constexpr (UPDATE) {
-                x_landed = tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u, a.wait.ns);
+                x_landed = tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u, a.wait);
                 if (x_landed) {
                     const float neg_lr = a.neg_lr;
 #pragma unroll
@@ -451,7 +453,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
             *abort_flag() = 1;
             if (tid == 0) atomicOr(a.status, DQ_STAT_WAIT);
             if constexpr (UPDATE) {
-                if (x_pending) (void)tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u, a.wait.ns);
+                if (x_pending) (void)tma::mbar_wait(x_bar(), (uint32_t)tiles_done & 1u, a.wait);
             }
         }
     }

@@ -123,7 +123,7 @@ def lib():
         L.dq_status_string.restype = C.c_char_p
         L.dq_status_string.argtypes = [C.c_int]
         L.dq_debug_set_wait_limits.restype = None
-        L.dq_debug_set_wait_limits.argtypes = [u64, u64]
+        L.dq_debug_set_wait_limits.argtypes = [u64, i32]
         _lib = L
     return _lib
 
@@ -132,9 +132,9 @@ def status_string(code: int) -> str:
     return lib().dq_status_string(int(code)).decode()
 
 
-def debug_set_wait_limits(limit_ns: int = 0, first_wait_limit_ns: int = 2 ** 64 - 1) -> None:
+def debug_set_wait_limits(limit_ns: int = 0, lose_first_wait: bool = False) -> None:
     """``dq_debug_set_wait_limits`` (test hook); the defaults restore normal operation."""
-    lib().dq_debug_set_wait_limits(int(limit_ns), int(first_wait_limit_ns))
+    lib().dq_debug_set_wait_limits(int(limit_ns), 1 if lose_first_wait else 0)
 
 
 def _check(rc: int, where: str) -> None:

@@ -74,6 +74,17 @@ def _full_round(w, b0, steps=2):
         want_out = oracle.unpack_dequant_average(ref, want_packed, norms, b)
         err = np.linalg.norm(out.astype(np.float64) - want_out) / max(np.linalg.norm(want_out), 1e-300)
         assert err <= AVG_RTOL, err
+        # and element by element (a single element off by a level would not move the L2 ratio at
+        # this size): within 1e-6 of the largest of its bucket's M norms -- the scale of the fp32 sums
+        # behind it -- plus the rounding of the result itself
+        scale = np.zeros(ref.D32)
+        top = norms.max(axis=0).astype(np.float64)
+        for k in range(ref.nb):
+            s0, n = int(ref.bucket_start[k]), int(ref.bucket_len[k])
+            scale[s0: s0 + n] = top[k]
+        bound = 1e-6 * scale + 2.0 ** -23 * np.abs(want_out) + 1e-300
+        worst = np.abs(out.astype(np.float64) - want_out) - bound
+        assert np.all(worst <= 0), (int(np.argmax(worst)), float(worst.max()))
         # next b: the rule on the same norms
         b_next, s_next, _ = oracle.choose_bits(norms, w.T, t + 1, eps_hat, w.alpha)
         assert rnd.bits() == b_next

@@ -1,7 +1,7 @@
 """What the kernels do after a bounded wait ran out, exercised without losing anything.
 
-``dq_debug_set_wait_limits(limit, 0)`` makes the FIRST wait of every consumer (a warp or a CTA)
-give up after one look at its barrier, while the copy it waited for is valid and lands a moment
+``dq_debug_set_wait_limits(limit, 1)`` declares the FIRST wait of every consumer (a warp or a CTA)
+lost without a look at its barrier, while the copy it waited for is valid and lands a moment
 later.  The kernel must then raise DQ_STAT_WAIT, decide to leave in all threads that would
 otherwise meet at a barrier, wait (with the ordinary limit) for every copy it has issued, and
 return: the call completes, nothing outside the output buffers is touched, and the very next
@@ -31,7 +31,7 @@ def G(dqlib):
 
 @pytest.fixture()
 def short_first_wait(G):
-    G.dq.debug_set_wait_limits(LIMIT_NS, 0)
+    G.dq.debug_set_wait_limits(LIMIT_NS, True)
     yield
     G.dq.debug_set_wait_limits()          # back to the defaults, whatever the test did
 
@@ -89,7 +89,7 @@ def test_quantizers_after_a_lost_first_wait(G, short_first_wait, bucket):
         G, r, lambda: r.quantize(SEED, 1), lambda got: np.testing.assert_array_equal(got[:, :nw], want))
     assert st & G.dq.STAT_WAIT
     # fused norms + quantizer (per-warp tiles, whole-bucket warps, warp pairs)
-    G.dq.debug_set_wait_limits(LIMIT_NS, 0)
+    G.dq.debug_set_wait_limits(LIMIT_NS, True)
 
     def fused():
         got_norms, packed = r.norms_quantize(SEED, 1)
@@ -122,7 +122,7 @@ def test_average_and_update_after_a_lost_first_wait(G, short_first_wait, M, b):
         G, r, lambda: r.average(fill=0.0).copy(), lambda got: _assert_rel_l2(G, got, want))
     assert st & G.dq.STAT_WAIT
     # the update epilogue waits for the tile of x as well
-    G.dq.debug_set_wait_limits(LIMIT_NS, 0)
+    G.dq.debug_set_wait_limits(LIMIT_NS, True)
     x = np.linspace(-1.0, 1.0, ref.D32, dtype=np.float32)
     lr = 0.25
     want_x = oracle.unpack_average_update(ref, packed, norms, b, lr, x)

@@ -141,23 +141,20 @@ def test_exact_expectation_by_enumeration(b, d):
     # the drawn code is one of the two neighbours of x, chosen by floor(x + v)
     assert np.array_equal(codes - s, np.floor(x + u).astype(np.int64))
     assert np.all(np.isin(codes - s - sgn * low, (0, 1, -1)))
-    mean = np.zeros(d)
-    var = np.zeros(d)
-    total = 0.0
+    outcomes = []
     for ups in itertools.product((0, 1), repeat=d):
         ups = np.array(ups)
         p = np.prod(np.where(ups == 1, frac, 1.0 - frac))
         q = _values((s + sgn * (low + ups)).astype(np.uint32), norms[0, 0], b)
-        total += p
-        mean += p * q
-        var += p * q * q
-    var -= mean * mean
+        outcomes.append((p, q))
+    total = sum(p for p, _ in outcomes)
+    mean = sum(p * q for p, q in outcomes)
+    var = sum(p * (q - mean) ** 2 for p, q in outcomes)          # centred: no difference of large squares
     assert abs(total - 1.0) < 1e-12
     # E[Q(v)] = v up to the two fp32 roundings (each toward zero, < 1 ulp) in x = g * (s / norm)
     assert np.all(np.abs(mean - v[0, :d]) <= 2.0 ** -22 * np.abs(v[0, :d]) + 1e-30)
     # Var = (norm/s)^2 p_r (1 - p_r) per coordinate, trace <= d norm^2 / (4 s^2)
-    # (the variance comes from a difference of squares: allow for its cancellation)
-    assert np.allclose(var, (norm / s) ** 2 * frac * (1 - frac), rtol=1e-6, atol=1e-14 * (norm / s) ** 2)
+    assert np.allclose(var, (norm / s) ** 2 * frac * (1 - frac), rtol=1e-9, atol=1e-18 * (norm / s) ** 2)
     assert var.sum() <= d * norm ** 2 / (4 * s * s) * (1 + 1e-12)
 
 

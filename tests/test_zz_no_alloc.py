@@ -17,6 +17,8 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
+
 pytestmark = pytest.mark.gpu
 
 
@@ -50,6 +52,8 @@ def test_noalloc_bit_rule_matches_on_two_calls_in_a_row(dqlib):
     eps_hat = T * alpha ** (T - 1) * G2 / 36.0                    # b = 4 at t = 0
     ref1, new1 = _both(dq, lay, M, norms1, dq.Rule.dynamic(T, 0, eps_hat, alpha))
     assert ref1 == new1 and ref1[0] == 4 and ref1[1] == 7
+    # and both agree with the CPU checker's rule on the same norms
+    assert new1 == oracle.choose_bits(norms1, T, 0, eps_hat, alpha)[:2]
 
     # second call: much smaller norms, a later step, another layout size sharing the array
     M2, nb2 = 2, 9000
@@ -57,6 +61,7 @@ def test_noalloc_bit_rule_matches_on_two_calls_in_a_row(dqlib):
     norms2 = (np.abs(rng.standard_normal((M2, nb2))) * 1e-3).astype(np.float32)
     ref2, new2 = _both(dq, lay2, M2, norms2, dq.Rule.dynamic(T, 60, eps_hat * 1e-7, alpha))
     assert ref2 == new2 and ref2 != ref1
+    assert new2 == oracle.choose_bits(norms2, T, 60, eps_hat * 1e-7, alpha)[:2]
 
     # fixed b never touches the array; and the first problem again gives the first answer
     ref3, new3 = _both(dq, lay, M, norms1, dq.Rule.fixed(9))
