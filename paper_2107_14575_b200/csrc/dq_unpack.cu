@@ -162,18 +162,21 @@ struct AccumulateAll<B, 32> {
                                                const uint32_t) {}
 };
 
+// The upper halves of the words whose codes need them (see decode_code) come straight from shared
+// memory as 16-bit loads, two bytes into the word: the load pipe has room, the logic pipe, which a
+// shift would use, is the busiest one of this kernel.
 template <int B, int W>
 struct UpperHalves {
-    static __device__ __forceinline__ void run(const uint32_t (&wd)[B], uint32_t (&hi)[B])
+    static __device__ __forceinline__ void run(const uint32_t* __restrict__ src, uint32_t (&hi)[B])
     {
-        if constexpr (NeedsUpper<B, W>::value) hi[W] = wd[W] >> 16;
+        if constexpr (NeedsUpper<B, W>::value) hi[W] = reinterpret_cast<const uint16_t*>(src)[2 * W + 1];
         else hi[W] = 0u;
-        UpperHalves<B, W + 1>::run(wd, hi);
+        UpperHalves<B, W + 1>::run(src, hi);
     }
 };
 template <int B>
 struct UpperHalves<B, B> {
-    static __device__ __forceinline__ void run(const uint32_t (&)[B], uint32_t (&)[B]) {}
+    static __device__ __forceinline__ void run(const uint32_t* __restrict__, uint32_t (&)[B]) {}
 };
 
 // removes the power of two each element's decoded value carried
@@ -381,12 +384,22 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                 }
                 if (!warp_out) {
                     const uint32_t* base = stage_words(st) + tid * B;
-#pragma unroll 2
-                    for (int j = 0; j < mc; ++j) {
-                        uint32_t wd[B], hi[B];
-                        load_words<B>(base + j * (kThreads * B), wd);
-                        UpperHalves<B, 0>::run(wd, hi);
-                        AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
+                    if (mc == MC) {              // a full unit: no loop
+#pragma unroll
+                        for (int j = 0; j < MC; ++j) {
+                            uint32_t wd[B], hi[B];
+                            load_words<B>(base + j * (kThreads * B), wd);
+                            UpperHalves<B, 0>::run(base + j * (kThreads * B), hi);
+                            AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
+                        }
+                    } else {
+#pragma unroll 1
+                        for (int j = 0; j < mc; ++j) {
+                            uint32_t wd[B], hi[B];
+                            load_words<B>(base + j * (kThreads * B), wd);
+                            UpperHalves<B, 0>::run(base + j * (kThreads * B), hi);
+                            AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
+                        }
                     }
                 }
 #pragma unroll
