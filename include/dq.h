@@ -88,7 +88,7 @@ extern "C" {
 #define DQ_MAX_BUCKET   4096
 #define DQ_MAX_WORKERS  4096
 
-/* ---- members of the quantizer family of Eq. 5 ("||g||_p is the l_p norm") ---- */
+/* ---- members of the quantizer family of Eq. 5 (the norm that scales the entries) ---- */
 #define DQ_NORM_L2      2   /* p = 2, the default                                      */
 #define DQ_NORM_LINF    0   /* p = infinity: the largest magnitude of the bucket        */
 #define DQ_BUCKET_WHOLE_TENSOR 0  /* bucket argument: one norm per tensor, as Eq. 5 is written */
@@ -232,8 +232,12 @@ int dq_choose_bits(const dq_layout_t* layout, const float* dev_norms, int32_t M,
  *    norms).  Beyond it the call returns DQ_ERR_TOO_LARGE and launches nothing;
  *    use dq_choose_bits with caller scratch for larger problems.
  *  - The first call on each device looks up the array's device address (that
- *    device must be current, as for every call).  Make that first call before
- *    any stream capture begins.
+ *    device must be current, as for every call) and keeps it for the life of
+ *    the process.  Make that first call before any stream capture begins.  The
+ *    address belongs to the device's primary context: after a cudaDeviceReset
+ *    (or any other teardown of that context) the library must not be used
+ *    again in the same process.  Devices with ordinal 64 and above are not
+ *    served (DQ_ERR_CUDA).
  *  - All calls on a device share the one array, and it keeps what the last call
  *    wrote.  Nothing in it needs clearing between calls (each call overwrites
  *    every entry it later reads), but two calls whose kernels overlap on the
@@ -289,10 +293,9 @@ int dq_quantize_pack_worker(const dq_layout_t* layout, const float* dev_grads, i
  * dq_bucket_norms followed by dq_quantize_pack on the same gradients, with every
  * gradient byte read once: dev_norms receives exactly what dq_bucket_norms
  * writes and dev_packed exactly what dq_quantize_pack writes for those norms.
- * Algorithm 1 sets b_{t+1} from the gradients of iteration t ("Update the
- * quantization bits b_{t+1} according to Eq. 17" follows the averaging of step
- * t), so dev_b is known before this step's gradients are and the two steps
- * need not be separate passes.  A step is then
+ * Algorithm 1 sets b_{t+1} from the gradients of iteration t (its bit-update step
+ * comes after the averaging of step t), so dev_b is known before this step's
+ * gradients are and the two steps need not be separate passes.  A step is then
  *   dq_norms_quantize_pack (b_t) -> dq_unpack_dequant_average -> dq_choose_bits (b_{t+1}).
  * in : dev_grads, dev_b
  * out: dev_norms fp32 [M][nb], dev_packed (as for dq_quantize_pack)
@@ -323,9 +326,9 @@ int dq_unpack_dequant_average(const dq_layout_t* layout, const uint32_t* dev_pac
 
 /* ------------- Algorithm 1, server side: "Average" and the parameter update
  * x <- x - eta * g_hat, with g_hat the average dq_unpack_dequant_average computes
- * (the step "x_{t+1} = x_t - eta * g_hat_t" that follows the averaging in
- * Algorithm 1; the prose around Eq. 17 prints "+ eta", the listing and Eq. 2
- * "- eta": descent is meant).  The averaged gradient is formed in registers and
+ * (Eq. 2; the parameter-update step that follows the averaging in Algorithm 1.
+ * The prose around Eq. 17 prints the step with a plus sign, the listing and
+ * Eq. 2 with a minus sign: descent is meant).  The averaged gradient is formed in registers and
  * never written: per element M*b/8 + 4 bytes are read and 4 written.
  *   dev_params[j] <- fmaf(-lr, g_hat[j], dev_params[j])   (one fp32 rounding)
  * Padding elements of dev_params keep their value (their g_hat is 0), and so does

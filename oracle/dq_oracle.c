@@ -343,7 +343,7 @@ void oracle_unpack_dequant_average(const uint32_t* packed, int64_t packed_stride
     free_table(&tb);
 }
 
-/* Eq. 2 / Algorithm 1 "Update the global parameters": x <- x - eta * g_hat, with g_hat the
+/* Eq. 2 / the parameter-update step of Algorithm 1: x <- x - eta * g_hat, with g_hat the
  * average above, all in fp64 and rounded to fp32 once.  Padding elements keep their value. */
 void oracle_unpack_average_update(const uint32_t* packed, int64_t packed_stride,
                                   const float* norms, int32_t M, int32_t b,

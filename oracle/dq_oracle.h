@@ -21,7 +21,7 @@
  *   pack / unpack     b-bit codes concatenated LSB-first into 32-bit words
  *   unpack_dequant_average   Algorithm 1, server step "Average", with Eq. 5
  *   unpack_average_update    the same followed by the parameter update of Eq. 2
- *                     (Algorithm 1, "Update the global parameters")
+ *                     (the parameter-update step of Algorithm 1)
  *   philox4x32_10     Salmon, Moraes, Dror, Shaw, "Parallel random numbers:
  *                     as easy as 1, 2, 3" (SC'11), Philox-4x32 with 10 rounds
  *

@@ -107,16 +107,18 @@ extern "C" size_t dq_choose_bits_scratch_bytes(const dq_layout_t* L, int32_t M)
     return (size_t)((c * sizeof(double) + 255) / 256 * 256);
 }
 
-extern "C" int dq_choose_bits(const dq_layout_t* L, const float* dev_norms, int32_t M, const dq_rule_t* rule,
-                              int32_t* dev_b, void* dev_scratch, size_t scratch_bytes,
-                              int32_t* dev_status, void* stream)
+namespace {
+
+// Argument checks shared by the two entry points (everything but the scratch memory).
+int check_rule_args(const dq_layout_t* L, const float* dev_norms, int32_t M, const dq_rule_t* rule, const int32_t* dev_b,
+                    const int32_t* dev_status)
 {
     if (!L || !rule) return DQ_ERR_ARG;
     if (M < 1) return DQ_ERR_ARG;
     if (M > DQ_MAX_WORKERS) return DQ_ERR_RANGE;
-    if (!dev_norms || !dev_b || !dev_status || !dev_scratch) return DQ_ERR_ARG;
+    if (!dev_norms || !dev_b || !dev_status) return DQ_ERR_ARG;
     if ((reinterpret_cast<uintptr_t>(dev_norms) & 3u) || (reinterpret_cast<uintptr_t>(dev_b) & 3u) ||
-        (reinterpret_cast<uintptr_t>(dev_status) & 3u) || !aligned16(dev_scratch))
+        (reinterpret_cast<uintptr_t>(dev_status) & 3u))
         return DQ_ERR_ALIGN;
     if (rule->fixed_b < 0 || rule->fixed_b > DQ_MAX_BITS) return DQ_ERR_RANGE;
     if (rule->b_min < 1 || rule->b_max > DQ_MAX_BITS || rule->b_min > rule->b_max) return DQ_ERR_RANGE;
@@ -124,25 +126,42 @@ extern "C" int dq_choose_bits(const dq_layout_t* L, const float* dev_norms, int3
         (rule->T < 1 || rule->t < 0 || rule->t >= rule->T || !(rule->eps_hat > 0.0) || !(rule->alpha > 0.0) ||
          !std::isfinite(rule->eps_hat) || !std::isfinite(rule->alpha)))
         return DQ_ERR_RANGE;
-    if (scratch_bytes < dq_choose_bits_scratch_bytes(L, M)) return DQ_ERR_RANGE;
+    return DQ_OK;
+}
 
+// The two kernels of the rule, with the chunk sums in `partial` (at least num_chunks(M * nb) doubles).
+int launch_rule(const dq_layout_t* L, const float* dev_norms, int32_t M, const dq_rule_t* rule, int32_t* dev_b,
+                double* partial, int32_t* dev_status, void* stream)
+{
     const int64_t n = (int64_t)M * L->nb;
     const int64_t chunks = num_chunks(n);
     double coef = 0.0;
     if (rule->fixed_b == 0)
         coef = std::sqrt((double)rule->T / rule->eps_hat) *
                std::pow(rule->alpha, (double)(rule->T - 1 - rule->t) / 2.0);
-
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    double* partial = static_cast<double*>(dev_scratch);
     if (rule->fixed_b == 0) {
         dq_launch(norm_square_partials, dim3((unsigned)chunks), dim3(kSumThreads), 0, st, dev_norms, n, partial);
         if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     }
     dq_launch(apply_rule, dim3(1), dim3(kThreads), 0, st, partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
-                                      rule->b_min, rule->b_max, rule->fixed_b, dev_b, dev_status);
+              rule->b_min, rule->b_max, rule->fixed_b, dev_b, dev_status);
     if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
     return DQ_OK;
+}
+
+}  // namespace
+
+extern "C" int dq_choose_bits(const dq_layout_t* L, const float* dev_norms, int32_t M, const dq_rule_t* rule,
+                              int32_t* dev_b, void* dev_scratch, size_t scratch_bytes,
+                              int32_t* dev_status, void* stream)
+{
+    const int rc = check_rule_args(L, dev_norms, M, rule, dev_b, dev_status);
+    if (rc != DQ_OK) return rc;
+    if (!dev_scratch) return DQ_ERR_ARG;
+    if (!aligned16(dev_scratch)) return DQ_ERR_ALIGN;
+    if (scratch_bytes < dq_choose_bits_scratch_bytes(L, M)) return DQ_ERR_RANGE;
+    return launch_rule(L, dev_norms, M, rule, dev_b, static_cast<double*>(dev_scratch), dev_status, stream);
 }
 
 // ---------------------------------------------------------------------------
@@ -191,40 +210,14 @@ extern "C" int64_t dq_choose_bits_noalloc_max_norms(void) { return (int64_t)kNoA
 extern "C" int dq_choose_bits_noalloc(const dq_layout_t* L, const float* dev_norms, int32_t M, const dq_rule_t* rule,
                                       int32_t* dev_b, int32_t* dev_status, void* stream)
 {
-    if (!L || !rule) return DQ_ERR_ARG;
-    if (M < 1) return DQ_ERR_ARG;
-    if (M > DQ_MAX_WORKERS) return DQ_ERR_RANGE;
-    if (!dev_norms || !dev_b || !dev_status) return DQ_ERR_ARG;
-    if ((reinterpret_cast<uintptr_t>(dev_norms) & 3u) || (reinterpret_cast<uintptr_t>(dev_b) & 3u) ||
-        (reinterpret_cast<uintptr_t>(dev_status) & 3u))
-        return DQ_ERR_ALIGN;
-    if (rule->fixed_b < 0 || rule->fixed_b > DQ_MAX_BITS) return DQ_ERR_RANGE;
-    if (rule->b_min < 1 || rule->b_max > DQ_MAX_BITS || rule->b_min > rule->b_max) return DQ_ERR_RANGE;
-    if (rule->fixed_b == 0 &&
-        (rule->T < 1 || rule->t < 0 || rule->t >= rule->T || !(rule->eps_hat > 0.0) || !(rule->alpha > 0.0) ||
-         !std::isfinite(rule->eps_hat) || !std::isfinite(rule->alpha)))
-        return DQ_ERR_RANGE;
-    const int64_t n = (int64_t)M * L->nb;
-    const int64_t chunks = num_chunks(n);
-    if (chunks > kNoAllocMaxChunks) return DQ_ERR_TOO_LARGE;     // more norms than the built-in array covers
+    const int rc0 = check_rule_args(L, dev_norms, M, rule, dev_b, dev_status);
+    if (rc0 != DQ_OK) return rc0;
+    if (num_chunks((int64_t)M * L->nb) > kNoAllocMaxChunks) return DQ_ERR_TOO_LARGE;     // more norms than the built-in array covers
 
     double* partial = nullptr;
     const int rc = noalloc_scratch(&partial);
     if (rc != DQ_OK) return rc;
-
-    double coef = 0.0;
-    if (rule->fixed_b == 0)
-        coef = std::sqrt((double)rule->T / rule->eps_hat) *
-               std::pow(rule->alpha, (double)(rule->T - 1 - rule->t) / 2.0);
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Nothing in the array has to start at zero: the first kernel writes every entry the
     // second one reads, so whatever an earlier call left behind is overwritten, never used.
-    if (rule->fixed_b == 0) {
-        dq_launch(norm_square_partials, dim3((unsigned)chunks), dim3(kSumThreads), 0, st, dev_norms, n, partial);
-        if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
-    }
-    dq_launch(apply_rule, dim3(1), dim3(kThreads), 0, st, partial, rule->fixed_b == 0 ? (int)chunks : 0, M, coef,
-                                      rule->b_min, rule->b_max, rule->fixed_b, dev_b, dev_status);
-    if (cudaGetLastError() != cudaSuccess) return DQ_ERR_CUDA;
-    return DQ_OK;
+    return launch_rule(L, dev_norms, M, rule, dev_b, partial, dev_status, stream);
 }

@@ -66,6 +66,7 @@ class DistTransport:
         self.group = group
         self.world = dist.get_world_size(group)
         self.rank = dist.get_rank(group)
+        self._stage = None
 
     def gather_rows(self, row: torch.Tensor, all_rows: torch.Tensor) -> None:
         """all_rows[q] <- rank q's row (rows of equal length)."""
@@ -74,15 +75,26 @@ class DistTransport:
     def exchange(self, send: torch.Tensor, send_ranges: Sequence, recv: torch.Tensor, recv_len: int) -> None:
         """recv[q, :recv_len] <- elements send_ranges[self.rank] of rank q's ``send``; rank q gets
         send[send_ranges[q]] of this rank.  ``send_ranges`` = (start, length) per destination, contiguous
-        and ascending, so the send side needs no staging."""
+        and ascending, so the send side needs no staging.  The receive side lands straight in ``recv``
+        when its rows are exactly ``recv_len`` long; otherwise the rows of ``recv`` keep their aligned
+        stride and the data passes through a staging buffer that is allocated once and reused."""
         world = self.world
         lo = send_ranges[0][0]
         hi = send_ranges[-1][0] + send_ranges[-1][1]
         flat_in = send.view(-1)[lo:hi]
-        stage = torch.empty(world * recv_len, dtype=send.dtype, device=send.device)
-        self.dist.all_to_all_single(stage, flat_in, output_split_sizes=[recv_len] * world,
+        direct = recv.is_contiguous() and recv.shape[1] == recv_len
+        if direct:
+            flat_out = recv.view(-1)
+        else:
+            need = world * recv.shape[1]
+            if (self._stage is None or self._stage.numel() < need or self._stage.dtype != send.dtype
+                    or self._stage.device != send.device):
+                self._stage = torch.empty(need, dtype=send.dtype, device=send.device)
+            flat_out = self._stage[: world * recv_len]
+        self.dist.all_to_all_single(flat_out, flat_in, output_split_sizes=[recv_len] * world,
                                     input_split_sizes=[n for _, n in send_ranges], group=self.group)
-        recv[:, :recv_len].copy_(stage.view(world, recv_len))      # rows of recv keep their aligned stride
+        if not direct:
+            recv[:, :recv_len].copy_(flat_out.view(world, recv_len))
 
 
 class LoopbackTransport:
@@ -172,7 +184,9 @@ class ShardedRound:
                              if self.norm_scratch_bytes else None)
 
     def set_bits(self, b: int) -> None:
-        self.dev_b.copy_(torch.tensor([b, (1 << (b - 1)) - 1, 0, 0], dtype=torch.int32))
+        """Puts (b, s) into ``dev_b``: the library's bit rule with a fixed b writes both numbers."""
+        dq.choose_bits(self.layout, self.norms_all, self.world, dq.Rule.fixed(b), self.dev_b, self.scratch,
+                       self.scratch_bytes, self.status)
 
     def quantize_(self, grad: torch.Tensor, seed: int, step: int) -> None:
         if self.layout.whole_tensor:             # one norm per tensor: norms first, then the codes

@@ -177,3 +177,59 @@ def test_sharded_step_on_a_model_shape(G):
         assert r.read_status() == 0
         assert G.rel_l2(r.out.cpu().numpy(), want) <= 1e-6
         assert r.read_bits() == bo
+
+
+@pytest.mark.parametrize("b", [3, 8])
+def test_sharded_step_over_nccl_with_one_rank(G, b):
+    """The NCCL transport itself (not the loopback): a process group of one rank on this GPU drives
+    ``ShardedRound.step`` through ``DistTransport`` -- all-gather of the norms, all-to-all of the packed
+    range into this rank's own memory, average, all-gather of the result -- and must reproduce the
+    unsharded round bit for bit and, through it, the oracle."""
+    import os
+    import socket
+
+    import torch.distributed as dist
+    from paper_2107_14575_b200 import exchange
+    from paper_2107_14575_b200.pipeline import Round
+    dq = G.dq
+    if dist.is_initialized():
+        pytest.skip("a process group is already up in this process")
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    os.environ.setdefault("NCCL_NVLS_ENABLE", "0")
+    dist.init_process_group("nccl", init_method="tcp://127.0.0.1:%d" % port, rank=0, world_size=1,
+                            device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        segs, bucket = RAGGED + [3 * 4096 + 77], 512
+        ref = oracle.Layout(segs, bucket)
+        g = _grads(segs, 1, ref, 40 + b)
+        dev_g = torch.from_numpy(g).cuda()
+        one = Round(segs, bucket, 1)
+        one.bits_(dq.Rule.fixed(b))
+        one.norms_quantize_(dev_g, SEED, 2)
+        one.average_()
+        T, alpha = 50, 0.93
+        G2 = float((one.norms.double() ** 2).sum().item())
+        eps_hat = T * alpha ** (T - 1) * G2 / 30.0
+        rule = dq.Rule.dynamic(T, 20, eps_hat, alpha)
+
+        r = exchange.ShardedRound(segs, bucket, exchange.DistTransport(), 0, 1)
+        r.set_bits(b)
+        assert r.dev_b[:2].tolist() == [b, (1 << (b - 1)) - 1]         # (b, s) written by the library
+        out = r.step(dev_g[0], b, SEED, 2).clone()
+        out2 = r.step(dev_g[0], b, SEED, 2, next_rule=rule).clone()      # a second round reuses the staging buffer
+        torch.cuda.synchronize()
+        assert r.read_status() == 0
+        one.bits_(rule)
+        assert r.read_bits() == one.bits()                               # the next b, from the gathered norms
+        nw = ref.packed_words(b)
+        assert np.array_equal(r.packed_local.cpu().numpy().view(np.uint32)[:nw],
+                              one.packed.cpu().numpy().view(np.uint32)[0, :nw])
+        assert torch.equal(r.norms_all, one.norms)
+        assert torch.equal(out, one.out) and torch.equal(out2, one.out)
+        norms = one.norms.cpu().numpy()
+        want = oracle.unpack_dequant_average(ref, oracle.quantize_pack(ref, g, norms, b, SEED, 2), norms, b)
+        assert G.rel_l2(out.cpu().numpy(), want) <= 1e-6
+    finally:
+        dist.destroy_process_group()
