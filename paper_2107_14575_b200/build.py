@@ -1,8 +1,13 @@
 """Builds the CUDA library ``libdq.so`` in-tree with nvcc for sm_100a.
 
-Usage: ``python -m paper_2107_14575_b200.build [--force] [--verbose]``
+Usage: ``python -m paper_2107_14575_b200.build [--force] [--verbose] [--checked]``
 Objects go to ``paper_2107_14575_b200/_build``; the shared library sits next
 to the Python binding so that it travels with the source tree.
+
+``--checked`` builds ``libdq_checked.so`` instead (objects in ``_build_checked``): the same
+sources with ``-DDQ_CHECKED``, under which every store of a kernel to global memory checks that
+it lies inside the buffer it belongs to and raises ``DQ_STAT_INTERNAL`` instead of storing if it
+does not.  ``DQ_LIBRARY=<path>`` makes the Python binding load that library.
 """
 from __future__ import annotations
 
@@ -35,13 +40,18 @@ def _deps_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+LIB_CHECKED = os.path.join(PKG, "libdq_checked.so")
+
+
+def build(force: bool = False, verbose: bool = False, checked: bool = False) -> str:
+    LIB = LIB_CHECKED if checked else globals()["LIB"]
+    OBJ = globals()["OBJ"] + ("_checked" if checked else "")
     newest = _deps_mtime()
     if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest:
         return LIB
     os.makedirs(OBJ, exist_ok=True)
     nvcc = _nvcc()
-    extra = ["-Xptxas", "-v"] if verbose else []
+    extra = (["-Xptxas", "-v"] if verbose else []) + (["-DDQ_CHECKED"] if checked else [])
 
     def compile_one(src: str) -> str:
         obj = os.path.join(OBJ, src.replace(".cu", ".o"))
@@ -69,4 +79,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, checked="--checked" in sys.argv))

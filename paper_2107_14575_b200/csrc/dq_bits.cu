@@ -63,7 +63,7 @@ norm_square_partials(const float* __restrict__ norms, const int64_t n, double* _
         }
     }
     const double s = block_sum<kSumThreads>(a0 + a1, sh);
-    if (threadIdx.x == 0) partial[blockIdx.x] = s;
+    if (threadIdx.x == 0) partial[blockIdx.x] = s;       // one entry per CTA of the grid: in bounds by construction
 }
 
 __global__ void __launch_bounds__(kThreads)

@@ -107,6 +107,24 @@ inline void dq_launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sm
     (void)cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);   // the caller reads cudaGetLastError()
 }
 
+// Every store of a kernel to global memory goes through DQ_STORE(pointer, value, base, extent in
+// bytes, status word).  In the normal build that is the plain store and nothing else is evaluated.
+// Built with -DDQ_CHECKED (build.py --checked -> libdq_checked.so) every store first checks that it
+// lies inside [base, base + extent) and, if it does not, raises DQ_STAT_INTERNAL instead of storing:
+// the stand-in for a memory checker where none can be run.
+#ifdef DQ_CHECKED
+template <class T>
+__device__ __forceinline__ void dq_checked_store(T* p, const T& v, const void* base, const int64_t extent_bytes, int32_t* status)
+{
+    const int64_t off = reinterpret_cast<const char*>(p) - reinterpret_cast<const char*>(base);
+    if (off < 0 || off + (int64_t)sizeof(T) > extent_bytes) atomicOr(status, DQ_STAT_INTERNAL);
+    else *p = v;
+}
+#define DQ_STORE(p, v, base, extent_bytes, status) dq_checked_store((p), (v), (base), (int64_t)(extent_bytes), (status))
+#else
+#define DQ_STORE(p, v, base, extent_bytes, status) (*(p) = (v))
+#endif
+
 // Index of the last entry of starts[0..n] (n + 1 entries, non-decreasing) that is <= x.
 // Tensors of zero size repeat a start; the last repeat is the non-empty one.
 __device__ __forceinline__ int last_not_above(const int32_t* __restrict__ starts, int n, int x)

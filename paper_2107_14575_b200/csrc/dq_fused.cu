@@ -189,7 +189,7 @@ __device__ __noinline__ int irregular_tile(const FusedArgs& a, unsigned char* ba
     }
     int bad = 0;
     if (l == 0 && k < nb) {
-        a.norms[(int64_t)m * nb + k] = nrm;
+        DQ_STORE(a.norms + ((int64_t)m * nb + k), nrm, a.norms, (int64_t)a.M * a.v.nb * 4, a.status);
         bad = isfinite(nrm) ? 0 : 256;
     }
 
@@ -358,7 +358,7 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 goto general_route;
             }
             if (l == 0) {
-                a.norms[(int64_t)m * nb + (kt * R + r)] = nrm;
+                DQ_STORE(a.norms + ((int64_t)m * nb + (kt * R + r)), nrm, a.norms, (int64_t)a.M * a.v.nb * 4, a.status);
                 bad |= !isfinite(nrm);
             }
             // ---- codes of this lane's group against that norm
@@ -385,7 +385,8 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 __syncwarp();
                 uint4* dst = reinterpret_cast<uint4*>(a.packed + (int64_t)m * a.packed_stride + (int64_t)row0 * B);
 #pragma unroll
-                for (int i = 0; i < B / 4; ++i) dst[lane + 32 * i] = reinterpret_cast<const uint4*>(out_words)[lane + 32 * i];
+                for (int i = 0; i < B / 4; ++i)
+                    DQ_STORE(dst + (lane + 32 * i), reinterpret_cast<const uint4*>(out_words)[lane + 32 * i], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
                 span = 0;                        // nothing left for the general copy below
             } else {
                 // 32 * B words from word `off` of a 16-byte unit: quads 0 (or 1) .. 8B - 1 in full, the
@@ -400,11 +401,11 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
                 for (int i = 0; i < (8 * B + 31) / 32; ++i) {
                     const int q = lane + 32 * i;
                     if (q < 8 * B && (q > 0 || off == 0))
-                        reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
+                        DQ_STORE(reinterpret_cast<uint4*>(aligned_dst) + q, reinterpret_cast<const uint4*>(out_words)[q], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
                 }
                 if (off != 0 && lane < 4) {
                     const int idx = lane >= off ? lane : 32 * B + lane;
-                    aligned_dst[idx] = out_words[idx];
+                    DQ_STORE(aligned_dst + idx, out_words[idx], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
                 }
                 span = 0;
             }
@@ -427,11 +428,11 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
             uint32_t* aligned_dst = a.packed + (int64_t)m * a.packed_stride + ((int64_t)row0 * B - off);
             const int q0 = off ? 1 : 0, q1 = jend >> 2;          // full quads [q0, q1)
             for (int q = q0 + lane; q < q1; q += 32)
-                reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
-            if (off && lane >= off && lane < 4 && lane < jend) aligned_dst[lane] = out_words[lane];   // head
+                DQ_STORE(reinterpret_cast<uint4*>(aligned_dst) + q, reinterpret_cast<const uint4*>(out_words)[q], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
+            if (off && lane >= off && lane < 4 && lane < jend) DQ_STORE(aligned_dst + lane, out_words[lane], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);   // head
             int ts = q1 * 4;                                                                          // tail
             if (off && ts < 4) ts = 4;
-            if (lane < jend - ts) aligned_dst[ts + lane] = out_words[ts + lane];
+            if (lane < jend - ts) DQ_STORE(aligned_dst + (ts + lane), out_words[ts + lane], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
         }
         __syncwarp();
 
@@ -647,11 +648,11 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         uint32_t* aligned_dst = a.packed + (int64_t)mm * a.packed_stride + ((int64_t)row0 * B - off);
         const int q0 = off ? 1 : 0, q1 = jend >> 2;          // full quads [q0, q1)
         for (int q = q0 + lane; q < q1; q += 32)
-            reinterpret_cast<uint4*>(aligned_dst)[q] = reinterpret_cast<const uint4*>(out_words)[q];
-        if (off && lane >= off && lane < 4 && lane < jend) aligned_dst[lane] = out_words[lane];   // head
+            DQ_STORE(reinterpret_cast<uint4*>(aligned_dst) + q, reinterpret_cast<const uint4*>(out_words)[q], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
+        if (off && lane >= off && lane < 4 && lane < jend) DQ_STORE(aligned_dst + lane, out_words[lane], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);   // head
         int ts = q1 * 4;                                                                          // tail
         if (off && ts < 4) ts = 4;
-        if (lane < jend - ts) aligned_dst[ts + lane] = out_words[ts + lane];
+        if (lane < jend - ts) DQ_STORE(aligned_dst + (ts + lane), out_words[ts + lane], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
         __syncwarp();
     };
 
@@ -698,7 +699,7 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
             }
         }
         if (lane == 0 && sub == 0) {
-            a.norms[(int64_t)m * nb + k] = nrm;
+            DQ_STORE(a.norms + ((int64_t)m * nb + k), nrm, a.norms, (int64_t)a.M * a.v.nb * 4, a.status);
             bad |= !isfinite(nrm);
         }
         const float inv = inv_scale(sf, nrm);

@@ -116,7 +116,7 @@ bucket_norms_kernel(const LayoutView v, const float* __restrict__ grads, const i
                 }
             }
             if (lane == 0 && active) {
-                nw[k] = nrm;
+                DQ_STORE(nw + k, nrm, norms, (int64_t)gridDim.y * v.nb * 4, status);
                 bad |= !isfinite(nrm);
             }
         }
@@ -248,7 +248,7 @@ bucket_norms_warp_kernel(const LayoutView v, const float* __restrict__ grads, co
             }
         }
         if (lane < kRun && k0 + lane < v.nb) {
-            nw[k0 + lane] = nrm;
+            DQ_STORE(nw + (k0 + lane), nrm, norms, (int64_t)gridDim.y * v.nb * 4, status);
             bad |= !isfinite(nrm);
         }
     }
@@ -448,7 +448,7 @@ bucket_norms_tma_kernel(const __grid_constant__ NormsArgs a, const __grid_consta
             }
         }
         if (writes) {
-            a.norms[(int64_t)m * nb + k] = nrm;
+            DQ_STORE(a.norms + ((int64_t)m * nb + k), nrm, a.norms, (int64_t)a.M * a.v.nb * 4, a.status);
             bad |= !isfinite(nrm);
         }
         if (ptile < tile_end && tid == 0) issue(st);
@@ -519,7 +519,7 @@ tensor_norms_join_kernel(const int32_t n_seg, const int32_t* __restrict__ piece0
         for (int w = 0; w < kJoinThreads / 32; ++w) total = max_nan(total, part_f[w]);
         nrm = total;
     }
-    norms[(int64_t)m * nb + k] = nrm;
+    DQ_STORE(norms + ((int64_t)m * nb + k), nrm, norms, (int64_t)gridDim.y * nb * 4, status);
     if (!isfinite(nrm)) atomicOr(status, DQ_STAT_NONFINITE);
 }
 

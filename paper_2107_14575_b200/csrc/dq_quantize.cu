@@ -211,8 +211,8 @@ __device__ __forceinline__ void quantize_tiles(const QuantizeArgs& a, const CUte
         uint32_t* dst = a.packed + (int64_t)m * a.packed_stride + (int64_t)row0 * B;
         const int n4 = nwords >> 2;
         for (int i = lane; i < n4; i += 32)
-            reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(out_words)[i];
-        if (lane < (nwords & 3)) dst[n4 * 4 + lane] = out_words[n4 * 4 + lane];
+            DQ_STORE(reinterpret_cast<uint4*>(dst) + i, reinterpret_cast<const uint4*>(out_words)[i], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
+        if (lane < (nwords & 3)) DQ_STORE(dst + (n4 * 4 + lane), out_words[n4 * 4 + lane], a.packed, (int64_t)a.M * a.packed_stride * 4, a.status);
         __syncwarp();
 
         // refill the stage

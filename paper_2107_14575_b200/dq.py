@@ -12,7 +12,8 @@ import os
 from typing import Optional, Sequence
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libdq.so")
+# DQ_LIBRARY selects another build of the same library (the bounds-checked one, libdq_checked.so)
+LIB_PATH = os.environ.get("DQ_LIBRARY") or os.path.join(_PKG, "libdq.so")
 
 OK, ERR_ARG, ERR_ALIGN, ERR_RANGE, ERR_CUDA, ERR_STATE, ERR_TOO_LARGE = 0, -1, -2, -3, -4, -5, -6
 STAT_NONFINITE, STAT_BAD_BITS, STAT_CAPACITY, STAT_WAIT, STAT_INTERNAL = 1, 2, 4, 8, 16
