@@ -282,9 +282,7 @@ def _bound(kernel_key, b, alg_bytes, units, ms, peak_gbs, sm_count, sm_mhz):
         t_hbm_ms = alg_bytes / (peak_gbs * 1e9) * 1e3
         rec["issue"] = {"warp_instructions_per_group": round(ipu, 1), "warp_instructions": inst,
                         "roof_ms": round(t_issue_ms, 5), "hbm_roof_ms": round(t_hbm_ms, 5),
-                        "frac_of_issue_roof": round(t_issue_ms / ms, 4),
-                        "lane_instructions_per_element": round(ipu, 1),     # 32 lanes x instructions / 32 elements
-                        "sm_mhz": sm_mhz}
+                        "frac_of_issue_roof": round(t_issue_ms / ms, 4), "sm_mhz": sm_mhz}
         if t_issue_ms > t_hbm_ms:
             rec["bound"] = "alu"
     return rec
@@ -480,7 +478,7 @@ def run_cuda(args) -> dict:
     per_b = {}
     n_single = min(K, 8)
     norms_ms = timer.train(lambda i: rnd.norms_(grads), K)
-    for b in PER_B:
+    for b in (() if args.no_per_b else PER_B):
         set_b(b)
         rec = {}
         rnd.norms_(grads)
@@ -595,6 +593,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     ap.add_argument("--no-models", action="store_true", help="skip the secondary timing of the model-shaped workloads")
+    ap.add_argument("--no-per-b", action="store_true", help="skip the per-b table (profiling runs)")
     ap.add_argument("--no-overlap", action="store_true",
                     help="run the bit rule after the average on the same stream instead of beside it")
     ap.add_argument("--source-digests", action="store_true",

@@ -12,6 +12,9 @@ counters kept under ``profiles/``.
     # the per-b table of a bench line as markdown
     python -m paper_2107_14575_b200.profiling table bench_line.json > profiles/bench_per_b.md
 
+    # per kernel launches / time / share from an `ncu --metrics gpu__time_duration.sum --csv --log-file` run
+    python -m paper_2107_14575_b200.profiling launches launches.csv --command "<the ncu command>" > profiles/bench_launch_list.md
+
 ``run`` needs a GPU; the other two run anywhere.  Nothing here is on the product path.
 """
 from __future__ import annotations
@@ -184,9 +187,10 @@ def cmd_summarize(a) -> None:
     if a.note:
         out += ["", a.note]
     name = a.out or os.path.join(ROOT, "profiles", "%s_flat_d%d_m%d_b%d.md" % (pattern.rstrip("_"), a.log2d, a.M, a.b))
-    with open(name, "w") as fh:
-        fh.write("\n".join(out) + "\n")
-    print("wrote", name)
+    if not a.counters_only:
+        with open(name, "w") as fh:
+            fh.write("\n".join(out) + "\n")
+        print("wrote", name)
     if a.update_counters:
         path = os.path.join(ROOT, "profiles", "counters.json")
         rec = {}
@@ -202,8 +206,9 @@ def cmd_summarize(a) -> None:
             cur["warp_instructions_per_group"][str(a.b)] = round(inst / n_groups, 2)
         if traffic is not None:
             cur["dram_bytes_per_group"][str(a.b)] = round(traffic / n_groups, 2)
-        cur["cases"][str(a.b)] = {"log2d": a.log2d, "M": a.M, "bucket": a.bucket,
-                                  "summary": os.path.relpath(name, ROOT)}
+        cur["cases"][str(a.b)] = {"log2d": a.log2d, "M": a.M, "bucket": a.bucket, "command": a.command}
+        if not a.counters_only:
+            cur["cases"][str(a.b)]["summary"] = os.path.relpath(name, ROOT)
         rec[a.kernel] = cur
         with open(path, "w") as fh:
             json.dump(rec, fh, indent=1, sort_keys=True)
@@ -252,6 +257,40 @@ def cmd_table(a) -> None:
                 w["unpack_dequant_average"]["ms"], w["unpack_dequant_average"]["frac_of_measured"]))
 
 
+def cmd_launches(a) -> None:
+    """Per kernel: launches, total time and share, from the CSV log of an
+    ``ncu --metrics gpu__time_duration.sum --csv --log-file`` run (one row per launch)."""
+    with open(a.csv, newline="") as fh:
+        rows = [r for r in csv.reader(l for l in fh if not l.startswith("==")) if r]
+    hdr, body = rows[0], rows[1:]
+    ki, vi, ui = hdr.index("Kernel Name"), hdr.index("Metric Value"), hdr.index("Metric Unit")
+    per = {}
+    for r in body:
+        full = r[ki].replace("(anonymous namespace)::", "").replace("<unnamed>::", "")
+        name = full.split("(")[0].split("<")[0].replace("void ", "").strip().split("::")[-1]
+        t = float(r[vi].replace(",", "")) * {"ns": 1e-3, "us": 1.0, "ms": 1e3}[r[ui]]
+        n, tot = per.get(name, (0, 0.0))
+        per[name] = (n + 1, tot + t)
+    library = ("norms_quantize_pack", "quantize_pack_kernel", "bucket_norms", "unpack_average_kernel", "tensor_norms_join",
+               "norm_square_partials", "apply_rule")
+    ours = {k: v for k, v in per.items() if any(k.startswith(p) for p in library)}
+    total_ours = sum(t for _, t in ours.values())
+    total_all = sum(t for _, t in per.values())
+    print("# Launch list of the bench command\n")
+    print("Command (one B200; the same command line had exited 0 without ncu directly before):\n\n```\n%s\n```\n" % a.command)
+    print("Every launch of the process with its device time (ncu serialises the launches and flushes the caches, so the "
+          "absolute times are cold-cache figures: the SHARES are what the bench line's must agree with).  %d launches, "
+          "%.1f us in the library's kernels, %.1f us in all kernels (the rest is torch: the generator, fills, copies).\n"
+          % (len(body), total_ours, total_all))
+    print("| kernel | launches | total us | mean us | share of the library's kernels |")
+    print("|---|---|---|---|---|")
+    for k, (n, t) in sorted(per.items(), key=lambda kv: -kv[1][1]):
+        share = "%.3f" % (t / total_ours) if k in ours else "(torch)"
+        print("| %s | %d | %.1f | %.1f | %s |" % (k, n, t, t / n, share))
+    if a.note:
+        print("\n" + a.note)
+
+
 def main(argv=None) -> None:
     ap = argparse.ArgumentParser(prog="python -m paper_2107_14575_b200.profiling")
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -273,10 +312,15 @@ def main(argv=None) -> None:
     s.add_argument("--note", default="")
     s.add_argument("--out", default=None)
     s.add_argument("--update-counters", action="store_true")
+    s.add_argument("--counters-only", action="store_true", help="no summary file, only profiles/counters.json")
     t = sub.add_parser("table")
     t.add_argument("json")
+    l = sub.add_parser("launches")
+    l.add_argument("csv")
+    l.add_argument("--command", required=True)
+    l.add_argument("--note", default="")
     a = ap.parse_args(argv)
-    {"run": cmd_run, "summarize": cmd_summarize, "table": cmd_table}[a.cmd](a)
+    {"run": cmd_run, "summarize": cmd_summarize, "table": cmd_table, "launches": cmd_launches}[a.cmd](a)
 
 
 if __name__ == "__main__":
