@@ -482,19 +482,23 @@ def run_cuda(args) -> dict:
         set_b(b)
         rec = {}
         rnd.norms_(grads)
-        sampler.start()
         for name, fn in (("quantize_pack", lambda i: rnd.quantize_(grads, SEED, i)),
                          ("norms_quantize_pack", lambda i: rnd.norms_quantize_(grads, SEED, i)),
                          ("unpack_dequant_average", lambda i: rnd.average_())):
+            # a train of launches runs long enough for the power cap to pull the SM clock down: the clock
+            # is sampled per train and the instruction roof of the point uses that sample
+            sampler.start()
             t_train = timer.train(fn, K)
+            clk = sampler.stop()
             t_single = timer.single(fn, n_single)
-            r = _bound(name, b, alg_bytes[name](b), units[name], t_train, peak, sm_count, sm_mhz)
+            r = _bound(name, b, alg_bytes[name](b), units[name], t_train, peak, sm_count, clk.get("sm_mhz") or sm_mhz)
+            r["sm_mhz"] = clk.get("sm_mhz")
+            r["clock_reasons"] = clk.get("reasons")
             r["single_launch_ms"] = round(t_single, 5)
             r["single_launch_frac_of_measured"] = round(alg_bytes[name](b) / (t_single * 1e-3) / 1e9 / peak, 4)
             r["gradient_gbs"] = round(4.0 * M * d / (t_train * 1e-3) / 1e9, 1)
             rec[name] = r
         step = timer.train(lambda i: rnd.step_fused(grads, rule_b(b, i + 1), SEED, i, overlap=not args.no_overlap), K)
-        rec["clocks"] = sampler.stop()
         rec["step_ms"] = round(step, 5)
         rec["step_gradient_gbs"] = round(4.0 * M * d / (step * 1e-3) / 1e9, 1)
         per_b[str(b)] = rec

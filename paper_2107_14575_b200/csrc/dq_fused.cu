@@ -114,6 +114,32 @@ __device__ __noinline__ float rescaled_team_norm(const uint32_t own, const int v
     return l2_sum_in_range(sum) ? nrm : rescaled_l2(mx, scaled, e);
 }
 
+// Called by the whole warp for a regular tile in which some bucket's l2 sum is out of range.  If
+// every entry of the tile is +0 or -0, stages the tile's words -- the same B words for every group:
+// all codes equal s -- in the stream's 16-byte phase, where the general copy expects them, and
+// returns true (in all lanes); otherwise touches nothing and returns false.  Out of line: the common
+// case does not pay for its registers.
+template <int B>
+__device__ __noinline__ bool stage_zero_tile(const uint32_t own, uint32_t* out_words, const int row0)
+{
+    uint32_t bits = 0u;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint4 x = *reinterpret_cast<const uint4*>(smem + (own ^ (uint32_t)(c << 4)));
+        bits |= x.x | x.y | x.z | x.w;
+    }
+    if (!__all_sync(0xffffffffu, (bits << 1) == 0u)) return false;
+    // (the vote is behind every lane's reads of its row: the rows may be overwritten now)
+    uint32_t z[B];
+    if constexpr (B == 1) z[0] = 0u;
+    else zero_group_words<B>(z);
+    const int lane = threadIdx.x & 31;
+    const int off = (int)(((int64_t)row0 * B) & 3);
+#pragma unroll
+    for (int i = 0; i < B; ++i) out_words[off + lane * B + i] = z[i];
+    return true;
+}
+
 // ---- buckets that fit one warp: a tile that touches the end of a tensor ---------------
 // General route of the per-warp pipelines, kept out of line so that the common case does
 // not pay for its registers: buckets may be short, rows of the tile may belong to nobody,
@@ -354,7 +380,14 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
             // zeros, tiny entries, an overflowed square.  The general route takes such a tile: it reduces
             // the bucket a second time where that is needed and skips the encoding of zero buckets.
             if (P == DQ_NORM_L2 && __any_sync(0xffffffffu, !l2_sum_in_range(sum))) {
-                span = -1;
+                // a tile of nothing but zeros (sparse gradients are full of them) needs no arithmetic at all:
+                // its norms are 0 and every code is s; the words are staged for the general copy below
+                if (stage_zero_tile<B>(own, out_words, row0)) {
+                    if (l == 0)
+                        DQ_STORE(a.norms + ((int64_t)m * nb + (kt * R + r)), 0.0f, a.norms, (int64_t)a.M * a.v.nb * 4, a.status);
+                } else {
+                    span = -1;
+                }
                 goto general_route;
             }
             if (l == 0) {

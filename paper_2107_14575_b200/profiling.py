@@ -230,11 +230,13 @@ def cmd_table(a) -> None:
     print("# Per-b figures of the bench workload\n")
     print(line["config"]["workload"] + ".  From one `python bench.py --steps %d --warmup %d` line; `train` = launches "
           "back to back between two CUDA events, `single` = one launch between its own events; fractions are of the "
-          "copy bandwidth %.0f GB/s (%s).\n" % (line["steps"], line["warmup"], line["roofline"]["hbm"]["achieved_gbs"] /
+          "copy bandwidth %.0f GB/s (%s).  `SM MHz` is the median NVML sample during the train: these trains run into "
+          "the 1000 W power cap (`sw_power_cap`), which pulls the clock below its 1965 MHz maximum, and the "
+          "instruction-bound kernels slow down with it.\n" % (line["steps"], line["warmup"], line["roofline"]["hbm"]["achieved_gbs"] /
                                               max(line["roofline"]["hbm"]["frac_of_measured"], 1e-9),
                                               line["roofline"].get("peak_source", "")))
     names = ("quantize_pack", "norms_quantize_pack", "unpack_dequant_average")
-    print("| b | " + " | ".join("%s train ms / GB/s / frac / bound | single ms / frac" % n for n in names) +
+    print("| b | " + " | ".join("%s train ms / GB/s / frac / bound / SM MHz | single ms / frac" % n for n in names) +
           " | step ms | step GB/s of gradient |")
     print("|---|" + "---|---|" * len(names) + "---|---|")
     for b in sorted(per_b, key=int):
@@ -242,9 +244,10 @@ def cmd_table(a) -> None:
         cells = []
         for n in names:
             k = r[n]
-            cells.append("%.3f / %.0f / %.3f / %s | %.3f / %.3f" % (k["ms"], k["achieved_gbs"], k["frac_of_measured"],
-                                                                   k["bound"], k["single_launch_ms"],
-                                                                   k["single_launch_frac_of_measured"]))
+            cells.append("%.3f / %.0f / %.3f / %s / %s | %.3f / %.3f" % (k["ms"], k["achieved_gbs"], k["frac_of_measured"],
+                                                                        k["bound"], ("%.0f" % k["sm_mhz"]) if k.get("sm_mhz") else "-",
+                                                                        k["single_launch_ms"],
+                                                                        k["single_launch_frac_of_measured"]))
         print("| %s | %s | %.3f | %.0f |" % (b, " | ".join(cells), r["step_ms"], r["step_gradient_gbs"]))
     if line.get("model_workloads"):
         print("\n## Model-shaped workloads (Algorithm-1 order, dynamic b)\n")
