@@ -136,6 +136,33 @@ __device__ __forceinline__ uint32_t and_or(const uint32_t a, const uint32_t mask
     return d;
 }
 
+// Two fp32 values in one 64-bit register pair, for the packed two-lane forms of sm_100
+// (add.f32x2, mul.f32x2, fma.f32x2).
+__device__ __forceinline__ uint64_t pack_pair(const uint32_t lo, const uint32_t hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_pair(const uint64_t v, float& lo, float& hi)
+{
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t add_pair(const uint64_t a, const uint64_t b)
+{
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma_pair(const uint64_t a, const uint64_t b, const uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
 // Eq. 5/6 for one element.  With x = RZ(g * inv), inv = RZ(s / norm), the element's
 // position on the level grid and v = (2k + 1) / 2^17 its uniform draw (k a 16-bit
 // half of a Philox word), the code is floor(x + v) + s: for either sign the
@@ -305,6 +332,37 @@ __device__ __forceinline__ float decode_code(const uint32_t (&wd)[B], const uint
         m = and_or(__funnelshift_r(wd[P::w], wd[P::w + 1], P::sh), kCode, magic);
     }
     return __uint_as_float(m) - (8388608.0f + (float)(s << P::k));      // sgn * level * 2^k, exact
+}
+
+// The same decoding for two neighbouring codes at once with the packed two-lane fp32 forms of
+// sm_100 (add.f32x2, fma.f32x2 on 64-bit register pairs): one packed subtract and one packed FMA
+// replace two of each, which halves the operand traffic of the accumulation (the scalar form
+// keeps 32 accumulators, a scale and an immediate in flight per code).  Results are bit for bit
+// those of decode_code: the same exact subtract, the same single rounding in the FMA.
+// bits of the float 2^23 + code * 2^k for code E of a group (the part of decode_code before the subtract)
+template <int B, int E>
+__device__ __forceinline__ uint32_t code_bits(const uint32_t (&wd)[B], const uint32_t (&hi)[B], const uint32_t magic)
+{
+    using P = CodePos<B, E>;
+    constexpr uint32_t kCode = (1u << B) - 1u;
+    if constexpr (P::in_place) return and_or(wd[P::w], kCode << P::k, magic);
+    else if constexpr (P::in_upper) return and_or(hi[P::w], kCode << P::k, magic);
+    else if constexpr (!P::straddles) return and_or(wd[P::w] >> P::sh, kCode, magic);
+    else return and_or(__funnelshift_r(wd[P::w], wd[P::w + 1], P::sh), kCode, magic);
+}
+// bits of the float -(2^23 + s * 2^k): 2^23 + n has the mantissa n for every integer n < 2^23
+template <int B, int E>
+struct NegOffsetBits {
+    static constexpr uint32_t value = 0xCB000000u + (uint32_t)(((1 << (B - 1)) - 1) << CodePos<B, E>::k);
+};
+// (sgn * level * 2^k0, sgn * level * 2^k1) of codes 2Q and 2Q + 1 times (scale, scale), added to acc2
+template <int B, int Q>
+__device__ __forceinline__ uint64_t accumulate_pair(const uint64_t acc2, const uint32_t (&wd)[B], const uint32_t (&hi)[B],
+                                                    const uint64_t scale2, const uint32_t magic)
+{
+    constexpr uint64_t kOff = (uint64_t)NegOffsetBits<B, 2 * Q>::value | ((uint64_t)NegOffsetBits<B, 2 * Q + 1>::value << 32);
+    const uint64_t m = pack_pair(code_bits<B, 2 * Q>(wd, hi, magic), code_bits<B, 2 * Q + 1>(wd, hi, magic));
+    return fma_pair(add_pair(m, kOff), scale2, acc2);
 }
 
 // does any code of word W need the word's upper half?

@@ -147,18 +147,19 @@ __device__ __forceinline__ void load_words(const uint32_t* __restrict__ src, uin
     }
 }
 
-template <int B, int E>
+// The 32 sums of a group live in 16 register pairs (elements 2q and 2q + 1), see accumulate_pair.
+template <int B, int Q>
 struct AccumulateAll {
-    static __device__ __forceinline__ void run(float (&acc)[32], const uint32_t (&wd)[B], const uint32_t (&hi)[B],
-                                               const float scale, const uint32_t magic)
+    static __device__ __forceinline__ void run(uint64_t (&acc2)[16], const uint32_t (&wd)[B], const uint32_t (&hi)[B],
+                                               const uint64_t scale2, const uint32_t magic)
     {
-        acc[E] = fmaf(decode_code<B, E>(wd, hi, magic), scale, acc[E]);
-        AccumulateAll<B, E + 1>::run(acc, wd, hi, scale, magic);
+        acc2[Q] = accumulate_pair<B, Q>(acc2[Q], wd, hi, scale2, magic);
+        AccumulateAll<B, Q + 1>::run(acc2, wd, hi, scale2, magic);
     }
 };
 template <int B>
-struct AccumulateAll<B, 32> {
-    static __device__ __forceinline__ void run(float (&)[32], const uint32_t (&)[B], const uint32_t (&)[B], const float,
+struct AccumulateAll<B, 16> {
+    static __device__ __forceinline__ void run(uint64_t (&)[16], const uint32_t (&)[B], const uint32_t (&)[B], const uint64_t,
                                                const uint32_t) {}
 };
 
@@ -332,6 +333,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         // A warp whose wait for a stage ran out raises the flag, decodes no more and releases no more
         // stages; it walks on to the barrier at the tile's end, where all consumers learn of it together
         // and leave.  (Warps that were still waiting for later stages run into their own limit first.)
+        uint64_t acc2[16];
         float acc[32];
         // (test hook: every warp's first wait counts as lost, so the warps start out that way)
         bool timed_out = false, warp_out = a.wait.lose_first != 0u, x_pending = false;
@@ -340,7 +342,7 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
         int tiles_done = 0;
         for (int tile = tile_begin; tile < tile_end; ++tile) {
 #pragma unroll
-            for (int e = 0; e < 32; ++e) acc[e] = 0.0f;
+            for (int q = 0; q < 16; ++q) acc2[q] = 0ull;
             for (int c = 0; c < nchunk; ++c, ++u) {
                 const int m0 = c * MC;
                 const int mc = (M - m0) < MC ? (M - m0) : MC;
@@ -390,7 +392,8 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                             uint32_t wd[B], hi[B];
                             load_words<B>(base + j * (kThreads * B), wd);
                             UpperHalves<B, 0>::run(base + j * (kThreads * B), hi);
-                            AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
+                            const uint32_t sc = __float_as_uint(my_scales[j * kThreads]);
+                            AccumulateAll<B, 0>::run(acc2, wd, hi, pack_pair(sc, sc), magic);
                         }
                     } else {
 #pragma unroll 1
@@ -398,7 +401,8 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                             uint32_t wd[B], hi[B];
                             load_words<B>(base + j * (kThreads * B), wd);
                             UpperHalves<B, 0>::run(base + j * (kThreads * B), hi);
-                            AccumulateAll<B, 0>::run(acc, wd, hi, my_scales[j * kThreads], magic);
+                            const uint32_t sc = __float_as_uint(my_scales[j * kThreads]);
+                            AccumulateAll<B, 0>::run(acc2, wd, hi, pack_pair(sc, sc), magic);
                         }
                     }
                 }
@@ -416,6 +420,8 @@ __device__ __forceinline__ void average_tiles(const AverageArgs& a, const CUtens
                 if (tid == 0) tma::store_wait_read();
             }
             if (consumer_sync_or(warp_out || *abort_flag() != 0)) { timed_out = true; break; }
+#pragma unroll
+            for (int q = 0; q < 16; ++q) unpack_pair(acc2[q], acc[2 * q], acc[2 * q + 1]);
             Normalise<B, 0>::run(acc);
             if (valid < 32) {
 #pragma unroll
