@@ -364,6 +364,44 @@ def _model_workload(torch, dq, Round, timer, w, gen_fn, dev, K, peak):
     return out
 
 
+SWEEP_B = (2, 4, 8)
+# the other axes of the bandwidth sweep: (M, log2 d, bucket); the per-b table covers (32, 26, 512)
+SWEEP_POINTS = ((1, 24, 512), (1, 26, 512), (1, 28, 512), (1, 30, 512), (32, 26, 128), (32, 26, 4096))
+
+
+def _sweep_point(torch, dq, Round, timer, M, log2d, bucket, K, dev, peak):
+    """Trains of the fused quantizer and of the average at one (M, d, bucket) of the bandwidth sweep.
+    Small cases rotate through several sets of buffers so that every launch reads more than the L2 holds
+    since it last saw the same addresses."""
+    d = 1 << log2d
+    n_rot = max(1, min(8, -(-(1 << 29) // (4 * M * d))))
+    rounds = [Round([d], bucket, M, device=str(dev)) for _ in range(n_rot)]
+    D32 = rounds[0].layout.D32
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(SEED + log2d + bucket)
+    grads = [torch.randn((M, D32), generator=gen, device=dev, dtype=torch.float32) for _ in range(n_rot)]
+    elems = M * D32
+    rec = {"M": M, "d": d, "bucket": bucket, "buffer_sets": n_rot, "mb_per_launch": (4 * elems) >> 20, "b": {}}
+    for b in SWEEP_B:
+        for r, g in zip(rounds, grads):
+            r.bits_(dq.Rule.fixed(b))
+            r.norms_quantize_(g, SEED, 0)
+        t_f = timer.train(lambda i: rounds[i % n_rot].norms_quantize_(grads[i % n_rot], SEED, i), K)
+        t_a = timer.train(lambda i: rounds[i % n_rot].average_(), K)
+        bytes_f = (4.0 + b / 8.0) * elems
+        bytes_a = (M * b / 8.0 + 4.0) * D32
+        rec["b"][str(b)] = {
+            "norms_quantize_pack": {"ms": round(t_f, 5), "achieved_gbs": round(bytes_f / (t_f * 1e-3) / 1e9, 1),
+                                    "frac_of_measured": round(bytes_f / (t_f * 1e-3) / 1e9 / peak, 4)},
+            "unpack_dequant_average": {"ms": round(t_a, 5), "achieved_gbs": round(bytes_a / (t_a * 1e-3) / 1e9, 1),
+                                       "frac_of_measured": round(bytes_a / (t_a * 1e-3) / 1e9 / peak, 4)}}
+        for r in rounds:
+            assert r.read_status() == 0, "device status %d" % r.read_status()
+    del rounds, grads
+    torch.cuda.empty_cache()
+    return rec
+
+
 def run_cuda(args) -> dict:
     import torch
     import torch.distributed as dist
@@ -512,12 +550,16 @@ def run_cuda(args) -> dict:
     if not args.no_e2e:
         e2e = _end_to_end(torch, dist, rnd, grads, rule_b, K, world, dev, M, d, D32)
 
-    # ---- the model-shaped workloads (secondary)
+    # ---- the other sizes and bucket lengths of the bandwidth sweep, then the model-shaped workloads (secondary)
     other = None
-    if not args.no_models:
+    sweep = None
+    if not (args.no_models and args.no_sweep):
         del grads
         rnd = None
         torch.cuda.empty_cache()
+    if not args.no_sweep:
+        sweep = [_sweep_point(torch, dq, Round, timer, m_, l_, bk_, K, dev, peak) for m_, l_, bk_ in SWEEP_POINTS]
+    if not args.no_models:
         other = {}
         for w, gen_fn in ((workloads.config_resnet18(), _gen_resnet), (workloads.config_vgg16(), _gen_vgg),
                           (workloads.config_text(), _gen_text)):
@@ -533,13 +575,15 @@ def run_cuda(args) -> dict:
                    "l2": "inputs larger than L2 (%d MB of gradients per step)" % ((4 * elems) >> 20),
                    "per_b": "b in %s: trains of %d launches and %d single event-bracketed launches per kernel"
                             % (list(PER_B), K, n_single),
+                   "size_sweep": "M=1 at d=2^24..2^30 and buckets 128/4096 at d=2^26, M=32, b in %s: trains of %d launches, "
+                                 "buffers rotated where one set would fit in the L2" % (list(SWEEP_B), K),
                    "multi_gpu": "independent replicas, no collective" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": 4 * K, "roofline": roofline,
         "per_b": per_b, "bucket_norms": _bound("bucket_norms", 0, 4.0 * elems, groups, norms_ms, peak, sm_count, sm_mhz),
         # what the workers would put on the wire per step (Eq. 7: d * b bits per worker, plus the fp32 norms)
         "wire": {"bytes_per_step": M * (d * HEADLINE_B / 8.0 + 4.0 * L.nb), "fp32_bytes_per_step": 4.0 * M * d,
                  "ratio": round((d * HEADLINE_B / 8.0 + 4.0 * L.nb) / (4.0 * d), 4)},
-        "model_workloads": other, "host_submit_ms_per_step": round(host_submit_ms, 5),
+        "size_sweep": sweep, "model_workloads": other, "host_submit_ms_per_step": round(host_submit_ms, 5),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = _cpu_baseline(torch, gen, dev)
@@ -596,6 +640,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the CPU checker timing (profiling runs)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the M = 1 sizes and the other bucket lengths of the bandwidth sweep")
     ap.add_argument("--no-models", action="store_true", help="skip the secondary timing of the model-shaped workloads")
     ap.add_argument("--no-per-b", action="store_true", help="skip the per-b table (profiling runs)")
     ap.add_argument("--no-overlap", action="store_true",

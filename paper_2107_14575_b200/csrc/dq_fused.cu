@@ -14,9 +14,8 @@
 // with 16-byte coalesced stores through the consumed stage.
 //  * Buckets of up to 1024 elements (gpb = bucket / 32 <= 32): tiles of 32 / gpb buckets, fetched
 //    two tiles ahead.
-//  * Buckets of 2048 elements: a warp takes a whole bucket through its two stages.
-//  * Buckets of 4096 elements: a pair of warps takes a bucket, 2048 elements each, and
-//    exchanges four partial results through shared memory.
+//  * Buckets of 2048 and 4096 elements: a team of 2 or 4 warps takes a bucket, 1024 elements each,
+//    and exchanges the partial results through shared memory; every warp fetches one bucket ahead.
 // HBM traffic: 4 + b/8 bytes per element.
 #include "dq_common.cuh"
 #include "dq_device.cuh"
@@ -39,11 +38,11 @@ constexpr int kWTileBytes = 32 * 128;
 constexpr int kWBarOffset = kWarps * kWStages * kWTileBytes;
 constexpr int kWTblOffset = kWBarOffset + kWarps * kWStages * 8;
 
-// The whole-bucket kernel adds, between the stage barriers and the tensor table, one barrier and two
-// slots of four partial results for each pair of warps that share a bucket of 4096 elements.
-constexpr int kPairBarOffset = kWTblOffset;
-constexpr int kPairPartOffset = kPairBarOffset + (kWarps / 2) * 8;
-constexpr int kBTblOffset = kPairPartOffset + (kWarps / 2) * 2 * 4 * 4;
+// The team kernel adds, between the stage barriers and the tensor table, one barrier and two
+// slots of four partial results for each team of warps that share a bucket (room for two teams).
+constexpr int kTeamBarOffset = kWTblOffset;
+constexpr int kTeamPartOffset = kTeamBarOffset + (kWarps / 2) * 8;
+constexpr int kBTblOffset = kTeamPartOffset + (kWarps / 2) * 2 * 4 * 4;
 
 __device__ __forceinline__ uint64_t* wbar(int warp, int st)
 {
@@ -492,6 +491,8 @@ __device__ __forceinline__ void fused_warp_tiles(const FusedArgs& a, const CUten
 // Five CTAs per SM (up to 102 registers per thread): at six (80 registers) the widest bit widths
 // spill in the tile loop, and the kernel, bound by instruction issue, loses nothing at 20 warps per SM.
 constexpr int kWarpKernelCtasPerSm = 5;
+// The team kernel likewise: five CTAs per SM measured 2-4 % faster than six and than four.
+constexpr int kTeamKernelCtasPerSm = 5;
 template <int P>
 __global__ void __launch_bounds__(kThreads, kWarpKernelCtasPerSm)
 norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
@@ -530,19 +531,20 @@ norms_quantize_pack_warp_kernel(const __grid_constant__ FusedArgs a, const __gri
     }
 }
 
-// ---- buckets of 2048 and 4096 elements: a warp takes 2048 elements through its two stages ----
+// ---- buckets of 2048 and 4096 elements: a team of T = 2 or 4 warps takes a bucket, one warp tile each ----
 //
-// A bucket of 64 groups is two warp tiles.  The warp fetches them into its two stages, every
-// lane squares its row of each, the two halves are reduced by the same butterflies and added
-// in the same order as dq_bucket_norms does, and the rows are then encoded half by half: as
-// soon as a half has left for the packed stream, its stage is refilled with the matching half
-// of the warp's next bucket, so that the fetch runs beside the encoding of the other half.
-// Short buckets (a tensor's last) and padding take the same route with per-lane valid counts.
-// H = 2: a bucket of 128 groups belongs to a pair of warps, 64 groups each; the pair exchanges its
-// four partial results through shared memory (a barrier of its own, waited for with the usual
-// limit) and both warps add them in the order of dq_bucket_norms.
-template <int B, int P, int H>
-__device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUtensorMap* map)
+// Warp `sub` of the team owns elements [1024 sub, 1024 sub + 1024) of every bucket of the team's range.
+// Its two stages alternate between consecutive buckets: while the tile of bucket i is reduced and
+// encoded in one stage, the tile of bucket i + 1 is on its way into the other, and as soon as the
+// words of bucket i have left, that stage is refilled with the tile of bucket i + 2 -- every warp
+// keeps one whole tile in flight for the length of a bucket.  Every lane squares its row, the warp
+// combines by the butterflies of dq_bucket_norms, and the T partial results are exchanged through
+// shared memory (a barrier of the team's own, waited for with the usual limit; every exchange is
+// one phase of it and uses the slots of that phase's parity) and added by every warp in the order
+// of dq_bucket_norms.  Short buckets (a tensor's last) and padding take the same route with
+// per-lane valid counts; a warp whose share of a bucket is empty fetches nothing and contributes 0.
+template <int B, int P, int T>
+__device__ __forceinline__ void fused_team_buckets(const FusedArgs& a, const CUtensorMap* map)
 {
     const int32_t* tbl_s = reinterpret_cast<const int32_t*>(smem + kBTblOffset);
     constexpr int s = (1 << (B - 1)) - 1;
@@ -550,51 +552,62 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n1 = a.v.n_seg + 1;
     const int nb = a.v.nb;
-    constexpr int kBucket = 2048 * H;
-    const int sub = warp % H;                     // which 2048 elements of the bucket this warp takes
+    constexpr int kBucket = 1024 * T;
+    const int sub = warp % T;                     // which 1024 elements of the bucket this warp takes
     const int64_t total = (int64_t)a.M * nb;
-    const int64_t nteams = (int64_t)gridDim.x * (kWarps / H);
-    const int64_t team = (int64_t)blockIdx.x * (kWarps / H) + warp / H;
+    const int64_t nteams = (int64_t)gridDim.x * (kWarps / T);
+    const int64_t team = (int64_t)blockIdx.x * (kWarps / T) + warp / T;
     const int64_t begin = team * total / nteams;
     const int n_tiles = (int)((team + 1) * total / nteams - begin);
-    if (n_tiles <= 0) return;
+    if (n_tiles <= 0) return;                     // (the whole team: its warps share `team`)
 
+    struct Pos { int m, k, g0, len; };            // worker, bucket, first group and valid elements of the warp's share
     int seg = 0;                                  // walking hint: buckets only move forward inside a worker
-    auto locate = [&](int k, int& g0, int& len) {
+    auto locate = [&](Pos& p) {
         int local, n, gs;
         if (a.v.n_seg == 1) {
-            local = k; n = a.v.seg0_elems; gs = 0;
+            local = p.k; n = a.v.seg0_elems; gs = 0;
         } else {
-            while (k >= tbl_s[n1 + seg + 1]) ++seg;
-            local = k - tbl_s[n1 + seg];
+            while (p.k >= tbl_s[n1 + seg + 1]) ++seg;
+            local = p.k - tbl_s[n1 + seg];
             n = tbl_s[2 * n1 + seg];
             gs = tbl_s[seg];
         }
-        g0 = gs + local * (64 * H) + 64 * sub;    // first group and valid elements of this warp's share
-        int left = n - local * kBucket - 2048 * sub;
+        p.g0 = gs + local * (32 * T) + 32 * sub;
+        int left = n - local * kBucket - 1024 * sub;
         left = left < 0 ? 0 : left;
-        len = left < 2048 ? left : 2048;
+        p.len = left < 1024 ? left : 1024;
     };
-    auto issue = [&](int st, int row0, int mm) {
+    // the bucket after p (located only if the team's range holds it)
+    auto successor = [&](const Pos& p, bool exists) -> Pos {
+        Pos q;
+        q.m = p.m; q.k = p.k + 1; q.g0 = 0; q.len = 0;
+        if (q.k == nb) { q.k = 0; ++q.m; seg = 0; }
+        if (exists) locate(q);
+        return q;
+    };
+    auto issue = [&](int st, const Pos& p) {
         tma::mbar_expect_tx(wbar(warp, st), kWTileBytes);
         if (a.stream_reads)
-            tma::load_tile_3d_hint(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? mm : 0,
+            tma::load_tile_3d_hint(wstage(warp, st), map, wbar(warp, st), 0, p.g0, a.map_has_worker_dim ? p.m : 0,
                                    tma::policy_evict_first());
         else
-            tma::load_tile_3d(wstage(warp, st), map, wbar(warp, st), 0, row0, a.map_has_worker_dim ? mm : 0);
+            tma::load_tile_3d(wstage(warp, st), map, wbar(warp, st), 0, p.g0, a.map_has_worker_dim ? p.m : 0);
     };
 
-    int m = (int)(begin / nb), k = (int)(begin - (int64_t)m * nb);
-    int g0, len;
-    locate(k, g0, len);
+    Pos cur;
+    cur.m = (int)(begin / nb);
+    cur.k = (int)(begin - (int64_t)cur.m * nb);
+    locate(cur);
+    Pos nxt = successor(cur, n_tiles > 1);
     if (lane == 0) {
-        if (len > 0) issue(0, g0, m);
-        if (len > 1024) issue(1, g0 + 32, m);
+        if (cur.len > 0) issue(0, cur);
+        if (nxt.len > 0) issue(1, nxt);
     }
-    bool pend_a = len > 0, pend_b = len > 1024;
-    uint32_t ph_a = 0, ph_b = 0;
-    uint64_t* pair_bar = reinterpret_cast<uint64_t*>(smem + kPairBarOffset) + warp / 2;
-    float* pair_part = reinterpret_cast<float*>(smem + kPairPartOffset) + (warp / 2) * 8;
+    bool pend0 = cur.len > 0, pend1 = nxt.len > 0;       // a copy into the stage has not been seen to land
+    uint32_t ph0 = 0, ph1 = 0;                            // copies into the stage seen to land
+    uint64_t* team_bar = reinterpret_cast<uint64_t*>(smem + kTeamBarOffset) + warp / T;
+    float* team_part = reinterpret_cast<float*>(smem + kTeamPartOffset) + (warp / T) * 8;
     bool timed_out = false, bad = false;
     // byte offset of this lane's row inside a stage, swizzle phase folded in: chunk c sits at own ^ (c << 4)
     const uint32_t own = (uint32_t)(lane * 128 + ((lane & 7) << 4));
@@ -619,31 +632,28 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
         for (int o = 16; o > 0; o >>= 1) sum = red.join(sum, __shfl_xor_sync(0xffffffffu, sum, o));
         return sum;
     };
-    // One reduction of the bucket: the warp's two halves and, for a pair of warps, the exchange of
-    // the four partial results (every exchange is one phase of the pair's barrier and uses the
-    // slot of that phase's parity).  False if the wait for the other warp ran out.
+    // One reduction of the bucket: the warp's tile, then the exchange of the team's T partial results.
+    // False if the wait for the other warps ran out.
     uint32_t exchanges = 0;
-    auto bucket_reduce = [&](const auto& red, int rows, int valid_a, int valid_b, float& result) -> bool {
-        const float part_a = rows > 0 ? row_reduce(red, wstage(warp, 0), valid_a) : 0.0f;
-        const float part_b = rows > 32 ? row_reduce(red, wstage(warp, 1), valid_b) : 0.0f;
-        if constexpr (H == 1) {
-            result = red.join(red.join(0.0f, part_a), part_b);
-        } else {
-            float* slot = pair_part + (exchanges & 1u) * 4;
-            if (lane == 0) {
-                slot[2 * sub] = part_a;
-                slot[2 * sub + 1] = part_b;
-                tma::mbar_arrive(pair_bar);
-            }
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(pair_bar, exchanges & 1u, a.wait))) return false;
-            ++exchanges;
-            result = red.join(red.join(red.join(red.join(0.0f, slot[0]), slot[1]), slot[2]), slot[3]);
+    auto bucket_reduce = [&](const auto& red, const unsigned char* base, int rows, int valid, float& result) -> bool {
+        const float part = rows > 0 ? row_reduce(red, base, valid) : 0.0f;
+        float* slot = team_part + (exchanges & 1u) * 4;
+        __syncwarp();                            // the lanes are done with the slots of two exchanges ago
+        if (lane == 0) {
+            slot[sub] = part;
+            tma::mbar_arrive(team_bar);
         }
+        if (!__all_sync(0xffffffffu, tma::mbar_wait(team_bar, exchanges & 1u, a.wait))) return false;
+        ++exchanges;
+        float r = red.join(0.0f, slot[0]);
+#pragma unroll
+        for (int i = 1; i < T; ++i) r = red.join(r, slot[i]);
+        result = r;
         return true;
     };
-    // encodes the lane's row of a stage against `inv`, stages the half's words in the stage itself and
-    // sends them to the packed stream; `row0` is the half's first group, `span` its number of groups
-    auto encode_half = [&](unsigned char* base, int row0, int valid, int span, float inv, int mm) {
+    // encodes the lane's row of a stage against `inv`, stages the tile's words in the stage itself and
+    // sends them to the packed stream; `row0` is the tile's first group, `span` its number of groups
+    auto encode_tile = [&](unsigned char* base, int row0, int valid, int span, float inv, int mm) {
         uint32_t acc[B];
         if (valid > 0) {
             unsigned char* rowp = base + lane * 128;
@@ -657,10 +667,10 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
             } else if (inv == 0.0f) {            // a zero bucket (the whole warp works on one bucket)
                 zero_group_words<B>(acc);
             } else {
-                uint32_t cur = 0;
+                uint32_t cur_bits = 0;
                 const uint32_t q0 = (uint32_t)(row0 + lane) * 4u;
 #define DQ_BLOCK(C)                                                                                             \
-                encode_block<B, C>(acc, cur,                                                                    \
+                encode_block<B, C>(acc, cur_bits,                                                               \
                                    *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C)) ^ sw) << 4)), \
                                    *reinterpret_cast<const float4*>(rowp + (((uint32_t)(2 * (C) + 1) ^ sw) << 4)), \
                                    inv, q0 + (C), (uint32_t)mm + a.worker0, a.step, a.keys, a.one_bits);
@@ -692,77 +702,60 @@ __device__ __forceinline__ void fused_warp_buckets(const FusedArgs& a, const CUt
     // test hook: the warp's first wait counts as lost, and the warp goes straight to what follows a time-out
     timed_out = a.wait.lose_first != 0u;
     for (int it = 0; it < n_tiles && !timed_out; ++it) {
-        const int rows = (len + 31) >> 5;
-        // the warp's next bucket (its halves are fetched as this one's halves leave)
-        int nm = m, nk = k + 1, ng0 = 0, nlen = 0;
-        const bool has_next = it + 1 < n_tiles;
-        if (nk == nb) { nk = 0; ++nm; }
-        if (has_next) {
-            if (nm != m) seg = 0;
-            locate(nk, ng0, nlen);
-        }
-
+        const int st = it & 1;
+        unsigned char* base = wstage(warp, st);
+        const int rows = (cur.len + 31) >> 5;
         if (rows > 0) {
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 0), ph_a & 1u, a.wait))) {
+            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, st), (st ? ph1 : ph0) & 1u, a.wait))) {
                 timed_out = true;
                 break;
             }
-            pend_a = false; ++ph_a;
+            if (st) { pend1 = false; ++ph1; } else { pend0 = false; ++ph0; }
         }
-        if (rows > 32) {
-            if (!__all_sync(0xffffffffu, tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait))) { timed_out = true; break; }
-            pend_b = false; ++ph_b;
-        }
-        int valid_a = len - lane * 32;
-        valid_a = valid_a < 0 ? 0 : (valid_a > 32 ? 32 : valid_a);
-        int valid_b = len - (lane + 32) * 32;
-        valid_b = valid_b < 0 ? 0 : (valid_b > 32 ? 32 : valid_b);
+        int valid = cur.len - lane * 32;
+        valid = valid < 0 ? 0 : (valid > 32 ? 32 : valid);
 
         float sum;
-        if (!bucket_reduce(typename FamilyReduction<P>::type{}, rows, valid_a, valid_b, sum)) { timed_out = true; break; }
+        if (!bucket_reduce(typename FamilyReduction<P>::type{}, base, rows, valid, sum)) { timed_out = true; break; }
         float nrm = finish<P>(sum);
         if constexpr (P == DQ_NORM_L2) {
-            // every lane of the warp, and both warps of a pair, hold the same sum: the verdict is uniform
+            // every lane of every warp of the team holds the same sum: the verdict is uniform
             if (!l2_sum_in_range(sum)) {
                 float mx, scaled;
-                if (!bucket_reduce(MaxMagnitude{}, rows, valid_a, valid_b, mx)) { timed_out = true; break; }
+                if (!bucket_reduce(MaxMagnitude{}, base, rows, valid, mx)) { timed_out = true; break; }
                 const int e = scale_exponent(mx);
-                if (!bucket_reduce(ScaledSquares{e}, rows, valid_a, valid_b, scaled)) { timed_out = true; break; }
+                if (!bucket_reduce(ScaledSquares{e}, base, rows, valid, scaled)) { timed_out = true; break; }
                 nrm = rescaled_l2(mx, scaled, e);
             }
         }
         if (lane == 0 && sub == 0) {
-            DQ_STORE(a.norms + ((int64_t)m * nb + k), nrm, a.norms, (int64_t)a.M * a.v.nb * 4, a.status);
+            DQ_STORE(a.norms + ((int64_t)cur.m * nb + cur.k), nrm, a.norms, (int64_t)a.M * a.v.nb * 4, a.status);
             bad |= !isfinite(nrm);
         }
         const float inv = inv_scale(sf, nrm);
 
-        if (rows > 0) encode_half(wstage(warp, 0), g0, valid_a, rows < 32 ? rows : 32, inv, m);
-        if (has_next && nlen > 0) {
-            if (lane == 0) issue(0, ng0, nm);
-            pend_a = true;
+        if (rows > 0) encode_tile(base, cur.g0, valid, rows, inv, cur.m);
+        // the stage is free: the warp's tile of the bucket after next goes there
+        const Pos after = successor(nxt, it + 2 < n_tiles);
+        if (after.len > 0) {
+            if (lane == 0) issue(st, after);
+            if (st) pend1 = true; else pend0 = true;
         }
-        if (rows > 32) {
-            encode_half(wstage(warp, 1), g0 + 32, valid_b, rows - 32, inv, m);
-        }
-        if (has_next && nlen > 1024) {
-            if (lane == 0) issue(1, ng0 + 32, nm);
-            pend_b = true;
-        }
-        m = nm; k = nk; g0 = ng0; len = nlen;
+        cur = nxt;
+        nxt = after;
     }
     if (bad) atomicOr(a.status, DQ_STAT_NONFINITE);
     if (timed_out) {
         if (lane == 0) atomicOr(a.status, DQ_STAT_WAIT);
         // every copy the warp has issued and not seen land, the one whose wait ran out included, gets the
         // full limit before the CTA's shared memory is released
-        if (pend_a) (void)tma::mbar_wait(wbar(warp, 0), ph_a & 1u, a.wait);
-        if (pend_b) (void)tma::mbar_wait(wbar(warp, 1), ph_b & 1u, a.wait);
+        if (pend0) (void)tma::mbar_wait(wbar(warp, 0), ph0 & 1u, a.wait);
+        if (pend1) (void)tma::mbar_wait(wbar(warp, 1), ph1 & 1u, a.wait);
     }
 }
 
-template <int P, int H>
-__global__ void __launch_bounds__(kThreads, 6)
+template <int P, int T>
+__global__ void __launch_bounds__(kThreads, kTeamKernelCtasPerSm)
 norms_quantize_pack_bucket_kernel(const __grid_constant__ FusedArgs a, const __grid_constant__ CUtensorMap map)
 {
     grid_dependency_wait();
@@ -778,7 +771,7 @@ norms_quantize_pack_bucket_kernel(const __grid_constant__ FusedArgs a, const __g
     if (threadIdx.x == 0) {
         tma::prefetch_tensor_map(&map);
         for (int i = 0; i < kWarps * kWStages; ++i) tma::mbar_init(wbar(0, i), 1);
-        for (int i = 0; i < kWarps / 2; ++i) tma::mbar_init(reinterpret_cast<uint64_t*>(smem + kPairBarOffset) + i, 2);
+        for (int i = 0; i < kWarps / T; ++i) tma::mbar_init(reinterpret_cast<uint64_t*>(smem + kTeamBarOffset) + i, T);
         tma::fence_barrier_init();
     }
     __syncthreads();
@@ -792,7 +785,7 @@ norms_quantize_pack_bucket_kernel(const __grid_constant__ FusedArgs a, const __g
     }
 
     switch (b) {
-#define DQ_CASE(BB) case BB: fused_warp_buckets<BB, P, H>(a, &map); break;
+#define DQ_CASE(BB) case BB: fused_team_buckets<BB, P, T>(a, &map); break;
         DQ_CASE(1) DQ_CASE(2) DQ_CASE(3) DQ_CASE(4) DQ_CASE(5) DQ_CASE(6) DQ_CASE(7) DQ_CASE(8)
         DQ_CASE(9) DQ_CASE(10) DQ_CASE(11) DQ_CASE(12) DQ_CASE(13) DQ_CASE(14) DQ_CASE(15) DQ_CASE(16)
 #undef DQ_CASE
@@ -848,7 +841,7 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
     a.map_has_worker_dim = worker_dim ? 1 : 0;
 
     const bool per_warp = gpb <= 32;
-    // otherwise gpb is 64 or 128: 2048 elements per warp through both of its stages
+    // otherwise gpb is 64 or 128: a team of 2 or 4 warps per bucket
     CUtensorMap map;
     const uint64_t dims[3] = {32, (uint64_t)a.v.total_groups, worker_dim ? (uint64_t)M : 1};
     const uint64_t strides[2] = {128, worker_dim ? (uint64_t)worker_stride_elems * 4 : (uint64_t)L->padded * 4};
@@ -875,17 +868,17 @@ extern "C" int dq_norms_quantize_pack_worker(const dq_layout_t* L, const float* 
     } else {
         const size_t smem_need = (size_t)kBTblOffset + tbl_bytes;
         const bool linf = (L->norm == DQ_NORM_LINF);
-        const auto kernel = gpb == 64 ? (linf ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF, 1>
-                                              : norms_quantize_pack_bucket_kernel<DQ_NORM_L2, 1>)
-                                      : (linf ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF, 2>
-                                              : norms_quantize_pack_bucket_kernel<DQ_NORM_L2, 2>);
+        const auto kernel = gpb == 64 ? (linf ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF, 2>
+                                              : norms_quantize_pack_bucket_kernel<DQ_NORM_L2, 2>)
+                                      : (linf ? norms_quantize_pack_bucket_kernel<DQ_NORM_LINF, 4>
+                                              : norms_quantize_pack_bucket_kernel<DQ_NORM_L2, 4>);
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)smem_need) != cudaSuccess) {
             (void)cudaGetLastError();
             return DQ_ERR_CUDA;
         }
-        const int64_t warp_tiles = (int64_t)M * L->nb * (gpb / 64);
-        int64_t blocks = (int64_t)dq_sm_count() * 6;   // six 33 KB CTAs per SM
+        const int64_t warp_tiles = (int64_t)M * L->nb * (gpb / 32);        // no more teams than buckets
+        int64_t blocks = (int64_t)dq_sm_count() * kTeamKernelCtasPerSm;
         if (blocks * kWarps > warp_tiles) blocks = (warp_tiles + kWarps - 1) / kWarps;
         dq_launch(kernel, dim3((unsigned)blocks), dim3(kThreads), smem_need, static_cast<cudaStream_t>(stream), a, map);
     }

@@ -249,6 +249,21 @@ def cmd_table(a) -> None:
                                                                         k["single_launch_ms"],
                                                                         k["single_launch_frac_of_measured"]))
         print("| %s | %s | %.3f | %.0f |" % (b, " | ".join(cells), r["step_ms"], r["step_gradient_gbs"]))
+    if line.get("size_sweep"):
+        print("\n## Other sizes and bucket lengths of the bandwidth sweep\n")
+        print("Trains of launches; cases whose buffers would fit in the L2 rotate through `sets` sets of buffers.  "
+              "Cells: ms per launch / GB/s of algorithmic bytes / fraction of the copy bandwidth.\n")
+        bs = sorted(line["size_sweep"][0]["b"], key=int)
+        print("| M | d | bucket | MB/launch | sets | " + " | ".join("fused b=%s | average b=%s" % (b, b) for b in bs) + " |")
+        print("|---|---|---|---|---|" + "---|---|" * len(bs))
+        for pt in line["size_sweep"]:
+            cells = []
+            for b in bs:
+                for n in ("norms_quantize_pack", "unpack_dequant_average"):
+                    k = pt["b"][b][n]
+                    cells.append("%.4f / %.0f / %.3f" % (k["ms"], k["achieved_gbs"], k["frac_of_measured"]))
+            print("| %d | 2^%d | %d | %d | %d | %s |" % (pt["M"], pt["d"].bit_length() - 1, pt["bucket"], pt["mb_per_launch"],
+                                                      pt["buffer_sets"], " | ".join(cells)))
     if line.get("model_workloads"):
         print("\n## Model-shaped workloads (Algorithm-1 order, dynamic b)\n")
         print("| workload | MB/step | ms/step | GB/s of gradient | b first..last | fused ms (frac) | average ms (frac) |")
