@@ -92,7 +92,11 @@ class Round:
         self.average_()
         return self.out
 
-    def step_fused(self, grads, next_rule: dq.Rule, seed: int, step: int, overlap: bool = True,
+    # below this many norms the bit rule takes a few microseconds and the hand-over between two
+    # streams costs more than running it behind the average on the same stream
+    OVERLAP_MIN_NORMS = 1 << 20
+
+    def step_fused(self, grads, next_rule: dq.Rule, seed: int, step: int, overlap: Optional[bool] = None,
                    events=None, params=None, lr: float = 0.0) -> torch.Tensor:
         """One round in the order of Algorithm 1: quantize with the b chosen after the
         previous round (one pass over the gradients), average, and choose the next b from
@@ -101,7 +105,10 @@ class Round:
 
         With ``overlap`` the bit rule runs on a second stream next to the average: it needs
         only the norms, and writes the other (b, s) slot.  The current stream waits for it
-        before it goes on.  ``events`` = (e0, e1, e2, s0, s1) are recorded around the three
+        before it goes on.  ``overlap=None`` decides by size: a second stream for
+        ``OVERLAP_MIN_NORMS`` norms or more, one stream below (measured on the ResNet-18
+        shape, 175k norms: 102.5 us per step on one stream, 104.2 us with two; at 4.2M
+        norms the second stream hides 85 us of bit rule).  ``events`` = (e0, e1, e2, s0, s1) are recorded around the three
         calls (e* on the current stream, s* around the bit rule on its own stream).
 
         With ``params`` (fp32 [D32] in the padded layout) the server step also applies the
@@ -114,6 +121,8 @@ class Round:
             else:
                 self.update_(params, lr)
         result = self.out if params is None else params
+        if overlap is None:
+            overlap = self.M * self.layout.nb >= self.OVERLAP_MIN_NORMS
         main = torch.cuda.current_stream(self.device)
         if events:
             events[0].record(main)
