@@ -14,7 +14,9 @@ point b = 4 (chosen on the device by the rule of Eq. 17, calibrated so); the
 in one pass, unpack+average -- for a list of bit widths, each as a train of launches
 and as single event-bracketed launches, with achieved GB/s of algorithmic bytes, the
 fraction of the measured copy bandwidth and of 8 TB/s, and which roof binds.
-The model-shaped workloads (ResNet-18 M = 8, VGG-16 M = 16, text classifier M = 16)
+``size_sweep`` times the fused quantizer and the average on the other axes of the
+sweep (M = 1 at d = 2^24 .. 2^30; buckets of 128 and 4096 at d = 2^26, M = 32), and the
+model-shaped workloads (ResNet-18 M = 8, VGG-16 M = 16, text classifier M = 16)
 are timed as secondary figures.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
