@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 FILES = ["tests/test_gpu_parity.py", "tests/test_gpu_fuzz.py", "tests/test_gpu_norm_range.py",
-         "tests/test_gpu_norm_family.py"]
+         "tests/test_gpu_norm_family.py", "tests/test_gpu_team_route.py"]
 
 
 def test_small_case_parity_files_pass_on_the_checked_build():
