@@ -348,19 +348,35 @@ def _model_workload(torch, dq, Round, timer, w, gen_fn, dev, K, peak):
     b0 = rnd.bits()
     ms = timer.train(lambda i: rnd.step_fused(pool[i % npool], rule_for(i + 1), SEED, i), K)
     b1 = rnd.bits()
-    # per call, event-bracketed, at the b the schedule has reached
+    # per call at the b the schedule has reached: event-bracketed single launches (the bracket leaves the GPU idle
+    # for some microseconds around every launch, which counts) and trains of launches; the trains rotate through
+    # `npool` sets of buffers (gradients for the quantizer, words and outputs for the average), more than the L2 holds
     elems = w.M * L.D32
     t_f = timer.single(lambda i: rnd.norms_quantize_(pool[i % npool], SEED, i), min(K, 10))
     t_a = timer.single(lambda i: rnd.average_(), min(K, 10))
-    assert rnd.read_status() == 0, "device status %d" % rnd.read_status()
+    rounds = [rnd] + [Round(w.segments, w.bucket, w.M, device=str(dev)) for _ in range(npool - 1)]
+    for r, g in zip(rounds, pool):
+        r.bits_(dq.Rule.fixed(b1))
+        r.norms_quantize_(g, SEED, 0)
+    t_f_train = timer.train(lambda i: rnd.norms_quantize_(pool[i % npool], SEED, i), 3 * K)
+    t_a_train = timer.train(lambda i: rounds[i % npool].average_(), 3 * K)
+    for r in rounds:
+        assert r.read_status() == 0, "device status %d" % r.read_status()
+    bytes_f = (4.0 + b1 / 8.0) * elems
+    bytes_a = (w.M * b1 / 8.0 + 4.0) * L.D32
     out = {"workload": "%s: %d tensors, d=%d fp32/worker, M=%d, bucket=%d, dynamic b over T=%d"
                        % (w.name, len(w.segments), w.d, w.M, w.bucket, w.T),
            "ms_per_step": round(ms, 5), "value": round(4.0 * w.M * w.d / (ms * 1e-3) / 1e9, 1),
            "bits_first_last": [b0, b1], "mb_per_step": (4 * elems) >> 20,
            "norms_quantize_pack": {"b": b1, "ms": round(t_f, 5),
-                                   "frac_of_measured": round((4.0 + b1 / 8.0) * elems / (t_f * 1e-3) / 1e9 / peak, 4)},
+                                   "frac_of_measured": round(bytes_f / (t_f * 1e-3) / 1e9 / peak, 4),
+                                   "train_ms": round(t_f_train, 5),
+                                   "train_frac_of_measured": round(bytes_f / (t_f_train * 1e-3) / 1e9 / peak, 4)},
            "unpack_dequant_average": {"b": b1, "ms": round(t_a, 5),
-                                      "frac_of_measured": round((w.M * b1 / 8.0 + 4.0) * L.D32 / (t_a * 1e-3) / 1e9 / peak, 4)}}
+                                      "frac_of_measured": round(bytes_a / (t_a * 1e-3) / 1e9 / peak, 4),
+                                      "train_ms": round(t_a_train, 5),
+                                      "train_frac_of_measured": round(bytes_a / (t_a_train * 1e-3) / 1e9 / peak, 4)}}
+    del rounds
     del pool, rnd
     torch.cuda.empty_cache()
     return out
@@ -552,20 +568,20 @@ def run_cuda(args) -> dict:
     if not args.no_e2e:
         e2e = _end_to_end(torch, dist, rnd, grads, rule_b, K, world, dev, M, d, D32)
 
-    # ---- the other sizes and bucket lengths of the bandwidth sweep, then the model-shaped workloads (secondary)
+    # ---- the model-shaped workloads, then the other sizes and bucket lengths of the bandwidth sweep (secondary)
     other = None
     sweep = None
     if not (args.no_models and args.no_sweep):
         del grads
         rnd = None
         torch.cuda.empty_cache()
-    if not args.no_sweep:
-        sweep = [_sweep_point(torch, dq, Round, timer, m_, l_, bk_, K, dev, peak) for m_, l_, bk_ in SWEEP_POINTS]
     if not args.no_models:
         other = {}
         for w, gen_fn in ((workloads.config_resnet18(), _gen_resnet), (workloads.config_vgg16(), _gen_vgg),
                           (workloads.config_text(), _gen_text)):
             other[w.name] = _model_workload(torch, dq, Round, timer, w, gen_fn, dev, K, peak)
+    if not args.no_sweep:
+        sweep = [_sweep_point(torch, dq, Round, timer, m_, l_, bk_, K, dev, peak) for m_, l_, bk_ in SWEEP_POINTS]
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,

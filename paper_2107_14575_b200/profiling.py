@@ -266,13 +266,17 @@ def cmd_table(a) -> None:
                                                       pt["buffer_sets"], " | ".join(cells)))
     if line.get("model_workloads"):
         print("\n## Model-shaped workloads (Algorithm-1 order, dynamic b)\n")
-        print("| workload | MB/step | ms/step | GB/s of gradient | b first..last | fused ms (frac) | average ms (frac) |")
-        print("|---|---|---|---|---|---|---|")
+        print("`single` = one launch between its own pair of events (the bracket leaves the GPU idle for some microseconds "
+              "around the launch); `train` = launches back to back, rotating through three sets of buffers.\n")
+        print("| workload | MB/step | ms/step | GB/s of gradient | b first..last | fused single ms (frac) | fused train ms (frac) "
+              "| average single ms (frac) | average train ms (frac) |")
+        print("|---|---|---|---|---|---|---|---|---|")
         for name, w in line["model_workloads"].items():
-            print("| %s | %d | %.4f | %.0f | %s | %.4f (%.3f) | %.4f (%.3f) |" % (
+            f, v = w["norms_quantize_pack"], w["unpack_dequant_average"]
+            print("| %s | %d | %.4f | %.0f | %s | %.4f (%.3f) | %.4f (%.3f) | %.4f (%.3f) | %.4f (%.3f) |" % (
                 w["workload"], w["mb_per_step"], w["ms_per_step"], w["value"], w["bits_first_last"],
-                w["norms_quantize_pack"]["ms"], w["norms_quantize_pack"]["frac_of_measured"],
-                w["unpack_dequant_average"]["ms"], w["unpack_dequant_average"]["frac_of_measured"]))
+                f["ms"], f["frac_of_measured"], f.get("train_ms", float("nan")), f.get("train_frac_of_measured", float("nan")),
+                v["ms"], v["frac_of_measured"], v.get("train_ms", float("nan")), v.get("train_frac_of_measured", float("nan"))))
 
 
 def cmd_launches(a) -> None:
