@@ -530,6 +530,31 @@ def run_cuda(args) -> dict:
                          "peak_source": "SMs x 4 schedulers x 32 lanes x sampled SM clock (one warp instruction per "
                                         "scheduler and cycle); instructions per group from profiles/counters.json"})
 
+    # ---- the same step with the parameter update of Eq. 2 applied by the averaging kernel (x <- x - eta * average)
+    with_update = None
+    if not args.no_per_b:
+        x = torch.zeros(D32, dtype=torch.float32, device=dev)
+        evu = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(min(K, 8))]
+        for i in range(W):
+            rnd.step_fused(grads, rule_b(HEADLINE_B, i + 1), SEED, i, params=x, lr=1e-3)
+        torch.cuda.synchronize()
+        su, eu = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        su.record()
+        for i in range(K):
+            rnd.step_fused(grads, rule_b(HEADLINE_B, i + 1), SEED, i, params=x, lr=1e-3,
+                           events=evu[i] if i < len(evu) else None)
+        eu.record()
+        torch.cuda.synchronize()
+        assert rnd.read_status() == 0 and rnd.bits() == HEADLINE_B
+        t_u = sum(e[1].elapsed_time(e[2]) for e in evu) / len(evu)
+        bytes_u = (M * HEADLINE_B / 8.0 + 8.0) * D32            # the words of M workers, x read and written
+        with_update = {"ms_per_step": round(su.elapsed_time(eu) / K, 5),
+                       "value": round(4.0 * M * d * K / (su.elapsed_time(eu) * 1e-3) / 1e9, 1),
+                       "unpack_average_update": {"ms": round(t_u, 5), "algorithmic_bytes": bytes_u,
+                                                 "achieved_gbs": round(bytes_u / (t_u * 1e-3) / 1e9, 1),
+                                                 "frac_of_measured": round(bytes_u / (t_u * 1e-3) / 1e9 / peak, 4)}}
+        del x
+
     # ---- per b: the three hot kernels, trains of K launches and single event-bracketed launches
     per_b = {}
     n_single = min(K, 8)
@@ -601,7 +626,7 @@ def run_cuda(args) -> dict:
         # what the workers would put on the wire per step (Eq. 7: d * b bits per worker, plus the fp32 norms)
         "wire": {"bytes_per_step": M * (d * HEADLINE_B / 8.0 + 4.0 * L.nb), "fp32_bytes_per_step": 4.0 * M * d,
                  "ratio": round((d * HEADLINE_B / 8.0 + 4.0 * L.nb) / (4.0 * d), 4)},
-        "size_sweep": sweep, "model_workloads": other, "host_submit_ms_per_step": round(host_submit_ms, 5),
+        "with_parameter_update": with_update, "size_sweep": sweep, "model_workloads": other, "host_submit_ms_per_step": round(host_submit_ms, 5),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = _cpu_baseline(torch, gen, dev)

@@ -249,6 +249,13 @@ def cmd_table(a) -> None:
                                                                         k["single_launch_ms"],
                                                                         k["single_launch_frac_of_measured"]))
         print("| %s | %s | %.3f | %.0f |" % (b, " | ".join(cells), r["step_ms"], r["step_gradient_gbs"]))
+    if line.get("with_parameter_update"):
+        u = line["with_parameter_update"]
+        k = u["unpack_average_update"]
+        print("\nThe headline step with the parameter update of Eq. 2 applied by the averaging kernel: %.3f ms per step "
+              "(%.0f GB/s of gradient); the update kernel %.3f ms = %.0f GB/s of its algorithmic bytes "
+              "((M b/8 + 8) B per element), %.3f of the copy bandwidth." % (u["ms_per_step"], u["value"], k["ms"],
+                                                                          k["achieved_gbs"], k["frac_of_measured"]))
     if line.get("size_sweep"):
         print("\n## Other sizes and bucket lengths of the bandwidth sweep\n")
         print("Trains of launches; cases whose buffers would fit in the L2 rotate through `sets` sets of buffers.  "
