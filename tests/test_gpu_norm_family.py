@@ -68,7 +68,7 @@ def test_linf_nan_and_inf_reach_the_status_word(G):
 @pytest.mark.parametrize("bucket", [64, 96, 512, 2048, 4096])
 def test_linf_fused_norms_and_words_bit_exact(G, bucket, b):
     """dq_norms_quantize_pack on an l_inf layout: per-warp tile pipelines (64, 512), the
-    whole-bucket route (2048), warp pairs (4096) and the two-pass route of other bucket sizes (96)."""
+    teams of two warps (2048), teams of four warps (4096) and the two-pass route of other bucket sizes (96)."""
     segs = RAGGED + [5 * 4096 + 33]
     ref = oracle.Layout(segs, bucket)
     g = _grads(segs, 2, ref, 10 * bucket + b, pad_value=-3.25, scale=0.02)

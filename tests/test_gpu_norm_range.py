@@ -86,7 +86,7 @@ def test_l2_norms_of_tiny_and_huge_buckets(G, bucket):
 @pytest.mark.parametrize("b", [2, 4, 7, 12, 16])
 @pytest.mark.parametrize("bucket", BUCKETS)
 def test_fused_and_separate_words_with_the_gpus_own_norms(G, bucket, b):
-    """dq_norms_quantize_pack (per-warp tiles, whole-bucket warps, warp pairs, two-pass route) and
+    """dq_norms_quantize_pack (per-warp tiles, teams of two and of four warps, two-pass route) and
     dq_bucket_norms + dq_quantize_pack on the same inputs: same norms, and words equal to the
     oracle's when it is given those norms."""
     segs = RAGGED + [5 * 4096 + 33]

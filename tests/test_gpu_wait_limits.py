@@ -88,7 +88,7 @@ def test_quantizers_after_a_lost_first_wait(G, short_first_wait, bucket):
     st = _expect_wait_status_then_recover(
         G, r, lambda: r.quantize(SEED, 1), lambda got: np.testing.assert_array_equal(got[:, :nw], want))
     assert st & G.dq.STAT_WAIT
-    # fused norms + quantizer (per-warp tiles, whole-bucket warps, warp pairs)
+    # fused norms + quantizer (per-warp tiles, teams of two and of four warps)
     G.dq.debug_set_wait_limits(LIMIT_NS, True)
 
     def fused():
