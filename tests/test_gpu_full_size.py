@@ -130,6 +130,8 @@ def _device_normal(M, d, seed):
     (1 << 28, 1, 128, 1, 1 << 22),
     (1 << 26, 32, 512, 3, 1 << 20),
     (1 << 26, 32, 128, 8, 1 << 20),
+    (1 << 26, 32, 4096, 4, 1 << 20),          # teams of four warps per bucket
+    (1 << 26, 32, 2048, 5, 1 << 20),          # teams of two
 ])
 def test_sweep_sizes_prefix_parity_and_whole_array_properties(d, M, bucket, b, prefix):
     s = (1 << (b - 1)) - 1
