@@ -163,6 +163,22 @@ def test_sweep_sizes_prefix_parity_and_whole_array_properties(d, M, bucket, b, p
     rnd.norms_(g)
     assert torch.equal(rnd.norms, fused_norms)
 
+    # ---- whole array, M > 1: the average of the workers' Q(v) lies within the mean of their levels of the
+    #      mean gradient (every Q(v) within one level of its v), and is unbiased
+    if M > 1 and b > 1:
+        rnd.average_()
+        torch.cuda.synchronize()
+        assert rnd.read_status() == 0
+        q = rnd.out[:d]
+        mean_g = g.mean(dim=0)
+        step = (rnd.norms / s).mean(dim=0).repeat_interleave(bucket)[:d]
+        diff = q - mean_g
+        # (fp32 roundings of positions, products and of the two means: 4 ulp of s levels and 1e-5 absolute cover them)
+        assert bool((diff.abs() <= step * (1.0 + 4.0 * s * 2.0 ** -23) + 1e-5).all())
+        mean_err = float((diff / step).double().mean())
+        assert abs(mean_err) <= 5 * 0.5 / np.sqrt(float(M) * d) + 1e-6
+        del mean_g, step, diff
+
     # ---- whole array, M = 1 only (the average of one worker is Q(v) itself)
     if M == 1:
         rnd.average_()
