@@ -112,11 +112,12 @@ class ClockSampler:
 
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown"}
 
-    def __init__(self, uuid: str, period_s: float = 0.004):
+    def __init__(self, uuid: str, period_s: float = 0.002):
         self.uuid, self.period = uuid, period_s
         self.samples = []
         self.handle = None
         self._run = False
+        self._active = False
         try:
             import pynvml
             pynvml.nvmlInit()
@@ -137,25 +138,35 @@ class ClockSampler:
 
     def _loop(self):
         while self._run:
-            try:
-                self._one()
-            except Exception:
-                pass
+            if self._active:
+                try:
+                    self._one()
+                except Exception:
+                    pass
             time.sleep(self.period)
 
     def start(self):
+        """Opens a sampling window.  The thread is started once, ahead of the first window, and idles between
+        windows, so that a window of a few tens of milliseconds is sampled from its first period on."""
         if self.handle is None:
             return
+        if not self._run:
+            self._run = True
+            self._active = False
+            self.thread = threading.Thread(target=self._loop, daemon=True)
+            self.thread.start()
+            try:
+                self._one()                      # the first NVML queries of a process are the slow ones
+            except Exception:
+                pass
         self.samples = []
-        self._run = True
-        self.thread = threading.Thread(target=self._loop, daemon=True)
-        self.thread.start()
+        self._active = True
 
     def stop(self):
         if self.handle is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["NVML unavailable"]}
-        self._run = False
-        self.thread.join(timeout=2)
+        self._active = False
+        time.sleep(self.period)                  # a query in flight ends
         sm = [m for m, _ in self.samples]
         reasons = set()
         for _, mask in self.samples:
