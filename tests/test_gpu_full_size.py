@@ -128,6 +128,7 @@ def _device_normal(M, d, seed):
     (1 << 30, 1, 512, 4, 1 << 22),
     (1 << 30, 1, 4096, 16, 1 << 22),
     (1 << 28, 1, 128, 1, 1 << 22),
+    (1 << 28, 1, 4096, 6, 1 << 22),
     (1 << 26, 32, 512, 3, 1 << 20),
     (1 << 26, 32, 128, 8, 1 << 20),
     (1 << 26, 32, 4096, 4, 1 << 20),          # teams of four warps per bucket
@@ -153,6 +154,28 @@ def test_sweep_sizes_prefix_parity_and_whole_array_properties(d, M, bucket, b, p
     want_packed = oracle.quantize_pack(ref, gp, norms_p, b, SEED, 3)
     got = rnd.packed[:, : ref.packed_words(b)].cpu().numpy().view(np.uint32)
     assert np.array_equal(got, want_packed)
+    # ---- worker 0 over its whole length, word for word (every boundary between the ranges of the warps
+    #      and CTAs that share it, and its end), where the oracle takes a few seconds
+    if d <= (1 << 28):
+        ref0 = oracle.Layout([d], bucket)
+        g0 = g[:1].cpu().numpy()
+        norms0 = rnd.norms[:1].cpu().numpy()
+        np.testing.assert_allclose(norms0, oracle.bucket_norms(ref0, g0), rtol=NORM_RTOL, atol=0)
+        want0 = oracle.quantize_pack(ref0, g0, norms0, b, SEED, 3)
+        got0 = rnd.packed[:1, : ref0.packed_words(b)].cpu().numpy().view(np.uint32)
+        assert np.array_equal(got0, want0)
+        if M == 1 and b > 1:
+            # one worker: the whole average against the oracle, element by element (bound as in _full_round)
+            rnd.average_()
+            torch.cuda.synchronize()
+            assert rnd.read_status() == 0
+            want_avg = oracle.unpack_dequant_average(ref0, want0, norms0, b)
+            got_avg = rnd.out[:d].cpu().numpy().astype(np.float64)
+            bound = 1e-6 * np.repeat(norms0[0].astype(np.float64), bucket)[:d] + 2.0 ** -23 * np.abs(want_avg) + 1e-300
+            assert np.all(np.abs(got_avg - want_avg[:d]) <= bound)
+            del want_avg, got_avg, bound
+        del g0, want0, got0
+
     # nothing written past the words in use
     nw = L.packed_words(b)
     if rnd.packed_stride > nw:
