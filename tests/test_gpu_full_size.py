@@ -245,3 +245,47 @@ def test_bench_workload_full_size_with_parameter_update():
     avg = oracle.unpack_dequant_average(ref, packed, norms, b)
     tol = 1e-6 * lr * np.abs(avg).max() + 2.0 ** -23 * np.abs(want) + 1e-30
     assert np.all(np.abs(got.cpu().numpy().astype(np.float64) - want) <= tol)
+
+
+def test_bench_step_at_its_full_size_every_word_and_every_element():
+    """The bench's own workload and call -- d = 2^26, M = 32, bucket 512, b = 4, one step_fused -- against the
+    oracle over everything it writes: 4.2 M norms, 2^28 packed words bit for bit, 2^26 averaged elements each
+    within its bound, and the next bit width.  (About 20 GB of host memory and half a minute of the oracle.)"""
+    import psutil
+    if psutil.virtual_memory().available < (48 << 30):
+        pytest.skip("needs 48 GB of free host memory")
+    d, M, bucket, b = 1 << 26, 32, 512, 4
+    rnd = Round([d], bucket, M, max_bits=b)
+    g = _device_normal(M, d, seed=77)
+    rnd.packed.fill_(-1)
+    rnd.bits_(dq.Rule.fixed(b))
+    T, t_next = 100, 1
+    rnd.norms_(g)
+    G2 = float((rnd.norms.double() ** 2).sum().item() / M)
+    eps_hat = T * G2 / 6.5 ** 2                    # x = 6.5: half a level below s(4) = 7, so the rule stays at b = 4
+    out = rnd.step_fused(g, dq.Rule.dynamic(T, t_next, eps_hat, 1.0), SEED, 0)
+    torch.cuda.synchronize()
+    assert rnd.read_status() == 0
+
+    ref = oracle.Layout([d], bucket)
+    gh = g.cpu().numpy()
+    del g
+    norms = rnd.norms.cpu().numpy()
+    np.testing.assert_allclose(norms, oracle.bucket_norms(ref, gh), rtol=NORM_RTOL, atol=0)
+    want_packed = oracle.quantize_pack(ref, gh, norms, b, SEED, 0)
+    del gh
+    nw = ref.packed_words(b)
+    got_packed = rnd.packed[:, :nw].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got_packed, want_packed)
+    del got_packed
+    if rnd.packed_stride > nw:
+        assert bool((rnd.packed[:, nw:] == -1).all())
+    want_out = oracle.unpack_dequant_average(ref, want_packed, norms, b)
+    del want_packed
+    got_out = out[:d].cpu().numpy().astype(np.float64)
+    rel = np.linalg.norm(got_out - want_out[:d]) / np.linalg.norm(want_out[:d])
+    assert rel <= AVG_RTOL
+    bound = 1e-6 * np.repeat(norms.max(axis=0).astype(np.float64), bucket)[:d] + 2.0 ** -23 * np.abs(want_out[:d]) + 1e-300
+    assert np.all(np.abs(got_out - want_out[:d]) <= bound)
+    b_next, _, _ = oracle.choose_bits(norms, T, t_next, eps_hat, 1.0)
+    assert rnd.bits() == b_next == b
