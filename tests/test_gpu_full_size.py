@@ -185,6 +185,14 @@ def test_sweep_sizes_prefix_parity_and_whole_array_properties(d, M, bucket, b, p
     fused_norms = rnd.norms.clone()
     rnd.norms_(g)
     assert torch.equal(rnd.norms, fused_norms)
+    # ---- and the separate quantizer, given those norms, the same words
+    fused_packed = rnd.packed[:, :nw].clone()
+    rnd.packed.fill_(-1)
+    rnd.quantize_(g, SEED, 3)
+    torch.cuda.synchronize()
+    assert rnd.read_status() == 0
+    assert torch.equal(rnd.packed[:, :nw], fused_packed)
+    del fused_packed
 
     # ---- whole array, M > 1: the average of the workers' Q(v) lies within the mean of their levels of the
     #      mean gradient (every Q(v) within one level of its v), and is unbiased
